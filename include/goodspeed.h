@@ -1,0 +1,165 @@
+/*
+ * goodspeed.h -- C ABI of the GoodSpeed verification-server hot path for NVIDIA B200 (sm_100a).
+ *
+ * One verification round of the paper's Algorithm 1 (the verification-server steps:
+ * batching, verification, estimator update, GoodSpeed-sched) is four calls:
+ *
+ *   gs_verify_attn      target attention of every server's gamma_i+1 new positions   (Sec. II-A2)
+ *   gs_lm_head_logits   W h of  P_M = softmax(W h)                                   (Sec. II-A1)
+ *   gs_spec_accept      softmax, accept/reject, correction/bonus token, estimators   (Sec. II-A2,
+ *                                                          Eq. updatealpha, Eq. updateX, Sec. III-C)
+ *   gs_schedule         next allocation S(t+1), Eq. goodspeed_sched                  (Sec. III-C)
+ *
+ * Conventions common to all entry points
+ *   - Every tensor pointer is caller-owned DEVICE memory unless a parameter says "host".
+ *     The library never allocates, frees or synchronises; scratch comes from a caller
+ *     workspace whose size the matching *_workspace() query returns (bytes, 256-aligned base
+ *     required).  Workspace contents need not be initialised and are clobbered.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls enqueue work
+ *     and return; outputs are valid once the stream has reached that point.
+ *   - Return value: GS_OK or a synchronous argument error (nothing was launched).  Errors that
+ *     only the device can see (non-monotone offsets, token id outside [0,V)) are written to
+ *     *d_status (device int32; sticky: the first non-zero code stays; the caller zeroes it
+ *     and reads it after its own synchronisation).  d_status may be NULL.
+ *   - Ragged layout.  N servers; server i drafts gamma_i tokens and owns gamma_i+1 verify
+ *     positions.  cu_q[N+1] (int32, cu_q[0]=0) are the row offsets of those positions:
+ *     rows cu_q[i] .. cu_q[i+1]-1, T_q = cu_q[N].  Arrays with one entry per DRAFT token
+ *     (Gamma = T_q - N entries: q_probs rows, draft_tok, u_accept, ratio, p_tok, margin)
+ *     place server i at offset cu_q[i]-i.  Row cu_q[i]+j (j = 0..gamma_i) conditions on the
+ *     prefix plus draft tokens s_1..s_j, i.e. it is the target distribution p_{j+1}; row
+ *     cu_q[i]+gamma_i is the bonus distribution p_{gamma_i+1}.
+ */
+#ifndef GOODSPEED_H_
+#define GOODSPEED_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  GS_OK = 0,
+  GS_ERR_INVALID_ARG = 1, /* null pointer, negative size, misaligned pointer */
+  GS_ERR_SHAPE = 2,       /* sizes inconsistent with each other or with the offsets */
+  GS_ERR_UNSUPPORTED = 3, /* a shape or dtype this build has no kernel for */
+  GS_ERR_WORKSPACE = 4,   /* workspace missing or smaller than the query says */
+  GS_ERR_CUDA = 5,        /* a CUDA runtime/driver call failed (launch, tensor-map encode) */
+  GS_ERR_TIMEOUT = 6      /* a bounded device-side wait ran out (device status only) */
+} gs_status;
+
+typedef enum { GS_F32 = 0, GS_BF16 = 1 } gs_dtype;
+
+const char* gs_status_str(gs_status s);
+
+/* Library/ABI version (major*100 + minor). */
+int gs_version(void);
+
+/* --------------------------------------------------------------------------------------------
+ * gs_verify_attn -- Sec. II-A2: the target model scores all drafted positions of all servers
+ * in one parallel pass.  The paper gives no attention formula; this is scaled-dot-product
+ * attention with grouped KV heads, causal among the new positions, full view of the prefix.
+ *
+ *   Q  [T_q, Hq, hd]            queries of the new positions (rotary etc. already applied)
+ *   K,V[total_kv, Hkv, hd]      per-server caches, concatenated; server i owns rows
+ *                               cu_kv[i] .. cu_kv[i+1]-1 and its last gamma_i+1 rows are the
+ *                               new positions themselves (already appended by the caller)
+ *   O  [T_q, Hq, hd]            output, same dtype as Q
+ *   New position t (0-based) of server i attends to keys 0 .. L_i+t of that server, with
+ *   L_i = (cu_kv[i+1]-cu_kv[i]) - (gamma_i+1).  Query head h reads KV head h / (Hq/Hkv).
+ *   dt: GS_F32 (fp32 in/out) or GS_BF16 (bf16 in/out); scores, softmax and accumulation fp32.
+ *   max_kv_len: an upper bound on any server's cu_kv[i+1]-cu_kv[i] (sizes the split-KV scratch).
+ *   scale: multiplies q.k (pass 1/sqrt(hd)).
+ * Errors: INVALID_ARG (null/negative), SHAPE (Hq % Hkv != 0), UNSUPPORTED (hd > 256 for
+ * GS_F32; for GS_BF16 hd must be 64 or 128 and Hq/Hkv <= 16), WORKSPACE.
+ * Device status: GS_ERR_SHAPE if a server has fewer keys than new positions, more keys than
+ * max_kv_len, or offsets that decrease; that server's rows are then left unwritten.
+ */
+size_t gs_verify_attn_workspace(int N, int Tq, int total_kv, int max_kv_len, int Hq, int Hkv, int hd,
+                                gs_dtype dt);
+gs_status gs_verify_attn(const void* Q, const void* K, const void* V, void* O,
+                         const int32_t* cu_q, const int32_t* cu_kv,
+                         int N, int Tq, int total_kv, int max_kv_len, int Hq, int Hkv, int hd,
+                         float scale, gs_dtype dt,
+                         void* ws, size_t ws_bytes, int32_t* d_status, void* stream);
+
+/* --------------------------------------------------------------------------------------------
+ * gs_lm_head_logits -- Sec. II-A1: logits = W h for every verify position.
+ *
+ *   H      [T, d]   hidden states, row-major (d contiguous)
+ *   W      [d, V]   head weight, row-major (V contiguous)
+ *   logits [T, V]   fp32, row-major
+ *   logits[t, v] = sum_c H[t, c] * W[c, v], products exact, accumulation fp32.
+ *   dt: dtype of H and W.  GS_BF16 runs on the tensor cores (tcgen05, accumulators in tensor
+ *   memory) and needs d % 8 == 0, V % 8 == 0 and 16-byte aligned H, W; GS_F32 is a plain FMA
+ *   kernel meant for small problems.
+ * Errors: INVALID_ARG, UNSUPPORTED (alignment rules above), WORKSPACE, CUDA.
+ */
+size_t gs_lm_head_workspace(int T, int d, int V, gs_dtype dt);
+gs_status gs_lm_head_logits(const void* H, const void* W, float* logits, int T, int d, int V,
+                            gs_dtype dt, void* ws, size_t ws_bytes, int32_t* d_status, void* stream);
+
+/* --------------------------------------------------------------------------------------------
+ * gs_spec_accept -- Sec. II-A2 (acceptance rule, accepted count m, correction / bonus token),
+ * with the estimator updates of Sec. III-C fused at its tail (Eq. updatealpha, Eq. updateX).
+ *
+ *   logits   [T_q, V] fp32     target logits (rows as described at the top)
+ *   q_probs  [Gamma, V] fp32   draft distributions q_{i,j}
+ *   draft_tok[Gamma] int32     draft tokens s_{i,j}
+ *   u_accept [Gamma] fp32      the uniforms r_j of the acceptance test, in (0,1)
+ *   u_sample [N] fp32          one uniform per server for the correction / bonus draw
+ *   temperature                p_j = softmax(logits_j / temperature); 0 means greedy: p_j is the
+ *                              one-hot at the lowest-index argmax
+ * Outputs
+ *   accepted [N] int32         a_i = number of accepted draft tokens, 0 <= a_i <= gamma_i
+ *   out_tok  [T_q] int32       server i's segment: a_i accepted draft tokens, then the
+ *                              correction (a_i < gamma_i) or bonus token, then -1 padding
+ *   n_out    [N] int32         a_i + 1
+ *   ratio    [Gamma] fp32      min(1, p_j(s_j)/q_j(s_j)) for EVERY draft position
+ *   p_tok    [Gamma] fp32      p_j(s_j)
+ *   margin   [Gamma + N] fp32  nullable.  First Gamma: u_j - p_j(s_j)/q_j(s_j) (signed).  Last N:
+ *                              distance of the sampling threshold to the nearer edge of the
+ *                              emitted token's CDF interval, in units of the total mass.
+ * Rules: s_j is accepted iff u_j <= p_j(s_j)/q_j(s_j); q_j(s_j)=0 accepts iff p_j(s_j)>0;
+ * verification stops at the first rejection.  The last token is drawn by inverse CDF in
+ * ascending token id, smallest v whose cumulative mass exceeds u_sample * total, from
+ * max(0, p - q) at the rejected position, or from p of the bonus row; if max(0, p - q) has no
+ * mass the draw falls back to p.
+ * Estimators (alpha_hat, X: [N] fp64 in/out, both NULL to skip):
+ *   alpha_hat_i <- clamp((1-eta) alpha_hat_i + eta * mean_j ratio_j, alpha_min, alpha_max)
+ *                  (unchanged when gamma_i = 0);  X_i <- (1-beta) X_i + beta (a_i + 1).
+ * Errors: INVALID_ARG, SHAPE (T_q < N), WORKSPACE.  Device status: GS_ERR_SHAPE for decreasing
+ * offsets, GS_ERR_INVALID_ARG for a draft token outside [0, V) (it is then rejected).
+ */
+size_t gs_spec_accept_workspace(int N, int Tq, int V);
+gs_status gs_spec_accept(const float* logits, const float* q_probs, const int32_t* draft_tok,
+                         const int32_t* cu_q, const float* u_accept, const float* u_sample,
+                         float temperature, int N, int Tq, int V,
+                         int32_t* accepted, int32_t* out_tok, int32_t* n_out,
+                         float* ratio, float* p_tok, float* margin,
+                         double* alpha_hat, double* X, double eta, double beta,
+                         double alpha_min, double alpha_max,
+                         void* ws, size_t ws_bytes, int32_t* d_status, void* stream);
+
+/* --------------------------------------------------------------------------------------------
+ * gs_schedule -- GoodSpeed-sched (Eq. goodspeed_sched, Sec. III-C) with U_i = log:
+ *   maximise sum_i (1/X_i) (1 - alpha_hat_i^(S_i+1)) / (1 - alpha_hat_i)
+ *   subject to sum_i S_i <= C, s_min_i <= S_i <= s_max_i, S_i integer.
+ * Solved exactly by marginal allocation: the gain of raising S_i from s to s+1 is
+ * alpha_hat_i^(s+1)/X_i, decreasing in s; start at s_min and give the remaining budget one token
+ * at a time to the largest gain (lowest index on ties).  Gains are formed as alpha_hat_i/X_i
+ * followed by repeated fp64 multiplication by alpha_hat_i, so results are reproducible bit for bit.
+ *
+ *   X, alpha_hat [N] fp64 (device);  s_min, s_max [N] int32 nullable (0 and C);  S_out [N] int32.
+ * Errors: INVALID_ARG, UNSUPPORTED (N > 1024).  If sum s_min > C the floors are returned as they
+ * are and *d_status = GS_ERR_SHAPE.
+ */
+gs_status gs_schedule(const double* X, const double* alpha_hat, int N, int C,
+                      const int32_t* s_min, const int32_t* s_max, int32_t* S_out,
+                      int32_t* d_status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GOODSPEED_H_ */

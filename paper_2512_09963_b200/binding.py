@@ -1,0 +1,160 @@
+"""ctypes binding of libgoodspeed.so: same names as include/goodspeed.h, argument marshalling only.
+
+Every function takes torch tensors that already live on the CUDA device (or, where the header
+says "host", on the CPU), checks dtype/contiguity, and passes raw pointers plus the current CUDA
+stream.  No arithmetic of the verification path happens in Python.  If the shared library has
+not been built, the first call raises; there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libgoodspeed.so")
+GS_F32, GS_BF16 = 0, 1
+GS_OK = 0
+STATUS_NAMES = {0: "GS_OK", 1: "GS_ERR_INVALID_ARG", 2: "GS_ERR_SHAPE", 3: "GS_ERR_UNSUPPORTED",
+                4: "GS_ERR_WORKSPACE", 5: "GS_ERR_CUDA", 6: "GS_ERR_TIMEOUT"}
+
+_vp, _i, _f, _d, _sz = C.c_void_p, C.c_int, C.c_float, C.c_double, C.c_size_t
+
+# name -> (restype, argtypes); mirrors include/goodspeed.h
+SIGNATURES = {
+    "gs_status_str": (C.c_char_p, [_i]),
+    "gs_version": (_i, []),
+    "gs_verify_attn_workspace": (_sz, [_i, _i, _i, _i, _i, _i, _i, _i]),
+    "gs_verify_attn": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _i, _f, _i,
+                            _vp, _sz, _vp, _vp]),
+    "gs_lm_head_workspace": (_sz, [_i, _i, _i, _i]),
+    "gs_lm_head_logits": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _vp, _sz, _vp, _vp]),
+    "gs_spec_accept_workspace": (_sz, [_i, _i, _i]),
+    "gs_spec_accept": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _f, _i, _i, _i,
+                            _vp, _vp, _vp, _vp, _vp, _vp,
+                            _vp, _vp, _d, _d, _d, _d, _vp, _sz, _vp, _vp]),
+    "gs_schedule": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp]),
+}
+
+_lib = None
+
+
+class GoodSpeedError(RuntimeError):
+    def __init__(self, fn: str, code: int):
+        self.code = code
+        super().__init__(f"{fn} returned {STATUS_NAMES.get(code, code)}")
+
+
+def lib() -> C.CDLL:
+    """Loads the library (once).  Raises if it was not built: there is no other code path."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with "
+                               "`python -m paper_2512_09963_b200.build` (needs nvcc)")
+        L = C.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(L, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = L
+    return _lib
+
+
+def _ptr(t: Optional[torch.Tensor], dtype=None, cuda=True):
+    if t is None:
+        return None
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"expected {dtype}, got {t.dtype}")
+    if not t.is_contiguous():
+        raise ValueError("tensor must be contiguous")
+    if cuda and not t.is_cuda:
+        raise ValueError("tensor must be on the CUDA device")
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _check(fn: str, code: int):
+    if code != GS_OK:
+        raise GoodSpeedError(fn, code)
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return GS_F32
+    if t.dtype == torch.bfloat16:
+        return GS_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def gs_version() -> int:
+    return lib().gs_version()
+
+
+def gs_status_str(code: int) -> str:
+    return lib().gs_status_str(code).decode()
+
+
+def gs_verify_attn_workspace(N, Tq, total_kv, max_kv_len, Hq, Hkv, hd, dt) -> int:
+    return lib().gs_verify_attn_workspace(N, Tq, total_kv, max_kv_len, Hq, Hkv, hd, dt)
+
+
+def gs_verify_attn(Q, K, V, O, cu_q, cu_kv, max_kv_len, scale, ws, d_status=None):
+    Tq, Hq, hd = Q.shape
+    total_kv, Hkv, _ = K.shape
+    N = cu_q.numel() - 1
+    code = lib().gs_verify_attn(_ptr(Q), _ptr(K, Q.dtype), _ptr(V, Q.dtype), _ptr(O, Q.dtype),
+                                _ptr(cu_q, torch.int32), _ptr(cu_kv, torch.int32),
+                                N, Tq, total_kv, int(max_kv_len), Hq, Hkv, hd, float(scale), _dt(Q),
+                                _ptr(ws), ws.numel() * ws.element_size(), _ptr(d_status, torch.int32),
+                                _stream())
+    _check("gs_verify_attn", code)
+
+
+def gs_lm_head_workspace(T, d, V, dt) -> int:
+    return lib().gs_lm_head_workspace(T, d, V, dt)
+
+
+def gs_lm_head_logits(H, W, logits, ws, d_status=None):
+    T, d = H.shape
+    V = W.shape[1]
+    if W.shape[0] != d or tuple(logits.shape) != (T, V):
+        raise ValueError("shape mismatch")
+    code = lib().gs_lm_head_logits(_ptr(H), _ptr(W, H.dtype), _ptr(logits, torch.float32), T, d, V, _dt(H),
+                                   _ptr(ws), ws.numel() * ws.element_size(),
+                                   _ptr(d_status, torch.int32), _stream())
+    _check("gs_lm_head_logits", code)
+
+
+def gs_spec_accept_workspace(N, Tq, V) -> int:
+    return lib().gs_spec_accept_workspace(N, Tq, V)
+
+
+def gs_spec_accept(logits, q_probs, draft_tok, cu_q, u_accept, u_sample, temperature,
+                   accepted, out_tok, n_out, ratio, p_tok, margin=None,
+                   alpha_hat=None, X=None, eta=0.0, beta=0.0, alpha_min=1e-3, alpha_max=0.999,
+                   ws=None, d_status=None):
+    Tq, V = logits.shape
+    N = cu_q.numel() - 1
+    f32, i32, f64 = torch.float32, torch.int32, torch.float64
+    code = lib().gs_spec_accept(_ptr(logits, f32), _ptr(q_probs, f32), _ptr(draft_tok, i32), _ptr(cu_q, i32),
+                                _ptr(u_accept, f32), _ptr(u_sample, f32), float(temperature), N, Tq, V,
+                                _ptr(accepted, i32), _ptr(out_tok, i32), _ptr(n_out, i32),
+                                _ptr(ratio, f32), _ptr(p_tok, f32), _ptr(margin, f32),
+                                _ptr(alpha_hat, f64), _ptr(X, f64), float(eta), float(beta),
+                                float(alpha_min), float(alpha_max),
+                                _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
+                                _ptr(d_status, i32), _stream())
+    _check("gs_spec_accept", code)
+
+
+def gs_schedule(X, alpha_hat, C_budget, S_out, s_min=None, s_max=None, d_status=None):
+    N = X.numel()
+    i32, f64 = torch.int32, torch.float64
+    code = lib().gs_schedule(_ptr(X, f64), _ptr(alpha_hat, f64), N, int(C_budget), _ptr(s_min, i32),
+                             _ptr(s_max, i32), _ptr(S_out, i32), _ptr(d_status, i32), _stream())
+    _check("gs_schedule", code)

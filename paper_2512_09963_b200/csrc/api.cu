@@ -1,0 +1,16 @@
+#include "common.cuh"
+
+extern "C" const char* gs_status_str(gs_status s) {
+  switch (s) {
+    case GS_OK: return "ok";
+    case GS_ERR_INVALID_ARG: return "invalid argument";
+    case GS_ERR_SHAPE: return "inconsistent shape or offsets";
+    case GS_ERR_UNSUPPORTED: return "unsupported shape or dtype";
+    case GS_ERR_WORKSPACE: return "workspace missing or too small";
+    case GS_ERR_CUDA: return "CUDA call failed";
+    case GS_ERR_TIMEOUT: return "bounded device wait ran out";
+  }
+  return "unknown status";
+}
+
+extern "C" int gs_version(void) { return 100; }

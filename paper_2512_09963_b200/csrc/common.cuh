@@ -1,0 +1,96 @@
+// Shared device/host helpers of the GoodSpeed CUDA library (sm_100a only).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <float.h>
+#include <limits.h>
+
+#include "../../include/goodspeed.h"
+
+#define GS_DEVINL __device__ __forceinline__
+
+namespace gs {
+
+constexpr int kNumSMsFallback = 148;
+
+// Sticky device status: the first non-zero code wins.
+GS_DEVINL void set_status(int32_t* st, int code) {
+  if (st != nullptr) atomicCAS(st, 0, code);
+}
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+inline gs_status launch_status() {
+  return cudaGetLastError() == cudaSuccess ? GS_OK : GS_ERR_CUDA;
+}
+
+inline int sm_count() {
+  static int cached = 0;
+  if (cached == 0) {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+      cached = n;
+    else
+      cached = kNumSMsFallback;
+  }
+  return cached;
+}
+
+// 2^x by the special-function unit (relative error about 2 ulp); 2^-inf = 0.
+GS_DEVINL float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+GS_DEVINL double shfl_xor_f64(double v, int mask) {
+  int lo = __double2loint(v), hi = __double2hiint(v);
+  lo = __shfl_xor_sync(0xffffffffu, lo, mask);
+  hi = __shfl_xor_sync(0xffffffffu, hi, mask);
+  return __hiloint2double(hi, lo);
+}
+
+GS_DEVINL double shfl_up_f64(double v, int delta) {
+  int lo = __double2loint(v), hi = __double2hiint(v);
+  lo = __shfl_up_sync(0xffffffffu, lo, delta);
+  hi = __shfl_up_sync(0xffffffffu, hi, delta);
+  return __hiloint2double(hi, lo);
+}
+
+// Butterfly sum: every lane ends with the same value, order fixed by the lane ids.
+GS_DEVINL double warp_sum_f64(double v) {
+#pragma unroll
+  for (int m = 16; m > 0; m >>= 1) v += shfl_xor_f64(v, m);
+  return v;
+}
+
+GS_DEVINL float warp_sum_f32(float v) {
+#pragma unroll
+  for (int m = 16; m > 0; m >>= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
+  return v;
+}
+
+GS_DEVINL float warp_max_f32(float v) {
+#pragma unroll
+  for (int m = 16; m > 0; m >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, m));
+  return v;
+}
+
+// (value, index) maximum with the lowest index winning ties.
+GS_DEVINL void argmax_merge(float& m, int& a, float m2, int a2) {
+  if (m2 > m || (m2 == m && a2 < a)) { m = m2; a = a2; }
+}
+
+GS_DEVINL void warp_argmax(float& m, int& a) {
+#pragma unroll
+  for (int k = 16; k > 0; k >>= 1) {
+    float m2 = __shfl_xor_sync(0xffffffffu, m, k);
+    int a2 = __shfl_xor_sync(0xffffffffu, a, k);
+    argmax_merge(m, a, m2, a2);
+  }
+}
+
+}  // namespace gs

@@ -1,0 +1,477 @@
+// gs_spec_accept: temperature softmax statistics, sequential accept/reject, correction or bonus
+// token by inverse CDF, and the estimator updates (Sec. II-A2; Eq. updatealpha, Eq. updateX).
+//
+// Four launches on one stream:
+//   1. sa_row_stats   every logit row is cut into chunks of 4096 floats; one CTA per (chunk,row)
+//                     streams its chunk once with 16-byte loads and writes (max, argmax, sum exp).
+//   2. sa_decide      one CTA per server merges the chunk statistics of its rows in chunk order,
+//                     evaluates p(s_j), q(s_j), the ratios, the accepted count, the estimators,
+//                     and selects the one row the last token is drawn from.
+//   3. sa_mass        one CTA per (chunk, server) sums the mass of the selected row's chunk:
+//                     max(0, p - q) after a rejection, p for the bonus row.
+//   4. sa_sample      one CTA per server scans the chunk masses in order, finds the chunk that
+//                     holds u * total, and does an ordered prefix scan inside that chunk.
+// Only one row per server is read a second time.  All cross-thread sums are fp64 in a fixed
+// order, so two runs give identical bits.
+#include "common.cuh"
+
+namespace gs {
+
+constexpr int kSaThreads = 256;
+constexpr int kSaChunk = 4096;                   // floats per CTA
+constexpr int kSaPerThread = kSaChunk / kSaThreads;  // 16
+constexpr float kLog2e = 1.4426950408889634f;
+
+struct ChunkStat {   // 16 bytes
+  float m;
+  int arg;
+  double z;
+};
+
+struct ServerSel {   // what sa_mass / sa_sample need about a server
+  int row;           // logits row the last token is drawn from
+  int qrow;          // q_probs row to subtract, or -1 for the bonus row
+  float M;           // row max
+  int arg;           // row argmax
+  double invZ;       // 1 / sum exp
+  int valid;
+  int pad;
+};
+
+struct SaWorkspace {
+  ChunkStat* stats;   // [Tq * n_chunk]
+  ServerSel* sel;     // [N]
+  double* mass;       // [N * n_chunk]
+};
+
+static size_t sa_layout(int N, int Tq, int V, SaWorkspace* w, char* base) {
+  size_t n_chunk = (size_t)(V + kSaChunk - 1) / kSaChunk;
+  size_t off = 0;
+  size_t stats = off; off = align_up(off + sizeof(ChunkStat) * n_chunk * (size_t)Tq, 256);
+  size_t sel = off;   off = align_up(off + sizeof(ServerSel) * (size_t)N, 256);
+  size_t mass = off;  off = align_up(off + sizeof(double) * n_chunk * (size_t)N, 256);
+  if (w != nullptr) {
+    w->stats = reinterpret_cast<ChunkStat*>(base + stats);
+    w->sel = reinterpret_cast<ServerSel*>(base + sel);
+    w->mass = reinterpret_cast<double*>(base + mass);
+  }
+  return off;
+}
+
+// Loads the 16 floats a thread owns in a chunk: element (k*256 + tid)*4 + j, k,j in 0..3.
+// Out-of-range elements read as -inf.
+template <bool VEC>
+GS_DEVINL void load_chunk(const float* __restrict__ row, int base, int V, int tid, float (&v)[kSaPerThread]) {
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    int idx = base + (k * kSaThreads + tid) * 4;
+    if (VEC && idx + 3 < V) {
+      float4 t = __ldg(reinterpret_cast<const float4*>(row + idx));
+      v[4 * k + 0] = t.x; v[4 * k + 1] = t.y; v[4 * k + 2] = t.z; v[4 * k + 3] = t.w;
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) v[4 * k + j] = (idx + j < V) ? __ldg(row + idx + j) : -INFINITY;
+    }
+  }
+}
+
+GS_DEVINL int chunk_elem_index(int base, int tid, int e) {
+  return base + ((e >> 2) * kSaThreads + tid) * 4 + (e & 3);
+}
+
+// Fixed-order block sum of one double per thread (256 threads): butterfly inside a warp,
+// then warp 0..7 added in order by thread 0.  Result valid in thread 0.
+GS_DEVINL double block_sum_f64(double v, double* smem8) {
+  v = warp_sum_f64(v);
+  int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  if (lane == 0) smem8[wid] = v;
+  __syncthreads();
+  double s = 0.0;
+  if (threadIdx.x == 0) {
+#pragma unroll
+    for (int w = 0; w < kSaThreads / 32; ++w) s += smem8[w];
+  }
+  return s;
+}
+
+template <bool VEC>
+__global__ void __launch_bounds__(kSaThreads)
+sa_row_stats(const float* __restrict__ logits, int V, int n_chunk, float k2, ChunkStat* __restrict__ stats) {
+  __shared__ float s_m[kSaThreads / 32];
+  __shared__ int s_a[kSaThreads / 32];
+  __shared__ double s_z[kSaThreads / 32];
+  __shared__ float s_bm;
+  const int tid = threadIdx.x, c = blockIdx.x, r = blockIdx.y;
+  const float* row = logits + (size_t)r * V;
+  const int base = c * kSaChunk;
+  float v[kSaPerThread];
+  load_chunk<VEC>(row, base, V, tid, v);
+
+  float m = -INFINITY;
+  int a = INT_MAX;
+#pragma unroll
+  for (int e = 0; e < kSaPerThread; ++e) {
+    if (v[e] > m) { m = v[e]; a = chunk_elem_index(base, tid, e); }
+  }
+  warp_argmax(m, a);
+  if ((tid & 31) == 0) { s_m[tid >> 5] = m; s_a[tid >> 5] = a; }
+  __syncthreads();
+  if (tid == 0) {
+    float bm = s_m[0]; int ba = s_a[0];
+#pragma unroll
+    for (int w = 1; w < kSaThreads / 32; ++w) argmax_merge(bm, ba, s_m[w], s_a[w]);
+    s_bm = bm; s_a[0] = ba;
+  }
+  __syncthreads();
+  const float bm = s_bm;
+  float z = 0.f;
+  if (k2 > 0.f && bm > -INFINITY) {
+#pragma unroll
+    for (int e = 0; e < kSaPerThread; ++e) z += fast_exp2((v[e] - bm) * k2);
+  }
+  double zs = block_sum_f64((double)z, s_z);
+  if (tid == 0) {
+    ChunkStat st;
+    st.m = bm; st.arg = (s_a[0] == INT_MAX) ? base : s_a[0]; st.z = zs;
+    stats[(size_t)r * n_chunk + c] = st;
+  }
+}
+
+struct SaDecideArgs {
+  const float* logits; const float* q_probs; const int32_t* draft_tok; const int32_t* cu_q;
+  const float* u_accept;
+  int N, Tq, V, n_chunk;
+  float tau;
+  int32_t* accepted; int32_t* out_tok; int32_t* n_out;
+  float* ratio; float* p_tok; float* margin;
+  double* alpha_hat; double* X; double eta, beta, alpha_min, alpha_max;
+  const ChunkStat* stats; ServerSel* sel;
+  int32_t* d_status;
+};
+
+constexpr int kDecideThreads = 128;
+
+// Merges the chunk statistics of row r in chunk order.
+GS_DEVINL void merge_row(const ChunkStat* __restrict__ st, int n_chunk, float tau, float& M, int& arg, double& Z) {
+  M = st[0].m; arg = st[0].arg;
+  for (int c = 1; c < n_chunk; ++c) argmax_merge(M, arg, st[c].m, st[c].arg);
+  Z = 0.0;
+  if (tau > 0.f) {
+    const double inv_tau = 1.0 / (double)tau;
+    for (int c = 0; c < n_chunk; ++c) {
+      if (st[c].m > -INFINITY) Z += st[c].z * exp(((double)st[c].m - (double)M) * inv_tau);
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kDecideThreads) sa_decide(SaDecideArgs A) {
+  extern __shared__ unsigned char smem_raw[];
+  const int i = blockIdx.x, tid = threadIdx.x;
+  const int r0 = A.cu_q[i], r1 = A.cu_q[i + 1];
+  const int gamma = r1 - r0 - 1;
+  if (r0 < 0 || gamma < 0 || r1 > A.Tq) {
+    if (tid == 0) {
+      set_status(A.d_status, GS_ERR_SHAPE);
+      A.sel[i].valid = 0;
+      A.accepted[i] = 0; A.n_out[i] = 0;
+    }
+    return;
+  }
+  const int g0 = r0 - i;
+  // per-row merged statistics, rows j = 0..gamma
+  float* sM = reinterpret_cast<float*>(smem_raw);                // [gamma+1]
+  int* sArg = reinterpret_cast<int*>(sM + (gamma + 1));          // [gamma+1]
+  int* sRej = sArg + (gamma + 1);                                // [gamma+1] 1 = would be rejected
+  size_t off = (size_t)(3 * (gamma + 1)) * 4;
+  off = (off + 7) / 8 * 8;
+  double* sZ = reinterpret_cast<double*>(smem_raw + off);        // [gamma+1]
+  double* sRatio = sZ + (gamma + 1);                             // [gamma+1] clipped ratios
+
+  for (int j = tid; j <= gamma; j += kDecideThreads) {
+    float M; int arg; double Z;
+    merge_row(A.stats + (size_t)(r0 + j) * A.n_chunk, A.n_chunk, A.tau, M, arg, Z);
+    sM[j] = M; sArg[j] = arg; sZ[j] = Z;
+    if (j < gamma) {
+      const int s = A.draft_tok[g0 + j];
+      double p = 0.0, q = 0.0, rho = 0.0;
+      if (s < 0 || s >= A.V) {
+        set_status(A.d_status, GS_ERR_INVALID_ARG);
+      } else {
+        const float l = A.logits[(size_t)(r0 + j) * A.V + s];
+        if (A.tau > 0.f) p = (Z > 0.0) ? exp(((double)l - (double)M) / (double)A.tau) / Z : 0.0;
+        else p = (s == arg) ? 1.0 : 0.0;
+        q = (double)A.q_probs[(size_t)(g0 + j) * A.V + s];
+        if (q > 0.0) rho = p / q;
+        else rho = (p > 0.0) ? (double)INFINITY : 0.0;
+      }
+      const double u = (double)A.u_accept[g0 + j];
+      sRej[j] = (u > rho) ? 1 : 0;
+      const double clipped = rho < 1.0 ? rho : 1.0;
+      sRatio[j] = clipped;
+      A.ratio[g0 + j] = (float)clipped;
+      A.p_tok[g0 + j] = (float)p;
+      if (A.margin != nullptr) A.margin[g0 + j] = (float)(u - rho);
+    }
+  }
+  __syncthreads();
+  __shared__ int s_acc;
+  if (tid == 0) {
+    int a = gamma;
+    for (int j = 0; j < gamma; ++j) {
+      if (sRej[j]) { a = j; break; }
+    }
+    s_acc = a;
+    A.accepted[i] = a;
+    A.n_out[i] = a + 1;
+    ServerSel sel;
+    sel.row = r0 + a;
+    sel.qrow = (a < gamma) ? (g0 + a) : -1;
+    sel.M = sM[a]; sel.arg = sArg[a];
+    sel.invZ = (sZ[a] > 0.0) ? 1.0 / sZ[a] : 0.0;
+    sel.valid = 1; sel.pad = 0;
+    A.sel[i] = sel;
+    if (A.alpha_hat != nullptr && A.X != nullptr) {
+      if (gamma > 0) {
+        double sum = 0.0;
+        for (int j = 0; j < gamma; ++j) sum += sRatio[j];
+        const double obs = sum / (double)gamma;
+        double ah = (1.0 - A.eta) * A.alpha_hat[i] + A.eta * obs;
+        ah = ah < A.alpha_min ? A.alpha_min : ah;
+        ah = ah > A.alpha_max ? A.alpha_max : ah;
+        A.alpha_hat[i] = ah;
+      }
+      A.X[i] = (1.0 - A.beta) * A.X[i] + A.beta * (double)(a + 1);
+    }
+  }
+  __syncthreads();
+  const int a = s_acc;
+  for (int j = tid; j <= gamma; j += kDecideThreads)
+    A.out_tok[r0 + j] = (j < a) ? A.draft_tok[g0 + j] : -1;
+}
+
+// Mass of element v of the selected row: max(0, p - q) or p, in fp64 from an fp32 exponential.
+GS_DEVINL double elem_mass(float l, float M, float k2, double invZ, bool resid, float q) {
+  double p = (double)fast_exp2((l - M) * k2) * invZ;
+  if (resid) { p -= (double)q; p = p > 0.0 ? p : 0.0; }
+  return p;
+}
+
+template <bool VEC>
+__global__ void __launch_bounds__(kSaThreads)
+sa_mass(const float* __restrict__ logits, const float* __restrict__ q_probs, int V, int n_chunk, float k2,
+        const ServerSel* __restrict__ sel, double* __restrict__ mass) {
+  __shared__ double s_z[kSaThreads / 32];
+  const int tid = threadIdx.x, c = blockIdx.x, i = blockIdx.y;
+  const ServerSel s = sel[i];
+  if (!s.valid) return;
+  const int base = c * kSaChunk;
+  float l[kSaPerThread], q[kSaPerThread];
+  load_chunk<VEC>(logits + (size_t)s.row * V, base, V, tid, l);
+  const bool resid = s.qrow >= 0;
+  if (resid) load_chunk<VEC>(q_probs + (size_t)s.qrow * V, base, V, tid, q);
+  double acc = 0.0;
+#pragma unroll
+  for (int e = 0; e < kSaPerThread; ++e) acc += elem_mass(l[e], s.M, k2, s.invZ, resid, resid ? q[e] : 0.f);
+  double tot = block_sum_f64(acc, s_z);
+  if (tid == 0) mass[(size_t)i * n_chunk + c] = tot;
+}
+
+struct SaSampleArgs {
+  const float* logits; const float* q_probs; const float* u_sample; const int32_t* cu_q;
+  int N, V, n_chunk, Gamma;
+  float k2;
+  const ServerSel* sel; const double* mass;
+  int32_t* out_tok; float* margin;
+};
+
+// Ordered scan of one chunk: thread t owns the 16 consecutive elements base + 16 t .. +15.
+// Returns through s_tok the smallest index whose inclusive prefix (offset by `before`) exceeds
+// thr, or INT_MAX; s_last = largest index with positive mass.
+GS_DEVINL void scan_chunk(const float* __restrict__ lrow, const float* __restrict__ qrow, int base, int V,
+                          float M, float k2, double invZ, double before, double thr,
+                          int* s_tok, int* s_last, double* s_lo, double* s_hi, double* s_warp) {
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const int first = base + tid * kSaPerThread;
+  double w[kSaPerThread];
+  double run = 0.0;
+  int last_pos = -1;
+#pragma unroll
+  for (int e = 0; e < kSaPerThread; ++e) {
+    const int idx = first + e;
+    double x = 0.0;
+    if (idx < V) x = elem_mass(lrow[idx], M, k2, invZ, qrow != nullptr, qrow != nullptr ? qrow[idx] : 0.f);
+    if (x > 0.0) last_pos = idx;
+    run += x;
+    w[e] = run;   // inclusive prefix inside the thread
+  }
+  // exclusive scan of the thread totals: inside warps by shuffles, across warps by thread order
+  double incl = run;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    double t = shfl_up_f64(incl, d);
+    if (lane >= d) incl += t;
+  }
+  if (lane == 31) s_warp[wid] = incl;
+  __syncthreads();
+  double woff = 0.0;
+  for (int k = 0; k < wid; ++k) woff += s_warp[k];
+  const double excl = before + woff + (incl - run);
+  int found = INT_MAX;
+  double lo = 0.0, hi = 0.0;
+#pragma unroll
+  for (int e = 0; e < kSaPerThread; ++e) {
+    const int idx = first + e;
+    if (found == INT_MAX && idx < V && excl + w[e] > thr) {
+      found = idx;
+      hi = excl + w[e];
+      lo = excl + (e > 0 ? w[e - 1] : 0.0);
+    }
+  }
+  if (found != INT_MAX) atomicMin(s_tok, found);
+  if (last_pos >= 0) atomicMax(s_last, last_pos);
+  __syncthreads();
+  if (found != INT_MAX && *s_tok == found) { *s_lo = lo; *s_hi = hi; }
+  __syncthreads();
+}
+
+__global__ void __launch_bounds__(kSaThreads) sa_sample(SaSampleArgs A) {
+  __shared__ int s_chunk, s_tok, s_last;
+  __shared__ double s_before, s_thr, s_total, s_lo, s_hi;
+  __shared__ double s_warp[kSaThreads / 32];
+  const int i = blockIdx.x, tid = threadIdx.x;
+  const ServerSel s = A.sel[i];
+  if (!s.valid) return;
+  if (A.k2 <= 0.f) {   // greedy target: the one-hot (and its residual) sits on the argmax
+    if (tid == 0) {
+      A.out_tok[s.row] = s.arg;
+      if (A.margin != nullptr) A.margin[A.Gamma + i] = 1.0f;
+    }
+    return;
+  }
+  const float* lrow = A.logits + (size_t)s.row * A.V;
+  const float* qrow = s.qrow >= 0 ? A.q_probs + (size_t)s.qrow * A.V : nullptr;
+  const double u = (double)A.u_sample[i];
+  if (tid == 0) {
+    const double* m = A.mass + (size_t)i * A.n_chunk;
+    double total = 0.0;
+    for (int c = 0; c < A.n_chunk; ++c) total += m[c];
+    const double thr = u * total;
+    double run = 0.0, before = 0.0;
+    int pick = -1, last_pos = -1;
+    for (int c = 0; c < A.n_chunk; ++c) {
+      if (m[c] > 0.0) last_pos = c;
+      if (run + m[c] > thr) { pick = c; before = run; break; }
+      run += m[c];
+    }
+    if (pick < 0 && last_pos >= 0) {   // rounding left no chunk: last chunk that has mass
+      pick = last_pos;
+      before = 0.0;
+      for (int c = 0; c < pick; ++c) before += m[c];
+    }
+    s_chunk = pick; s_before = before; s_thr = thr; s_total = total;
+    s_tok = INT_MAX; s_last = -1; s_lo = 0.0; s_hi = 0.0;
+  }
+  __syncthreads();
+  if (s_chunk >= 0) {
+    scan_chunk(lrow, qrow, s_chunk * kSaChunk, A.V, s.M, A.k2, s.invZ, s_before, s_thr,
+               &s_tok, &s_last, &s_lo, &s_hi, s_warp);
+  } else {
+    // max(0, p - q) has no mass at all: draw from p itself, scanning the whole row in order.
+    qrow = nullptr;
+    double before = 0.0;   // total of p is 1 by construction of invZ
+    const double thr = u;
+    if (tid == 0) { s_thr = thr; s_total = 1.0; }
+    for (int c = 0; c < A.n_chunk; ++c) {
+      __syncthreads();
+      if (tid == 0) s_before = before;
+      __syncthreads();
+      scan_chunk(lrow, nullptr, c * kSaChunk, A.V, s.M, A.k2, s.invZ, s_before, thr,
+                 &s_tok, &s_last, &s_lo, &s_hi, s_warp);
+      if (s_tok != INT_MAX) break;
+      // advance `before` by this chunk's mass (recomputed in the same order by every thread 0)
+      double part = 0.0;
+      for (int k = 0; k < kSaThreads / 32; ++k) part += s_warp[k];
+      before += part;
+    }
+  }
+  if (tid == 0) {
+    int tok = s_tok;
+    float marg = 0.f;
+    if (tok == INT_MAX) {
+      tok = s_last >= 0 ? s_last : s.arg;
+    } else if (s_total > 0.0) {
+      const double a = s_thr - s_lo, b = s_hi - s_thr;
+      marg = (float)((a < b ? a : b) / s_total);
+    }
+    A.out_tok[s.row] = tok;
+    if (A.margin != nullptr) A.margin[A.Gamma + i] = marg;
+  }
+}
+
+}  // namespace gs
+
+extern "C" size_t gs_spec_accept_workspace(int N, int Tq, int V) {
+  if (N <= 0 || Tq <= 0 || V <= 0) return 256;
+  return gs::sa_layout(N, Tq, V, nullptr, nullptr);
+}
+
+extern "C" gs_status gs_spec_accept(const float* logits, const float* q_probs, const int32_t* draft_tok,
+                                    const int32_t* cu_q, const float* u_accept, const float* u_sample,
+                                    float temperature, int N, int Tq, int V,
+                                    int32_t* accepted, int32_t* out_tok, int32_t* n_out,
+                                    float* ratio, float* p_tok, float* margin,
+                                    double* alpha_hat, double* X, double eta, double beta,
+                                    double alpha_min, double alpha_max,
+                                    void* ws, size_t ws_bytes, int32_t* d_status, void* stream) {
+  using namespace gs;
+  if (N < 0 || Tq < 0 || V < 0 || !(temperature >= 0.f)) return GS_ERR_INVALID_ARG;
+  if (N == 0) return GS_OK;
+  if (Tq < N) return GS_ERR_SHAPE;
+  if (V == 0) return GS_ERR_SHAPE;
+  const int Gamma = Tq - N;
+  if (!logits || !cu_q || !u_sample || !accepted || !out_tok || !n_out) return GS_ERR_INVALID_ARG;
+  if (Gamma > 0 && (!q_probs || !draft_tok || !u_accept || !ratio || !p_tok)) return GS_ERR_INVALID_ARG;
+  if ((alpha_hat == nullptr) != (X == nullptr)) return GS_ERR_INVALID_ARG;
+  if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return GS_ERR_WORKSPACE;
+  if (ws_bytes < gs_spec_accept_workspace(N, Tq, V)) return GS_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  SaWorkspace w;
+  sa_layout(N, Tq, V, &w, static_cast<char*>(ws));
+  const int n_chunk = (V + kSaChunk - 1) / kSaChunk;
+  const float k2 = temperature > 0.f ? kLog2e / temperature : 0.f;
+  const bool vec = (V % 4 == 0) && (reinterpret_cast<uintptr_t>(logits) % 16 == 0) &&
+                   (q_probs == nullptr || reinterpret_cast<uintptr_t>(q_probs) % 16 == 0);
+
+  dim3 g1(n_chunk, Tq);
+  if (vec) sa_row_stats<true><<<g1, kSaThreads, 0, st>>>(logits, V, n_chunk, k2, w.stats);
+  else sa_row_stats<false><<<g1, kSaThreads, 0, st>>>(logits, V, n_chunk, k2, w.stats);
+
+  SaDecideArgs A;
+  A.logits = logits; A.q_probs = q_probs; A.draft_tok = draft_tok; A.cu_q = cu_q; A.u_accept = u_accept;
+  A.N = N; A.Tq = Tq; A.V = V; A.n_chunk = n_chunk; A.tau = temperature;
+  A.accepted = accepted; A.out_tok = out_tok; A.n_out = n_out;
+  A.ratio = ratio; A.p_tok = p_tok; A.margin = margin;
+  A.alpha_hat = alpha_hat; A.X = X; A.eta = eta; A.beta = beta; A.alpha_min = alpha_min; A.alpha_max = alpha_max;
+  A.stats = w.stats; A.sel = w.sel; A.d_status = d_status;
+  // rows of one server are bounded by Tq - (N-1); size the dynamic shared memory for that
+  const size_t max_rows = (size_t)(Tq - N + 1);
+  const size_t smem = align_up(3 * max_rows * 4, 8) + 2 * max_rows * 8;
+  if (smem > 200 * 1024) return GS_ERR_UNSUPPORTED;
+  if (smem > 48 * 1024) {
+    if (cudaFuncSetAttribute(sa_decide, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return GS_ERR_CUDA;
+  }
+  sa_decide<<<N, kDecideThreads, smem, st>>>(A);
+
+  if (k2 > 0.f) {
+    dim3 g3(n_chunk, N);
+    if (vec) sa_mass<true><<<g3, kSaThreads, 0, st>>>(logits, q_probs, V, n_chunk, k2, w.sel, w.mass);
+    else sa_mass<false><<<g3, kSaThreads, 0, st>>>(logits, q_probs, V, n_chunk, k2, w.sel, w.mass);
+  }
+  SaSampleArgs S;
+  S.logits = logits; S.q_probs = q_probs; S.u_sample = u_sample; S.cu_q = cu_q;
+  S.N = N; S.V = V; S.n_chunk = n_chunk; S.Gamma = Gamma; S.k2 = k2;
+  S.sel = w.sel; S.mass = w.mass; S.out_tok = out_tok; S.margin = margin;
+  sa_sample<<<N, kSaThreads, 0, st>>>(S);
+  return launch_status();
+}

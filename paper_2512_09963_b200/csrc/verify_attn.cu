@@ -1,0 +1,33 @@
+// gs_verify_attn: dispatch between the tensor-core split-KV kernel (bf16) and the plain kernel.
+#include "common.cuh"
+#include "attn_generic.cuh"
+
+extern "C" size_t gs_verify_attn_workspace(int N, int Tq, int total_kv, int max_kv_len, int Hq, int Hkv,
+                                           int hd, gs_dtype dt) {
+  (void)N; (void)Tq; (void)total_kv; (void)max_kv_len; (void)Hq; (void)Hkv; (void)hd; (void)dt;
+  return 256;
+}
+
+extern "C" gs_status gs_verify_attn(const void* Q, const void* K, const void* V, void* O,
+                                    const int32_t* cu_q, const int32_t* cu_kv,
+                                    int N, int Tq, int total_kv, int max_kv_len, int Hq, int Hkv, int hd,
+                                    float scale, gs_dtype dt,
+                                    void* ws, size_t ws_bytes, int32_t* d_status, void* stream) {
+  using namespace gs;
+  if (N < 0 || Tq < 0 || total_kv < 0 || max_kv_len < 0 || Hq <= 0 || Hkv <= 0 || hd <= 0)
+    return GS_ERR_INVALID_ARG;
+  if (dt != GS_F32 && dt != GS_BF16) return GS_ERR_INVALID_ARG;
+  if (N == 0 || Tq == 0) return GS_OK;
+  if (!Q || !K || !V || !O || !cu_q || !cu_kv) return GS_ERR_INVALID_ARG;
+  if (Hq % Hkv != 0) return GS_ERR_SHAPE;
+  if (hd > 32 * kGenAttnMaxPerLane) return GS_ERR_UNSUPPORTED;
+  if (Tq > 65535) return GS_ERR_UNSUPPORTED;
+  if (ws == nullptr || ws_bytes < gs_verify_attn_workspace(N, Tq, total_kv, max_kv_len, Hq, Hkv, hd, dt))
+    return GS_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (dt == GS_F32)
+    return launch_attn_generic<float>(Q, K, V, O, cu_q, cu_kv, N, Tq, total_kv, max_kv_len, Hq, Hkv, hd,
+                                      scale, d_status, st);
+  return launch_attn_generic<__nv_bfloat16>(Q, K, V, O, cu_q, cu_kv, N, Tq, total_kv, max_kv_len, Hq, Hkv,
+                                            hd, scale, d_status, st);
+}

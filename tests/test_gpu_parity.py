@@ -1,0 +1,376 @@
+"""Parity of the CUDA library (through its C ABI) against the fp64 CPU oracle on the same seeded
+inputs.  Small cases compare every element; the full-size configurations compare everything the
+oracle can compute in seconds (attention and acceptance in full, the LM head on sampled columns
+plus the complete chain where the host has the memory for it)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import goodspeed_oracle as orc
+from paper_2512_09963_b200 import binding as B
+from paper_2512_09963_b200 import workloads as wl
+from paper_2512_09963_b200.runner import VerifyRound
+
+import parity_utils as pu
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def to_dev(inp):
+    return {k: (v.to(DEV) if isinstance(v, torch.Tensor) else v) for k, v in inp.items()}
+
+
+def tau32(tau):
+    """The library takes the temperature as fp32; the oracle gets the same value."""
+    return float(np.float32(tau))
+
+
+def run_accept_only(inp, update=False):
+    """spec_accept on the generator's fp32 logits: both sides read identical logits."""
+    d = to_dev(inp)
+    logits = d["target_logits_f32"].contiguous()
+    Tq, V = logits.shape
+    N = d["cu_q"].numel() - 1
+    rnd = VerifyRound(N=N, Tq=Tq, total_kv=1, max_kv_len=1, Hq=1, Hkv=1, hd=8, d=8, V=V,
+                      dtype=torch.float32, C=0, device=DEV)
+    rnd.accept(d["q_probs"], d["draft_tok"], d["cu_q"], d["u_accept"], d["u_sample"], inp["tau"],
+               logits=logits, update=update)
+    torch.cuda.synchronize()
+    assert int(rnd.d_status.item()) == 0
+    return rnd
+
+
+def check_accept(inp, rnd):
+    tau = tau32(inp["tau"])
+    ref = orc.ref_spec_accept(inp["target_logits_f32"], inp["q_probs"], inp["draft_tok"], inp["cu_q"],
+                              inp["u_accept"], inp["u_sample"], tau)
+    log = pu.compare_accept(pu.gpu_accept_dict(rnd), ref, inp["target_logits_f32"], inp["q_probs"],
+                            inp["cu_q"].cpu().numpy(), inp["u_sample"], tau, inp["target_logits_f32"].shape[1])
+    return ref, log
+
+
+# ------------------------------------------------------------------ cfg1: the whole round
+@pytest.mark.parametrize("tau", [1.0, 0.0])
+def test_cfg1_full_round(tau):
+    cfg = wl.CONFIGS["cfg1"]
+    inp = wl.make_step(cfg, tau=tau)
+    d = to_dev(inp)
+    rnd = VerifyRound.for_inputs(d, C=10)
+    rnd.run(d)
+    torch.cuda.synchronize()
+    assert int(rnd.d_status.item()) == 0
+    ref = orc.ref_verify_round(inp, np.full(cfg.N, 0.5), np.ones(cfg.N), 0.1, 0.5, 10)
+    pu.assert_close_rel(rnd.O, ref["O"], "attention output")
+    pu.assert_close_rel(rnd.logits, ref["logits"], "logits")
+    log = pu.compare_accept(pu.gpu_accept_dict(rnd), ref, ref["logits"], inp["q_probs"],
+                            inp["cu_q"].numpy(), inp["u_sample"], tau32(tau), cfg.V)
+    assert not log["accept_near_ties"] and not log["sample_near_ties"], log
+    np.testing.assert_allclose(rnd.alpha_hat.cpu().numpy(), ref["alpha_hat"], atol=1e-6)
+    np.testing.assert_allclose(rnd.X.cpu().numpy(), ref["X"], atol=1e-12)
+    assert np.array_equal(rnd.S_next.cpu().numpy(), ref["S_next"])
+    # fp32 path: far tighter than the bf16 bar
+    pu.assert_close_rel(rnd.logits, ref["logits"], "logits (fp32 bar)", rel=1e-4)
+    pu.assert_close_rel(rnd.O, ref["O"], "attention (fp32 bar)", rel=1e-4)
+
+
+def test_cfg1_matches_stored_golden():
+    """The oracle-written fixture (tests/golden) and the library agree on the integer outputs."""
+    import json, os
+    path = os.path.join(os.path.dirname(__file__), "golden", "cfg1_round.json")
+    gold = json.load(open(path))
+    for tau_key, tau in (("tau1", 1.0), ("tau0", 0.0)):
+        inp = wl.make_step(wl.CONFIGS["cfg1"], tau=tau)
+        d = to_dev(inp)
+        rnd = VerifyRound.for_inputs(d, C=10)
+        rnd.run(d)
+        torch.cuda.synchronize()
+        assert rnd.accepted.cpu().tolist() == gold[tau_key]["accepted"]
+        assert rnd.out_tok.cpu().tolist() == gold[tau_key]["out_tok"]
+        assert rnd.S_next.cpu().tolist() == gold[tau_key]["S_next"]
+
+
+# ------------------------------------------------------------------ spec_accept
+ACCEPT_CASES = [
+    # name, base cfg, V, tau   (V spans several 4096-chunks plus a ragged tail, or breaks the 16-byte path)
+    ("cfg2-shaped", "cfg2", 20000, 0.7),
+    ("cfg3-shaped", "cfg3", 12000, 1.0),
+    ("cfg4-shaped", "cfg4", 9000, 1.0),
+    ("odd-V", "cfg2", 4099, 0.7),
+    ("tiny-V", "cfg2", 5, 1.0),
+    ("greedy", "cfg3", 12000, 0.0),
+    ("cold", "cfg4", 8192, 0.05),
+]
+
+
+@pytest.mark.parametrize("name,base,V,tau", ACCEPT_CASES)
+def test_spec_accept_small(name, base, V, tau):
+    cfg = wl.shrink(wl.CONFIGS[base], V=V, d=64, prefix_scale=0.01, name=f"{base}_acc_{V}")
+    inp = wl.make_step(cfg, tau=tau, synthetic_logits=True, allocator=orc.ref_schedule_greedy)
+    rnd = run_accept_only(inp)
+    ref, log = check_accept(inp, rnd)
+    # identical logits on both sides: flips must be rare
+    assert len(log["accept_near_ties"]) <= 1
+    assert len(log["sample_near_ties"]) <= max(1, cfg.N // 8)
+    # run it again: bit-identical outputs (fixed summation order, no float atomics)
+    first = {k: v.copy() for k, v in pu.gpu_accept_dict(rnd).items()}
+    rnd2 = run_accept_only(inp)
+    for k, v in pu.gpu_accept_dict(rnd2).items():
+        assert np.array_equal(v, first[k]), k
+
+
+def test_spec_accept_zero_length_drafts_and_single_server():
+    cfg = wl.shrink(wl.CONFIGS["cfg2"], V=10000, d=64, prefix_scale=0.01, name="acc_gamma0")
+    inp = wl.make_step(cfg, gamma=[0, 3, 0, 0, 5, 1, 0, 2], synthetic_logits=True)
+    rnd = run_accept_only(inp)
+    ref, _ = check_accept(inp, rnd)
+    assert rnd.accepted.cpu().tolist()[0] == 0 and rnd.n_out.cpu().tolist()[0] == 1
+    cfg1 = wl.shrink(wl.CONFIGS["cfg2"], V=10000, d=64, N=1, prefix_scale=0.01, name="acc_single")
+    inp = wl.make_step(cfg1, gamma=[7], synthetic_logits=True)
+    check_accept(inp, run_accept_only(inp))
+    inp = wl.make_step(cfg1, gamma=[0], synthetic_logits=True)     # Gamma = 0: no draft arrays at all
+    check_accept(inp, run_accept_only(inp))
+
+
+def test_spec_accept_identical_draft_accepts_everything():
+    cfg = wl.shrink(wl.CONFIGS["cfg4"], V=8200, d=64, prefix_scale=0.01, name="acc_same")
+    inp = wl.make_step(cfg, sigma=np.zeros(cfg.N), synthetic_logits=True)
+    rnd = run_accept_only(inp)
+    # q == p up to fp32 rounding of the generator's softmax: ratios are 1 within 1e-5
+    assert np.all(rnd.ratio.cpu().numpy() > 1 - 1e-4)
+    check_accept(inp, rnd)
+
+
+def test_spec_accept_estimators_and_device_status():
+    cfg = wl.shrink(wl.CONFIGS["cfg2"], V=6000, d=64, prefix_scale=0.01, name="acc_ema")
+    inp = wl.make_step(cfg, synthetic_logits=True)
+    rnd = run_accept_only(inp, update=True)
+    ref, _ = check_accept(inp, rnd)
+    a_hat, X = orc.ref_ema(np.full(cfg.N, 0.5), np.ones(cfg.N), ref["ratio"], ref["accepted"],
+                           inp["cu_q"].numpy(), 0.1, 0.5)
+    if np.array_equal(rnd.accepted.cpu().numpy(), ref["accepted"]):
+        np.testing.assert_allclose(rnd.alpha_hat.cpu().numpy(), a_hat, atol=1e-6)
+        np.testing.assert_allclose(rnd.X.cpu().numpy(), X, atol=1e-12)
+    # a draft token outside the vocabulary: flagged on the device, treated as a rejection
+    bad = dict(inp)
+    bad["draft_tok"] = inp["draft_tok"].clone()
+    bad["draft_tok"][0] = cfg.V + 7
+    d = to_dev(bad)
+    r2 = VerifyRound(N=cfg.N, Tq=d["target_logits_f32"].shape[0], total_kv=1, max_kv_len=1, Hq=1, Hkv=1,
+                     hd=8, d=8, V=cfg.V, dtype=torch.float32, C=0, device=DEV)
+    r2.accept(d["q_probs"], d["draft_tok"], d["cu_q"], d["u_accept"], d["u_sample"], inp["tau"],
+              logits=d["target_logits_f32"], update=False)
+    torch.cuda.synchronize()
+    assert int(r2.d_status.item()) == 1      # GS_ERR_INVALID_ARG
+    assert int(r2.accepted[0].item()) == 0
+    # decreasing offsets: flagged, nothing written for that server, no fault
+    d2 = to_dev(inp)
+    cu = d2["cu_q"].clone()
+    cu[1] = cu[2] + 1
+    r3 = VerifyRound(N=cfg.N, Tq=d2["target_logits_f32"].shape[0], total_kv=1, max_kv_len=1, Hq=1, Hkv=1,
+                     hd=8, d=8, V=cfg.V, dtype=torch.float32, C=0, device=DEV)
+    r3.accept(d2["q_probs"], d2["draft_tok"], cu, d2["u_accept"], d2["u_sample"], inp["tau"],
+              logits=d2["target_logits_f32"], update=False)
+    torch.cuda.synchronize()
+    assert int(r3.d_status.item()) == 2      # GS_ERR_SHAPE
+
+
+# ------------------------------------------------------------------ scheduler
+@pytest.mark.parametrize("N,C", [(1, 5), (4, 10), (16, 128), (32, 256), (33, 64), (100, 300), (1024, 512), (8, 0)])
+def test_schedule_bit_exact(N, C):
+    r = np.random.default_rng(N * 1000 + C)
+    for trial in range(4):
+        X = r.uniform(0.5, 8.0, N)
+        al = r.uniform(0.001, 0.999, N)
+        if trial == 1:                      # many exact ties
+            X[:] = 2.0
+            al[:] = 0.75
+        lo = hi = None
+        if trial >= 2:
+            lo = r.integers(0, 2, N).astype(np.int32)
+            hi = (lo + r.integers(0, 20, N)).astype(np.int32)
+            if lo.sum() > C:
+                lo[:] = 0
+        S = torch.empty(N, dtype=torch.int32, device=DEV)
+        st = torch.zeros(1, dtype=torch.int32, device=DEV)
+        B.gs_schedule(torch.from_numpy(X).to(DEV), torch.from_numpy(al).to(DEV), C, S,
+                      None if lo is None else torch.from_numpy(lo).to(DEV),
+                      None if hi is None else torch.from_numpy(hi).to(DEV), st)
+        torch.cuda.synchronize()
+        want = orc.ref_schedule_greedy(X, al, C, lo, hi)
+        assert np.array_equal(S.cpu().numpy(), want), (N, C, trial)
+        assert int(st.item()) == 0
+        assert S.sum().item() <= C
+
+
+def test_schedule_floor_above_budget_is_flagged():
+    N = 4
+    S = torch.empty(N, dtype=torch.int32, device=DEV)
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    B.gs_schedule(torch.ones(N, dtype=torch.float64, device=DEV), torch.full((N,), 0.5, dtype=torch.float64, device=DEV),
+                  3, S, torch.full((N,), 2, dtype=torch.int32, device=DEV), None, st)
+    torch.cuda.synchronize()
+    assert S.cpu().tolist() == [2, 2, 2, 2] and int(st.item()) == 2
+
+
+# ------------------------------------------------------------------ attention
+def attn_case(cfg, gamma=None):
+    gamma = wl.draw_gamma(cfg, allocator=orc.ref_schedule_greedy) if gamma is None else np.asarray(gamma)
+    prefix = wl.draw_prefix(cfg)
+    return wl.make_attention_inputs(cfg, gamma, prefix)
+
+
+def run_attn(inp):
+    d = to_dev(inp)
+    Tq, Hq, hd = d["Q"].shape
+    total_kv, Hkv, _ = d["K"].shape
+    cu_kv = inp["cu_kv"]
+    max_len = int((cu_kv[1:] - cu_kv[:-1]).max())
+    N = cu_kv.numel() - 1
+    dt = B.GS_F32 if d["Q"].dtype == torch.float32 else B.GS_BF16
+    ws = torch.empty(max(256, B.gs_verify_attn_workspace(N, Tq, total_kv, max_len, Hq, Hkv, hd, dt)),
+                     dtype=torch.uint8, device=DEV)
+    O = torch.full_like(d["Q"], float("nan"))
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    B.gs_verify_attn(d["Q"], d["K"], d["V"], O, d["cu_q"], d["cu_kv"], max_len, hd ** -0.5, ws, st)
+    torch.cuda.synchronize()
+    return O, int(st.item())
+
+
+ATTN_CASES = [
+    ("cfg2-shaped", wl.shrink(wl.CONFIGS["cfg2"], prefix_scale=0.15, name="attn2")),       # 307-key prefixes
+    ("cfg3-shaped", wl.shrink(wl.CONFIGS["cfg3"], prefix_scale=0.08, name="attn3")),       # ragged 10..655
+    ("cfg4-shaped", wl.shrink(wl.CONFIGS["cfg4"], prefix_scale=0.07, N=5, name="attn4")),
+]
+
+
+@pytest.mark.parametrize("name,cfg", ATTN_CASES)
+def test_attention_small(name, cfg):
+    inp = attn_case(cfg)
+    O, st = run_attn(inp)
+    assert st == 0
+    ref = orc.ref_attention(inp["Q"], inp["K"], inp["V"], inp["cu_q"], inp["cu_kv"])
+    pu.assert_close_rel(O, ref, f"attention {name}")
+    O2, _ = run_attn(inp)
+    assert torch.equal(O, O2)                     # deterministic
+
+
+def test_attention_edge_shapes():
+    base = wl.shrink(wl.CONFIGS["cfg2"], prefix_scale=0.0, N=4, name="attn_edge")   # prefix 1
+    inp = wl.make_attention_inputs(base, np.array([0, 1, 16, 3]), np.array([1, 1, 1, 700]))
+    O, st = run_attn(inp)
+    assert st == 0
+    pu.assert_close_rel(O, orc.ref_attention(inp["Q"], inp["K"], inp["V"], inp["cu_q"], inp["cu_kv"]), "edge")
+    # empty prefix: position t sees only the t+1 new keys
+    inp = wl.make_attention_inputs(base, np.array([2, 0, 5, 1]), np.array([0, 0, 0, 0]))
+    O, st = run_attn(inp)
+    assert st == 0
+    pu.assert_close_rel(O, orc.ref_attention(inp["Q"], inp["K"], inp["V"], inp["cu_q"], inp["cu_kv"]), "no prefix")
+
+
+def test_attention_causality_and_server_permutation():
+    cfg = wl.shrink(wl.CONFIGS["cfg2"], prefix_scale=0.1, N=3, name="attn_prop")
+    inp = wl.make_attention_inputs(cfg, np.array([3, 2, 4]), np.array([200, 150, 90]))
+    O, _ = run_attn(inp)
+    # perturb the K/V of server 0's last new position: only its last query row may change
+    inp2 = dict(inp)
+    inp2["K"], inp2["V"] = inp["K"].clone(), inp["V"].clone()
+    last = int(inp["cu_kv"][1]) - 1
+    inp2["K"][last] += 3.0
+    inp2["V"][last] -= 2.0
+    O2, _ = run_attn(inp2)
+    assert torch.equal(O[:3], O2[:3]) and torch.equal(O[4:], O2[4:]) and not torch.equal(O[3], O2[3])
+    # swap servers 0 and 2: outputs move with them
+    cq, ck = inp["cu_q"].numpy(), inp["cu_kv"].numpy()
+    order = [2, 1, 0]
+    Q = torch.cat([inp["Q"][cq[i]:cq[i + 1]] for i in order])
+    K = torch.cat([inp["K"][ck[i]:ck[i + 1]] for i in order])
+    V = torch.cat([inp["V"][ck[i]:ck[i + 1]] for i in order])
+    perm = wl.make_attention_inputs(cfg, np.array([4, 2, 3]), np.array([90, 150, 200]))
+    perm["Q"], perm["K"], perm["V"] = Q, K, V
+    Op, _ = run_attn(perm)
+    want = torch.cat([O[cq[i]:cq[i + 1]] for i in order])
+    assert torch.equal(Op, want)
+
+
+def test_attention_bad_offsets_are_flagged():
+    cfg = wl.shrink(wl.CONFIGS["cfg2"], prefix_scale=0.05, N=2, name="attn_bad")
+    inp = wl.make_attention_inputs(cfg, np.array([2, 2]), np.array([50, 50]))
+    inp["cu_kv"] = inp["cu_kv"].clone()
+    inp["cu_kv"][1] = 1          # server 0 would have fewer keys than new positions
+    O, st = run_attn(inp)
+    assert st == 2
+
+
+# ------------------------------------------------------------------ LM head
+@pytest.mark.parametrize("T,d,V", [(44, 512, 9000), (96, 1024, 4104), (288, 256, 8192), (1, 64, 8), (130, 136, 1000)])
+def test_lm_head_small(T, d, V):
+    cfg = wl.shrink(wl.CONFIGS["cfg2"], d=d, V=V, name=f"head_{T}_{d}_{V}")
+    W = wl.make_layer(cfg)["W"]
+    H = wl.make_hidden(cfg, T)
+    logits = torch.full((T, V), float("nan"), dtype=torch.float32, device=DEV)
+    ws = torch.empty(max(256, B.gs_lm_head_workspace(T, d, V, B.GS_BF16)), dtype=torch.uint8, device=DEV)
+    B.gs_lm_head_logits(H.to(DEV), W.to(DEV), logits, ws)
+    torch.cuda.synchronize()
+    ref = orc.ref_lm_head(H, W)
+    pu.assert_close_rel(logits, ref, "logits")
+    # bf16 products are exact in fp32 and only the accumulation rounds: far inside the 2e-2 bar
+    pu.assert_close_rel(logits, ref, "logits (accumulation bar)", rel=2e-4)
+
+
+# ------------------------------------------------------------------ full-size configurations
+def _full_round(cfg_name, C, max_head_bytes=40e9):
+    cfg = wl.CONFIGS[cfg_name]
+    # big tensors are drawn on the device (seconds instead of minutes), then copied to the host
+    d = wl.make_step(cfg, allocator=orc.ref_schedule_greedy, device=DEV)
+    inp = {k: (v.cpu() if isinstance(v, torch.Tensor) else v) for k, v in d.items()}
+    rnd = VerifyRound.for_inputs(d, C=C)
+    rnd.run(d)
+    torch.cuda.synchronize()
+    assert int(rnd.d_status.item()) == 0
+    tau = tau32(inp["tau"])
+    # attention: every element
+    ref_O = orc.ref_attention(inp["Q"], inp["K"], inp["V"], inp["cu_q"], inp["cu_kv"])
+    pu.assert_close_rel(rnd.O, ref_O, f"{cfg_name} attention")
+    # LM head: the oracle's full fp64 product, column block by column block
+    V = cfg.V
+    ref_logits = np.empty((rnd.Tq, V))
+    step = 8192
+    for c0 in range(0, V, step):
+        cols = np.arange(c0, min(V, c0 + step))
+        ref_logits[:, cols] = orc.ref_lm_head(inp["H"], inp["W"], cols=cols)
+    pu.assert_close_rel(rnd.logits, ref_logits, f"{cfg_name} logits")
+    # acceptance, chained: library on its own logits vs oracle on its own logits
+    ref = orc.ref_spec_accept(ref_logits, inp["q_probs"], inp["draft_tok"], inp["cu_q"], inp["u_accept"],
+                              inp["u_sample"], tau)
+    log = pu.compare_accept(pu.gpu_accept_dict(rnd), ref, ref_logits, inp["q_probs"], inp["cu_q"].numpy(),
+                            inp["u_sample"], tau, V)
+    assert len(log["accept_near_ties"]) <= 1, log
+    # acceptance alone on identical logits (the generator's fp32 product)
+    rnd_a = run_accept_only(inp)
+    _, log2 = check_accept(inp, rnd_a)
+    # estimators and next allocation where the counts agree
+    a_hat, X = orc.ref_ema(np.full(cfg.N, 0.5), np.ones(cfg.N), ref["ratio"], ref["accepted"],
+                           inp["cu_q"].numpy(), 0.1, 0.5)
+    if not log["accept_near_ties"]:
+        np.testing.assert_allclose(rnd.alpha_hat.cpu().numpy(), a_hat, atol=1e-5)
+        np.testing.assert_allclose(rnd.X.cpu().numpy(), X, atol=1e-12)
+        S_ref = orc.ref_schedule_greedy(X, a_hat, C)
+        S_gpu = rnd.S_next.cpu().numpy()
+        if not np.array_equal(S_gpu, S_ref):     # estimator rounding moved a near-tied marginal
+            assert S_gpu.sum() == S_ref.sum()
+            o1, o2 = orc.ref_sched_objective(X, a_hat, S_gpu), orc.ref_sched_objective(X, a_hat, S_ref)
+            assert abs(o1 - o2) <= 1e-6 * abs(o2)
+    print(cfg_name, "chain log", log, "accept-only log", log2)
+
+
+def test_cfg2_full_size():
+    _full_round("cfg2", C=64)
+
+
+def test_cfg3_full_size():
+    _full_round("cfg3", C=256)
+
+
+def test_cfg4_full_size():
+    _full_round("cfg4", C=128)
