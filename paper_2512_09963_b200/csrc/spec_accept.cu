@@ -59,9 +59,10 @@ static size_t sa_layout(int N, int Tq, int V, SaWorkspace* w, char* base) {
 }
 
 // Loads the 16 floats a thread owns in a chunk: element (k*256 + tid)*4 + j, k,j in 0..3.
-// Out-of-range elements read as -inf.
+// Out-of-range elements read as `fill`.
 template <bool VEC>
-GS_DEVINL void load_chunk(const float* __restrict__ row, int base, int V, int tid, float (&v)[kSaPerThread]) {
+GS_DEVINL void load_chunk(const float* __restrict__ row, int base, int V, int tid, float (&v)[kSaPerThread],
+                          float fill = -INFINITY) {
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
     int idx = base + (k * kSaThreads + tid) * 4;
@@ -70,7 +71,7 @@ GS_DEVINL void load_chunk(const float* __restrict__ row, int base, int V, int ti
       v[4 * k + 0] = t.x; v[4 * k + 1] = t.y; v[4 * k + 2] = t.z; v[4 * k + 3] = t.w;
     } else {
 #pragma unroll
-      for (int j = 0; j < 4; ++j) v[4 * k + j] = (idx + j < V) ? __ldg(row + idx + j) : -INFINITY;
+      for (int j = 0; j < 4; ++j) v[4 * k + j] = (idx + j < V) ? __ldg(row + idx + j) : fill;
     }
   }
 }
@@ -268,7 +269,7 @@ sa_mass(const float* __restrict__ logits, const float* __restrict__ q_probs, int
   float l[kSaPerThread], q[kSaPerThread];
   load_chunk<VEC>(logits + (size_t)s.row * V, base, V, tid, l);
   const bool resid = s.qrow >= 0;
-  if (resid) load_chunk<VEC>(q_probs + (size_t)s.qrow * V, base, V, tid, q);
+  if (resid) load_chunk<VEC>(q_probs + (size_t)s.qrow * V, base, V, tid, q, 0.f);
   double acc = 0.0;
 #pragma unroll
   for (int e = 0; e < kSaPerThread; ++e) acc += elem_mass(l[e], s.M, k2, s.invZ, resid, resid ? q[e] : 0.f);
