@@ -97,6 +97,11 @@ gs_status gs_verify_attn(const void* Q, const void* K, const void* V, void* O,
  * Errors: INVALID_ARG, UNSUPPORTED (alignment rules above), WORKSPACE, CUDA.
  */
 size_t gs_lm_head_workspace(int T, int d, int V, gs_dtype dt);
+/* Tuning knobs of the bf16 kernel (process-wide, not thread-safe; 0 = choose automatically):
+ * m_tiles = upper bound on the blocks of 128 vocabulary columns a CTA owns per tile (1..9),
+ * stages = upper bound on the depth of the shared-memory ring of W, k_rows = rows of W per ring
+ * stage (16, 32 or 64).  Results do not depend on them.  Errors: INVALID_ARG. */
+gs_status gs_lm_head_configure(int m_tiles, int stages, int k_rows);
 gs_status gs_lm_head_logits(const void* H, const void* W, float* logits, int T, int d, int V,
                             gs_dtype dt, void* ws, size_t ws_bytes, int32_t* d_status, void* stream);
 

@@ -1,9 +1,30 @@
-// gs_lm_head_logits: logits = H W (Sec. II-A1).  fp32 inputs use a plain FMA kernel.
+// gs_lm_head_logits: logits = H W (Sec. II-A1).
+//
+// bf16 path (tcgen05 / tensor memory).  The product is computed transposed, logits^T = W^T H^T:
+// the vocabulary dimension is the MMA's M (128 columns of W per MMA, read as an MN-major A
+// operand straight from W's [d, V] layout) and the verify positions are the MMA's N (H is the
+// K-major B operand).  A CTA owns a tile of up to 9 consecutive 128-column units for ALL
+// positions, so W is streamed from HBM exactly once and each k row of a tile is one long
+// contiguous run; H (a few MB) is re-read from L2 through its own small ring.  With the
+// vocabulary on the TMEM lanes, an epilogue thread holds one vocabulary column and a warp's
+// store of one position is 32 consecutive floats of the row-major [T, V] output.
+//
+//   warp 0     TMA producer: W boxes (kw k rows x 64 v, 128-byte swizzle) into a deep ring of
+//              stages, H boxes (n_tile rows x 64 k) into a 3-stage ring
+//   warp 1     allocates tensor memory, issues tcgen05.mma (one thread), commits stages back
+//   warps 2-5  epilogue: tcgen05.ld the fp32 accumulators, store logits
+// Tiles are spread so that every SM gets the same number of them and widths differ by at most
+// one unit.  Accumulators are double-buffered in tensor memory when they fit.  Every barrier
+// wait is time-bounded.
+//
+// fp32 inputs use a plain FMA kernel (small problems only).
 #include "common.cuh"
 #include "attn_generic.cuh"
+#include "sm100_ptx.cuh"
 
 namespace gs {
 
+// ------------------------------------------------------------------ plain kernel (fp32)
 constexpr int kHeadRows = 16;      // rows of H per CTA
 constexpr int kHeadCols = 256;     // one column per thread
 constexpr int kHeadKc = 64;        // k-slice staged in shared memory
@@ -50,7 +71,286 @@ inline gs_status launch_lm_head_plain(const void* H, const void* W, float* logit
   return launch_status();
 }
 
+// ------------------------------------------------------------------ tcgen05 kernel (bf16)
+constexpr int kTcThreads = 192;
+constexpr uint32_t kBlockK = 64;            // k depth of one H stage = one 128-byte swizzle row
+constexpr uint32_t kTileM = 128;            // vocabulary columns per MMA ("unit")
+constexpr uint32_t kMaxSmem = 232448;       // 227 KB
+constexpr int kMaxRowsPerLaunch = 512;      // tensor memory has 512 fp32 columns
+constexpr int kHStages = 3;
+
+struct HeadTcParams {
+  float* logits;
+  int32_t* d_status;
+  int T, d, V;
+  int row0;              // first row of H / logits this launch covers
+  int nt, n_tile;        // N tiles and rows of H per N tile
+  int n_acc;             // accumulator buffers in tensor memory
+  int kw;                // k rows of W per W stage (16, 32 or 64)
+  int w_stages, k_blocks;
+  int num_tiles;         // tiles of the vocabulary; tile i is `unit_base + (i < unit_rem)` units wide
+  int unit_base, unit_rem;
+  uint32_t w_stage_bytes, h_stage_bytes, acc_cols, tmem_cols;
+};
+
+// Tile i covers units [unit0, unit0 + width) of 128 vocabulary columns each.
+GS_DEVINL void head_tile(const HeadTcParams& P, int i, int& unit0, int& width) {
+  width = P.unit_base + (i < P.unit_rem ? 1 : 0);
+  unit0 = i * P.unit_base + min(i, P.unit_rem);
+}
+
+__global__ void __launch_bounds__(kTcThreads, 1)
+lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmapW, const __grid_constant__ CUtensorMap tmapH,
+                  const HeadTcParams P) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;            // stages need 1024-byte alignment
+  uint8_t* sm = smem_raw + (base - raw);
+  const uint32_t h_base = base + (uint32_t)P.w_stages * P.w_stage_bytes;
+  const uint32_t bars = h_base + (uint32_t)kHStages * P.h_stage_bytes;
+  const int WS = P.w_stages;
+  auto wfull_bar = [&](int s) { return bars + 8u * (uint32_t)s; };
+  auto wempty_bar = [&](int s) { return bars + 8u * (uint32_t)(WS + s); };
+  auto hfull_bar = [&](int s) { return bars + 8u * (uint32_t)(2 * WS + s); };
+  auto hempty_bar = [&](int s) { return bars + 8u * (uint32_t)(2 * WS + kHStages + s); };
+  auto tfull_bar = [&](int a) { return bars + 8u * (uint32_t)(2 * WS + 2 * kHStages + a); };
+  auto tempty_bar = [&](int a) { return bars + 8u * (uint32_t)(2 * WS + 2 * kHStages + 2 + a); };
+  const uint32_t n_bars = (uint32_t)(2 * WS + 2 * kHStages + 4);
+  uint8_t* tail = sm + (bars - base) + 8u * n_bars;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 4);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < WS; ++s) { mbar_init(wfull_bar(s), 1); mbar_init(wempty_bar(s), 1); }
+    for (int s = 0; s < kHStages; ++s) { mbar_init(hfull_bar(s), 1); mbar_init(hempty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    *abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+    tma_prefetch_desc(&tmapW);
+    tma_prefetch_desc(&tmapH);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), P.tmem_cols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int subs = (int)kBlockK / P.kw;                 // W stages per H stage
+  const uint32_t w_box_bytes = (uint32_t)P.kw * 128u;   // one box: kw k rows x 64 v
+
+  if (warp == 0) {
+    // ---------------- TMA producer (loads are issued in the order the MMA warp consumes them)
+    if (lane == 0) {
+      uint32_t ws = 0, wph = 0, hs = 0, hph = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < P.num_tiles && ok; tile += gridDim.x) {
+        int unit0, width;
+        head_tile(P, tile, unit0, width);
+        const int v0 = unit0 * (int)kTileM;
+        const int boxes = 2 * width;
+        for (int kb = 0; kb < P.k_blocks && ok; ++kb) {
+          const int k0 = kb * (int)kBlockK;
+          if (!mbar_wait(hempty_bar(hs), hph ^ 1u, abort_flag)) { ok = false; break; }
+          mbar_arrive_expect_tx(hfull_bar(hs), P.h_stage_bytes);
+          for (int j = 0; j < P.nt; ++j)
+            tma_load_2d(h_base + hs * P.h_stage_bytes + (uint32_t)(j * P.n_tile) * 128u, &tmapH, k0,
+                        P.row0 + j * P.n_tile, hfull_bar(hs));
+          if (++hs == (uint32_t)kHStages) { hs = 0; hph ^= 1u; }
+          for (int sub = 0; sub < subs; ++sub) {
+            if (!mbar_wait(wempty_bar(ws), wph ^ 1u, abort_flag)) { ok = false; break; }
+            mbar_arrive_expect_tx(wfull_bar(ws), (uint32_t)boxes * w_box_bytes);
+            const uint32_t dst = base + ws * P.w_stage_bytes;
+            for (int b = 0; b < boxes; ++b)
+              tma_load_2d(dst + (uint32_t)b * w_box_bytes, &tmapW, v0 + b * 64, k0 + sub * P.kw, wfull_bar(ws));
+            if (++ws == (uint32_t)WS) { ws = 0; wph ^= 1u; }
+          }
+        }
+      }
+      if (!ok) {
+        // Let loads that are still in flight land before the CTA goes away (bounded).
+        const uint64_t t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 200000ull) { }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ---------------- MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = idesc_bf16(kTileM, (uint32_t)P.n_tile, /*A (W^T) MN-major*/ true, /*B (H) K-major*/ false);
+      uint32_t ws = 0, wph = 0, hs = 0, hph = 0;
+      int it = 0;
+      bool ok = true;
+      const int k16_per_stage = P.kw / 16;
+      for (int tile = blockIdx.x; tile < P.num_tiles && ok; tile += gridDim.x, ++it) {
+        int unit0, width;
+        head_tile(P, tile, unit0, width);
+        const int acc = it % P.n_acc;
+        const uint32_t acc_ph = (uint32_t)(it / P.n_acc) & 1u;
+        if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        for (int kb = 0; kb < P.k_blocks && ok; ++kb) {
+          if (!mbar_wait(hfull_bar(hs), hph, abort_flag)) { ok = false; break; }
+          const uint32_t b_base = h_base + hs * P.h_stage_bytes;
+          for (int sub = 0; sub < subs; ++sub) {
+            if (!mbar_wait(wfull_bar(ws), wph, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t a_base = base + ws * P.w_stage_bytes;
+            for (int kk = 0; kk < k16_per_stage; ++kk) {
+              const int k16 = sub * k16_per_stage + kk;       // position inside the 64-deep H stage
+              for (int m = 0; m < width; ++m) {
+                // A: two 64-column boxes kw*128 bytes apart; 16 k = two 1024-byte groups of 8 k rows
+                const uint64_t adesc = smem_desc_sw128(a_base + (uint32_t)m * 2u * w_box_bytes + (uint32_t)kk * 2048u,
+                                                       w_box_bytes, 1024u);
+                for (int j = 0; j < P.nt; ++j) {
+                  // B: rows of 128 bytes, 8-row groups of 1024 bytes; 16 k = 32 bytes along the row
+                  const uint64_t bdesc = smem_desc_sw128(b_base + (uint32_t)(j * P.n_tile) * 128u + (uint32_t)k16 * 32u,
+                                                         16u, 1024u);
+                  const uint32_t d_tmem = tmem_base + (uint32_t)acc * P.acc_cols + (uint32_t)((m * P.nt + j) * P.n_tile);
+                  umma_bf16(d_tmem, adesc, bdesc, idesc, (kb | k16) != 0 ? 1u : 0u);
+                }
+              }
+            }
+            umma_commit(wempty_bar(ws));      // frees the W stage once these MMAs have read it
+            if (++ws == (uint32_t)WS) { ws = 0; wph ^= 1u; }
+          }
+          if (ok) umma_commit(hempty_bar(hs));
+          if (++hs == (uint32_t)kHStages) { hs = 0; hph ^= 1u; }
+        }
+        if (ok) umma_commit(tfull_bar(acc));
+      }
+      if (!ok) {
+        // MMAs may still be running: give them (bounded) time before TMEM is freed.
+        const uint64_t t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 200000ull) { }
+      }
+    }
+    __syncwarp();
+  } else {
+    // ---------------- epilogue (warps 2..5): TMEM lane quadrant = warp % 4
+    const int q = warp & 3;
+    int it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < P.num_tiles && ok; tile += gridDim.x, ++it) {
+      int unit0, width;
+      head_tile(P, tile, unit0, width);
+      const int acc = it % P.n_acc;
+      const uint32_t acc_ph = (uint32_t)(it / P.n_acc) & 1u;
+      if (!mbar_wait(tfull_bar(acc), acc_ph, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      for (int m = 0; m < width; ++m) {
+        const int v = (unit0 + m) * (int)kTileM + q * 32 + lane;
+        for (int j = 0; j < P.nt; ++j) {
+          for (int c0 = 0; c0 < P.n_tile; c0 += 16) {
+            const int t_first = j * P.n_tile + c0;
+            if (t_first >= P.T) break;                       // warp-uniform
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * P.acc_cols +
+                                   (uint32_t)((m * P.nt + j) * P.n_tile + c0);
+            uint32_t r[16];
+            tmem_ld16(taddr, r);
+            tmem_ld_wait();
+            if (v < P.V) {
+              float* out = P.logits + (size_t)(P.row0 + t_first) * P.V + v;
+#pragma unroll
+              for (int c = 0; c < 16; ++c)
+                if (t_first + c < P.T) out[(size_t)c * P.V] = __uint_as_float(r[c]);
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(acc));
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) set_status(P.d_status, GS_ERR_TIMEOUT);
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, P.tmem_cols);
+  }
+}
+
+static int g_head_mt = 0;       // 0 = choose automatically
+static int g_head_stages = 0;
+static int g_head_kw = 0;
+
+inline gs_status launch_lm_head_tc(const void* H, const void* W, float* logits, int T, int d, int V,
+                                   int32_t* d_status, cudaStream_t st) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(lm_head_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem) !=
+        cudaSuccess)
+      return GS_ERR_CUDA;
+    attr_set = true;
+  }
+  const int sms = sm_count();
+  const int units = (V + (int)kTileM - 1) / (int)kTileM;
+  for (int row0 = 0; row0 < T; row0 += kMaxRowsPerLaunch) {
+    const int rows = min(kMaxRowsPerLaunch, T - row0);
+    HeadTcParams P;
+    P.logits = logits; P.d_status = d_status;
+    P.T = rows; P.d = d; P.V = V; P.row0 = row0;
+    P.nt = (rows + 255) / 256;
+    P.n_tile = (((rows + P.nt - 1) / P.nt) + 15) / 16 * 16;
+    const int total_n = P.nt * P.n_tile;
+    // Widest tile (in units of 128 columns) whose accumulators fit the 512 TMEM columns.
+    int max_mt = min(512 / total_n, 9);
+    if (g_head_mt > 0) max_mt = min(max_mt, g_head_mt);
+    if (max_mt < 1) return GS_ERR_UNSUPPORTED;
+    // Every SM gets the same number of tiles; tile widths differ by at most one unit.
+    const int per_sm = (units + sms - 1) / sms;
+    const int tiles_per_sm = (per_sm + max_mt - 1) / max_mt;
+    const int num_tiles = min(units, sms * tiles_per_sm);
+    P.num_tiles = num_tiles;
+    P.unit_base = units / num_tiles;
+    P.unit_rem = units % num_tiles;
+    const int mt = P.unit_base + (P.unit_rem ? 1 : 0);                // widest tile
+    P.acc_cols = (uint32_t)(mt * total_n);
+    P.n_acc = (2 * P.acc_cols <= 512) ? 2 : 1;
+    uint32_t cols = 32;
+    while (cols < (uint32_t)P.n_acc * P.acc_cols) cols <<= 1;
+    P.tmem_cols = cols;
+    // k rows per W stage: wide tiles use shallow stages so that a stage is a few long rows.
+    const int kw = g_head_kw > 0 ? g_head_kw : (mt >= 4 ? 16 : (mt >= 2 ? 32 : 64));
+    P.kw = kw;
+    P.w_stage_bytes = (uint32_t)mt * 2u * (uint32_t)kw * 128u;
+    P.h_stage_bytes = (uint32_t)total_n * 128u;
+    const uint32_t fixed = 1024u /*alignment*/ + (uint32_t)kHStages * P.h_stage_bytes + 8u * 64u + 64u;
+    if (fixed + 2 * P.w_stage_bytes > kMaxSmem) return GS_ERR_UNSUPPORTED;
+    int stages = (int)((kMaxSmem - fixed) / P.w_stage_bytes);
+    if (stages > 24) stages = 24;
+    if (g_head_stages > 0 && g_head_stages < stages) stages = g_head_stages;
+    if (stages < 2) return GS_ERR_UNSUPPORTED;
+    P.w_stages = stages;
+    P.k_blocks = (d + (int)kBlockK - 1) / (int)kBlockK;
+    CUtensorMap tmapW, tmapH;
+    if (!make_tmap_bf16_2d(&tmapW, W, (uint64_t)d, (uint64_t)V, (uint64_t)V, (uint32_t)kw, 64)) return GS_ERR_CUDA;
+    if (!make_tmap_bf16_2d(&tmapH, H, (uint64_t)T, (uint64_t)d, (uint64_t)d, (uint32_t)P.n_tile, 64))
+      return GS_ERR_CUDA;
+    const size_t smem = 1024u + (size_t)stages * P.w_stage_bytes + (size_t)kHStages * P.h_stage_bytes +
+                        8u * (2u * (uint32_t)stages + 2u * kHStages + 4u) + 64u;
+    const int grid = min(P.num_tiles, sms);
+    lm_head_tc_kernel<<<grid, kTcThreads, smem, st>>>(tmapW, tmapH, P);
+    if (cudaGetLastError() != cudaSuccess) return GS_ERR_CUDA;
+  }
+  return GS_OK;
+}
+
 }  // namespace gs
+
+extern "C" gs_status gs_lm_head_configure(int m_tiles, int stages, int k_rows) {
+  if (m_tiles < 0 || m_tiles > 9 || stages < 0) return GS_ERR_INVALID_ARG;
+  if (k_rows != 0 && k_rows != 16 && k_rows != 32 && k_rows != 64) return GS_ERR_INVALID_ARG;
+  gs::g_head_mt = m_tiles;
+  gs::g_head_stages = stages;
+  gs::g_head_kw = k_rows;
+  return GS_OK;
+}
 
 extern "C" size_t gs_lm_head_workspace(int T, int d, int V, gs_dtype dt) {
   (void)T; (void)d; (void)V; (void)dt;
@@ -61,7 +361,6 @@ extern "C" gs_status gs_lm_head_logits(const void* H, const void* W, float* logi
                                        gs_dtype dt, void* ws, size_t ws_bytes, int32_t* d_status,
                                        void* stream) {
   using namespace gs;
-  (void)d_status;
   if (T < 0 || d < 0 || V < 0) return GS_ERR_INVALID_ARG;
   if (dt != GS_F32 && dt != GS_BF16) return GS_ERR_INVALID_ARG;
   if (T == 0 || V == 0) return GS_OK;
@@ -70,5 +369,8 @@ extern "C" gs_status gs_lm_head_logits(const void* H, const void* W, float* logi
   if ((T + kHeadRows - 1) / kHeadRows > 65535) return GS_ERR_UNSUPPORTED;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (dt == GS_F32) return launch_lm_head_plain<float>(H, W, logits, T, d, V, st);
-  return launch_lm_head_plain<__nv_bfloat16>(H, W, logits, T, d, V, st);
+  const bool tma_ok = d > 0 && (d % 8 == 0) && (V % 8 == 0) && (reinterpret_cast<uintptr_t>(H) % 16 == 0) &&
+                      (reinterpret_cast<uintptr_t>(W) % 16 == 0);
+  if (!tma_ok) return GS_ERR_UNSUPPORTED;
+  return launch_lm_head_tc(H, W, logits, T, d, V, d_status, st);
 }

@@ -38,9 +38,21 @@ def assert_close_rel(got, ref, what, rel=REL_TOL):
     return float(np.max(err / np.maximum(bound, 1e-300)))
 
 
-def compare_accept(gpu, ref, logits, q_probs, cu_q, u_sample, tau, V):
+def chain_slack(gpu_logits, ref_logits, tau):
+    """Extra probability tolerance when the two sides ran on their OWN logits (library: bf16
+    products accumulated in fp32 on the tensor cores; oracle: fp64).  A logit error e moves
+    log p(s) = l_s/tau - logsumexp(l/tau) by at most 2e/tau, and p, min(1, p/q) <= 1, so the
+    probabilities move by at most 2e/tau.  e is the largest observed logit difference."""
+    e = float(np.max(np.abs(np64(gpu_logits) - np64(ref_logits))))
+    return 2.0 * e / tau if tau > 0 else 0.0
+
+
+def compare_accept(gpu, ref, logits, q_probs, cu_q, u_sample, tau, V, slack=0.0):
     """gpu: dict of numpy arrays accepted/out_tok/n_out/ratio/p_tok from the library;
-    ref: ref_spec_accept output on the same inputs.  Returns a log dict."""
+    ref: ref_spec_accept output on the same inputs.  slack widens the probability tolerance and
+    the near-tie band (see chain_slack); it is 0 when both sides read identical logits.
+    Returns a log dict."""
+    PROB_ATOL_, NEAR_TIE_ = PROB_ATOL + slack, NEAR_TIE + slack
     cu_q = np.asarray(cu_q, dtype=np.int64)
     N = len(cu_q) - 1
     log = {"accept_near_ties": [], "sample_near_ties": [], "sample_exact": 0, "servers": N}
@@ -54,16 +66,16 @@ def compare_accept(gpu, ref, logits, q_probs, cu_q, u_sample, tau, V):
         assert 0 <= a_g <= gamma, f"server {i}: accepted {a_g} outside [0,{gamma}]"
         assert int(gpu["n_out"][i]) == a_g + 1
         np.testing.assert_allclose(gpu["ratio"][g0:g0 + gamma], ref["ratio"][g0:g0 + gamma], rtol=0,
-                                   atol=PROB_ATOL, err_msg=f"ratio, server {i}")
+                                   atol=PROB_ATOL_, err_msg=f"ratio, server {i}")
         np.testing.assert_allclose(gpu["p_tok"][g0:g0 + gamma], ref["p_tok"][g0:g0 + gamma], rtol=0,
-                                   atol=PROB_ATOL, err_msg=f"p_tok, server {i}")
+                                   atol=PROB_ATOL_, err_msg=f"p_tok, server {i}")
         seg = gpu["out_tok"][r0:r0 + gamma + 1]
         assert np.all(seg[a_g + 1:] == -1), f"server {i}: padding after the last token"
         assert 0 <= seg[a_g] < V, f"server {i}: emitted id {seg[a_g]} outside the vocabulary"
         if a_g != a_r:
             j = min(a_g, a_r)
             marg = abs(ref["margin_acc"][g0 + j])
-            assert marg < NEAR_TIE, (f"server {i}: accepted {a_g} vs oracle {a_r}, decision {j} has "
+            assert marg < NEAR_TIE_, (f"server {i}: accepted {a_g} vs oracle {a_r}, decision {j} has "
                                      f"|u - p/q| = {marg:.3e}")
             log["accept_near_ties"].append((i, j, float(marg)))
             continue
@@ -80,7 +92,7 @@ def compare_accept(gpu, ref, logits, q_probs, cu_q, u_sample, tau, V):
         lo = (F[tok_g - 1] if tok_g > 0 else 0.0) / R
         hi = F[tok_g] / R
         dist = max(0.0, lo - u_sample[i], u_sample[i] - hi)
-        assert w[tok_g] > 0 and dist < NEAR_TIE, (
+        assert w[tok_g] > 0 and dist < NEAR_TIE_, (
             f"server {i}: emitted {tok_g}, oracle {tok_r}; u={u_sample[i]:.8f} is {dist:.3e} away from "
             f"the emitted token's CDF interval [{lo:.8f},{hi:.8f}]")
         log["sample_near_ties"].append((i, tok_g, tok_r, float(dist)))

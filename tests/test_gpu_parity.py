@@ -343,8 +343,10 @@ def _full_round(cfg_name, C, max_head_bytes=40e9):
     # acceptance, chained: library on its own logits vs oracle on its own logits
     ref = orc.ref_spec_accept(ref_logits, inp["q_probs"], inp["draft_tok"], inp["cu_q"], inp["u_accept"],
                               inp["u_sample"], tau)
+    slack = pu.chain_slack(rnd.logits, ref_logits, tau)
+    assert slack < 5e-4, slack
     log = pu.compare_accept(pu.gpu_accept_dict(rnd), ref, ref_logits, inp["q_probs"], inp["cu_q"].numpy(),
-                            inp["u_sample"], tau, V)
+                            inp["u_sample"], tau, V, slack=slack)
     assert len(log["accept_near_ties"]) <= 1, log
     # acceptance alone on identical logits (the generator's fp32 product)
     rnd_a = run_accept_only(inp)
