@@ -99,6 +99,13 @@ GS_DEVINL void head_tile(const HeadTcParams& P, int i, int& unit0, int& width) {
   unit0 = i * P.unit_base + min(i, P.unit_rem);
 }
 
+constexpr int kMaxUnits = 9;                // widest tile, in units
+
+// KW = k rows of W per ring stage, NT = number of N tiles.  Both are compile-time so that the
+// MMA issue loop unrolls completely: every descriptor is then "a per-stage base plus a constant",
+// which keeps the single issuing thread ahead of the tensor core even when an MMA is short
+// (a 128 x 48 x 16 MMA occupies the tensor core for about 45 cycles).
+template <int KW, int NT>
 __global__ void __launch_bounds__(kTcThreads, 1)
 lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmapW, const __grid_constant__ CUtensorMap tmapH,
                   const HeadTcParams P) {
@@ -139,8 +146,8 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmapW, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const int subs = (int)kBlockK / P.kw;                 // W stages per H stage
-  const uint32_t w_box_bytes = (uint32_t)P.kw * 128u;   // one box: kw k rows x 64 v
+  constexpr int subs = (int)kBlockK / KW;               // W stages per H stage
+  constexpr uint32_t w_box_bytes = (uint32_t)KW * 128u; // one box: KW k rows x 64 v
 
   if (warp == 0) {
     // ---------------- TMA producer (loads are issued in the order the MMA warp consumes them)
@@ -156,7 +163,7 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmapW, const __grid_consta
           const int k0 = kb * (int)kBlockK;
           if (!mbar_wait(hempty_bar(hs), hph ^ 1u, abort_flag)) { ok = false; break; }
           mbar_arrive_expect_tx(hfull_bar(hs), P.h_stage_bytes);
-          for (int j = 0; j < P.nt; ++j)
+          for (int j = 0; j < NT; ++j)
             tma_load_2d(h_base + hs * P.h_stage_bytes + (uint32_t)(j * P.n_tile) * 128u, &tmapH, k0,
                         P.row0 + j * P.n_tile, hfull_bar(hs));
           if (++hs == (uint32_t)kHStages) { hs = 0; hph ^= 1u; }
@@ -165,7 +172,7 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmapW, const __grid_consta
             mbar_arrive_expect_tx(wfull_bar(ws), (uint32_t)boxes * w_box_bytes);
             const uint32_t dst = base + ws * P.w_stage_bytes;
             for (int b = 0; b < boxes; ++b)
-              tma_load_2d(dst + (uint32_t)b * w_box_bytes, &tmapW, v0 + b * 64, k0 + sub * P.kw, wfull_bar(ws));
+              tma_load_2d(dst + (uint32_t)b * w_box_bytes, &tmapW, v0 + b * 64, k0 + sub * KW, wfull_bar(ws));
             if (++ws == (uint32_t)WS) { ws = 0; wph ^= 1u; }
           }
         }
@@ -181,10 +188,21 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmapW, const __grid_consta
     // ---------------- MMA issuer
     if (lane == 0) {
       const uint32_t idesc = idesc_bf16(kTileM, (uint32_t)P.n_tile, /*A (W^T) MN-major*/ true, /*B (H) K-major*/ false);
+      // Descriptors differ only in their low word (the start address >> 4).
+      //   A (W^T, MN-major): two 64-column boxes KW*128 bytes apart (leading offset), 8-k groups
+      //                      1024 bytes apart (stride offset); 16 k further = +2048 bytes.
+      //   B (H, K-major):    rows of 128 bytes, 8-row groups 1024 bytes apart; 16 k further = +32 bytes.
+      const uint64_t a_desc0 = smem_desc_sw128(base, w_box_bytes, 1024u);
+      const uint64_t b_desc0 = smem_desc_sw128(h_base, 16u, 1024u);
+      const uint32_t a_hi = (uint32_t)(a_desc0 >> 32), a_lo0 = (uint32_t)a_desc0;
+      const uint32_t b_hi = (uint32_t)(b_desc0 >> 32), b_lo0 = (uint32_t)b_desc0;
+      const uint32_t w_stage_u = P.w_stage_bytes >> 4, h_stage_u = P.h_stage_bytes >> 4;
+      const uint32_t n_tile_u = ((uint32_t)P.n_tile * 128u) >> 4;       // one N tile of H, in 16-byte units
+      const uint32_t n_tile = (uint32_t)P.n_tile;
       uint32_t ws = 0, wph = 0, hs = 0, hph = 0;
       int it = 0;
       bool ok = true;
-      const int k16_per_stage = P.kw / 16;
+      constexpr int k16_per_stage = KW / 16;
       for (int tile = blockIdx.x; tile < P.num_tiles && ok; tile += gridDim.x, ++it) {
         int unit0, width;
         head_tile(P, tile, unit0, width);
@@ -192,25 +210,30 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmapW, const __grid_consta
         const uint32_t acc_ph = (uint32_t)(it / P.n_acc) & 1u;
         if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
+        const uint32_t d_acc = tmem_base + (uint32_t)acc * P.acc_cols;
         for (int kb = 0; kb < P.k_blocks && ok; ++kb) {
           if (!mbar_wait(hfull_bar(hs), hph, abort_flag)) { ok = false; break; }
-          const uint32_t b_base = h_base + hs * P.h_stage_bytes;
+          const uint32_t b_lo_stage = b_lo0 + hs * h_stage_u;
+#pragma unroll
           for (int sub = 0; sub < subs; ++sub) {
             if (!mbar_wait(wfull_bar(ws), wph, abort_flag)) { ok = false; break; }
             tc_fence_after();
-            const uint32_t a_base = base + ws * P.w_stage_bytes;
+            const uint32_t a_lo_stage = a_lo0 + ws * w_stage_u;
+            const uint32_t fresh = (kb == 0 && sub == 0) ? 1u : 0u;    // first MMAs of the tile overwrite
+#pragma unroll
             for (int kk = 0; kk < k16_per_stage; ++kk) {
-              const int k16 = sub * k16_per_stage + kk;       // position inside the 64-deep H stage
-              for (int m = 0; m < width; ++m) {
-                // A: two 64-column boxes kw*128 bytes apart; 16 k = two 1024-byte groups of 8 k rows
-                const uint64_t adesc = smem_desc_sw128(a_base + (uint32_t)m * 2u * w_box_bytes + (uint32_t)kk * 2048u,
-                                                       w_box_bytes, 1024u);
-                for (int j = 0; j < P.nt; ++j) {
-                  // B: rows of 128 bytes, 8-row groups of 1024 bytes; 16 k = 32 bytes along the row
-                  const uint64_t bdesc = smem_desc_sw128(b_base + (uint32_t)(j * P.n_tile) * 128u + (uint32_t)k16 * 32u,
-                                                         16u, 1024u);
-                  const uint32_t d_tmem = tmem_base + (uint32_t)acc * P.acc_cols + (uint32_t)((m * P.nt + j) * P.n_tile);
-                  umma_bf16(d_tmem, adesc, bdesc, idesc, (kb | k16) != 0 ? 1u : 0u);
+              const uint32_t accum = (kk == 0) ? (fresh ^ 1u) : 1u;
+#pragma unroll
+              for (int m = 0; m < kMaxUnits; ++m) {
+                if (m < width) {
+                  const uint64_t adesc = ((uint64_t)a_hi << 32) |
+                                         (a_lo_stage + (uint32_t)(m * 2 * (int)(w_box_bytes >> 4) + kk * 128));
+#pragma unroll
+                  for (int j = 0; j < NT; ++j) {
+                    const uint64_t bdesc = ((uint64_t)b_hi << 32) |
+                                           (b_lo_stage + (uint32_t)j * n_tile_u + (uint32_t)((sub * k16_per_stage + kk) * 2));
+                    umma_bf16(d_acc + (uint32_t)(m * NT + j) * n_tile, adesc, bdesc, idesc, accum);
+                  }
                 }
               }
             }
@@ -243,12 +266,12 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmapW, const __grid_consta
       tc_fence_after();
       for (int m = 0; m < width; ++m) {
         const int v = (unit0 + m) * (int)kTileM + q * 32 + lane;
-        for (int j = 0; j < P.nt; ++j) {
+        for (int j = 0; j < NT; ++j) {
           for (int c0 = 0; c0 < P.n_tile; c0 += 16) {
             const int t_first = j * P.n_tile + c0;
             if (t_first >= P.T) break;                       // warp-uniform
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * P.acc_cols +
-                                   (uint32_t)((m * P.nt + j) * P.n_tile + c0);
+                                   (uint32_t)((m * NT + j) * P.n_tile + c0);
             uint32_t r[16];
             tmem_ld16(taddr, r);
             tmem_ld_wait();
@@ -281,11 +304,18 @@ static int g_head_kw = 0;
 
 inline gs_status launch_lm_head_tc(const void* H, const void* W, float* logits, int T, int d, int V,
                                    int32_t* d_status, cudaStream_t st) {
+  using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const HeadTcParams);
+  static const KernelFn kernels[3][2] = {
+      {lm_head_tc_kernel<16, 1>, lm_head_tc_kernel<16, 2>},
+      {lm_head_tc_kernel<32, 1>, lm_head_tc_kernel<32, 2>},
+      {lm_head_tc_kernel<64, 1>, lm_head_tc_kernel<64, 2>}};
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(lm_head_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem) !=
-        cudaSuccess)
-      return GS_ERR_CUDA;
+    for (int a = 0; a < 3; ++a)
+      for (int b = 0; b < 2; ++b)
+        if (cudaFuncSetAttribute(kernels[a][b], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem) !=
+            cudaSuccess)
+          return GS_ERR_CUDA;
     attr_set = true;
   }
   const int sms = sm_count();
@@ -299,7 +329,7 @@ inline gs_status launch_lm_head_tc(const void* H, const void* W, float* logits, 
     P.n_tile = (((rows + P.nt - 1) / P.nt) + 15) / 16 * 16;
     const int total_n = P.nt * P.n_tile;
     // Widest tile (in units of 128 columns) whose accumulators fit the 512 TMEM columns.
-    int max_mt = min(512 / total_n, 9);
+    int max_mt = min(512 / total_n, kMaxUnits);
     if (g_head_mt > 0) max_mt = min(max_mt, g_head_mt);
     if (max_mt < 1) return GS_ERR_UNSUPPORTED;
     // Every SM gets the same number of tiles; tile widths differ by at most one unit.
@@ -335,7 +365,7 @@ inline gs_status launch_lm_head_tc(const void* H, const void* W, float* logits, 
     const size_t smem = 1024u + (size_t)stages * P.w_stage_bytes + (size_t)kHStages * P.h_stage_bytes +
                         8u * (2u * (uint32_t)stages + 2u * kHStages + 4u) + 64u;
     const int grid = min(P.num_tiles, sms);
-    lm_head_tc_kernel<<<grid, kTcThreads, smem, st>>>(tmapW, tmapH, P);
+    kernels[kw == 16 ? 0 : (kw == 32 ? 1 : 2)][P.nt - 1]<<<grid, kTcThreads, smem, st>>>(tmapW, tmapH, P);
     if (cudaGetLastError() != cudaSuccess) return GS_ERR_CUDA;
   }
   return GS_OK;
