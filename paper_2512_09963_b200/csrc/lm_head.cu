@@ -345,12 +345,17 @@ inline gs_status launch_lm_head_tc(const void* H, const void* W, float* logits, 
     uint32_t cols = 32;
     while (cols < (uint32_t)P.n_acc * P.acc_cols) cols <<= 1;
     P.tmem_cols = cols;
-    // k rows per W stage: wide tiles use shallow stages so that a stage is a few long rows.
-    const int kw = g_head_kw > 0 ? g_head_kw : (mt >= 4 ? 16 : (mt >= 2 ? 32 : 64));
-    P.kw = kw;
-    P.w_stage_bytes = (uint32_t)mt * 2u * (uint32_t)kw * 128u;
+    // k rows per W stage: the deepest stage that still leaves a ring of two (measured: fewer,
+    // larger TMA boxes and fewer barrier round trips beat a deeper ring of small stages).
     P.h_stage_bytes = (uint32_t)total_n * 128u;
     const uint32_t fixed = 1024u /*alignment*/ + (uint32_t)kHStages * P.h_stage_bytes + 8u * 64u + 64u;
+    int kw = g_head_kw;
+    if (kw <= 0) {
+      kw = 64;
+      while (kw > 16 && fixed + 2u * ((uint32_t)mt * 2u * (uint32_t)kw * 128u) > kMaxSmem) kw >>= 1;
+    }
+    P.kw = kw;
+    P.w_stage_bytes = (uint32_t)mt * 2u * (uint32_t)kw * 128u;
     if (fixed + 2 * P.w_stage_bytes > kMaxSmem) return GS_ERR_UNSUPPORTED;
     int stages = (int)((kMaxSmem - fixed) / P.w_stage_bytes);
     if (stages > 24) stages = 24;
