@@ -1,0 +1,453 @@
+#!/usr/bin/env python
+"""Benchmark of one GoodSpeed verification round on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config cfg2]
+
+A step is one pass of the whole hot path (verify attention, LM head, acceptance + estimator
+update, next allocation) over one batch of synthetic drafts.  The default workload is the
+Qwen3-32B-shaped configuration (8 servers, prefix 2048, d=5120, V=151936, bf16).  Rank 0 prints
+one JSON line.  `--impl reference` times the fp64 CPU oracle instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import dataclasses
+import hashlib
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+sys.path.insert(0, os.path.join(ROOT, "tests"))
+
+from paper_2512_09963_b200 import workloads as wl  # noqa: E402
+
+METRIC = "verified tokens/sec per verify step"
+UNIT = "tokens/s"
+FALLBACK_HBM_GBS = 6650.0
+ETA, BETA = 0.1, 0.5
+
+# DRAM traffic of the LM-head kernel from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum
+# per launch), keyed by the sha256 of the kernel source it was taken on; a changed kernel reports null.
+# cfg2's full launch is within ncu's single-pass size rule only for the launch list, so the counters
+# were taken on a smaller vocabulary and scale with the units processed (see profiles/).
+NCU_TRAFFIC = {}
+
+
+def _kernel_hash():
+    h = hashlib.sha256()
+    for f in ("lm_head.cu", "sm100_ptx.cuh"):
+        h.update(open(os.path.join(ROOT, "paper_2512_09963_b200", "csrc", f), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return float(p["hbm_gbs"]), "measured", p
+    return FALLBACK_HBM_GBS, "fallback", {}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.samples = []
+        self.proc = None
+        try:
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", uuid, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append((time.time(), line.strip()))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        rows = [s for t, s in self.samples if t0 - 0.05 <= t <= t1 + 0.15] or [s for _, s in self.samples]
+        sm, mx, reasons, power = [], [], set(), []
+        for r in rows:
+            f = [x.strip() for x in r.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); power.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def subset_servers(inp, n_srv):
+    """The first n_srv servers of a step's inputs (host tensors): a bounded sample for the CPU oracle."""
+    cu_q, cu_kv = inp["cu_q"].numpy(), inp["cu_kv"].numpy()
+    q1, k1 = int(cu_q[n_srv]), int(cu_kv[n_srv])
+    g1 = q1 - n_srv
+    out = dict(inp)
+    out.update(Q=inp["Q"][:q1], H=inp["H"][:q1], K=inp["K"][:k1], V=inp["V"][:k1],
+               cu_q=inp["cu_q"][:n_srv + 1], cu_kv=inp["cu_kv"][:n_srv + 1],
+               q_probs=inp["q_probs"][:g1], draft_tok=inp["draft_tok"][:g1], u_accept=inp["u_accept"][:g1],
+               u_sample=inp["u_sample"][:n_srv], gamma=inp["gamma"][:n_srv])
+    return out
+
+
+def oracle_round(inp, N, C):
+    from oracle import goodspeed_oracle as orc
+    host = dict(inp)
+    host["tau"] = float(np.float32(inp["tau"]))
+    return orc.ref_verify_round(host, np.full(N, 0.5), np.ones(N), ETA, BETA, C)
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 0) for p in threadpool_info()]
+        return max(n) if n else os.cpu_count()
+    except Exception:
+        return os.cpu_count()
+
+
+def library_allocator(device):
+    """Budgeted allocation for workloads whose draft lengths come from a scheduler run: the
+    library's own gs_schedule (bit-identical to the oracle's greedy, see the GPU tests)."""
+    def alloc(X, alpha_hat, C, s_min, s_max):
+        from paper_2512_09963_b200 import binding as B
+        t = lambda a, dt: torch.as_tensor(np.asarray(a), dtype=dt, device=device)
+        S = torch.empty(len(X), dtype=torch.int32, device=device)
+        B.gs_schedule(t(X, torch.float64), t(alpha_hat, torch.float64), C, S, t(s_min, torch.int32),
+                      t(s_max, torch.int32))
+        torch.cuda.synchronize()
+        return S.cpu().numpy()
+    return alloc
+
+
+def make_host_inputs(cfg, device):
+    alloc = library_allocator(device) if cfg.gamma_mode == "alloc" else None
+    dev_inp = wl.make_step(cfg, device=device, allocator=alloc)
+    host = {k: (v.cpu() if isinstance(v, torch.Tensor) else v) for k, v in dev_inp.items()}
+    return dev_inp, host
+
+
+# ------------------------------------------------------------------------------------------------
+def run_reference(args, cfg, rank, world):
+    """The CPU oracle as it stands, on a bounded sample of the same workload."""
+    if rank != 0:
+        return
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    _, host = make_host_inputs(cfg, dev)
+    if dev == "cuda":
+        torch.cuda.empty_cache()
+    C = 8 * cfg.N
+    t0 = time.time()
+    oracle_round(subset_servers(host, 1), 1, 8)            # calibration: one server
+    t1 = time.time() - t0
+    budget = 150.0 / max(1, args.steps + args.warmup)      # seconds per step
+    n_srv = int(max(1, min(cfg.N, budget // max(t1, 1e-3))))
+    sample = subset_servers(host, n_srv)
+    gamma = int(sample["gamma"].sum())
+    for _ in range(args.warmup):
+        oracle_round(sample, n_srv, C)
+    t0 = time.time()
+    for _ in range(args.steps):
+        oracle_round(sample, n_srv, C)
+    dt = (time.time() - t0) / max(1, args.steps)
+    val = gamma / dt
+    cores = blas_threads()
+    desc = f"servers 0..{n_srv - 1} of {cfg.N} ({gamma} draft tokens): their attention, LM-head rows against the full W, acceptance, estimators, schedule"
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name, "note": "fp64 CPU oracle on host cores"},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------
+def run_ours(args, cfg, rank, world, local_rank):
+    from paper_2512_09963_b200 import binding as B
+    from paper_2512_09963_b200 import build as gs_build
+    from paper_2512_09963_b200.runner import VerifyRound
+    import torch.distributed as dist
+
+    if rank == 0:
+        gs_build.build()
+    if world > 1:
+        dist.barrier()
+    B.lib()
+    dev = torch.device("cuda", local_rank)
+    cfg_r = dataclasses.replace(cfg, seed_tag=f"/rank{rank}") if world > 1 else cfg
+    inp, host = make_host_inputs(cfg_r, dev)
+    N, Tq = cfg.N, int(inp["cu_q"][-1])
+    Gamma = int(inp["gamma"].sum())
+    C = 8 * N
+    rnd = VerifyRound.for_inputs(inp, C=C, eta=ETA, beta=BETA)
+    s_min = torch.ones(N * world, dtype=torch.int32, device=dev)
+    s_max = torch.full((N * world,), 8, dtype=torch.int32, device=dev)
+    # multi-GPU: servers are sharded over ranks; only the scheduler couples them, through an
+    # all-gather of the estimator state (16 bytes per server) before every rank runs the same greedy.
+    if world > 1:
+        est_local = torch.empty(2 * N, dtype=torch.float64, device=dev)
+        est_all = torch.empty(2 * N * world, dtype=torch.float64, device=dev)
+        X_all = torch.empty(N * world, dtype=torch.float64, device=dev)
+        a_all = torch.empty(N * world, dtype=torch.float64, device=dev)
+        S_all = torch.empty(N * world, dtype=torch.int32, device=dev)
+
+    def reset_state():
+        rnd.alpha_hat.fill_(0.5)
+        rnd.X.fill_(1.0)
+
+    def step():
+        rnd.attn(inp["Q"], inp["K"], inp["V"], inp["cu_q"], inp["cu_kv"])
+        rnd.head(inp["H"], inp["W"])
+        rnd.accept(inp["q_probs"], inp["draft_tok"], inp["cu_q"], inp["u_accept"], inp["u_sample"], inp["tau"])
+        if world == 1:
+            rnd.schedule(s_min, s_max)
+        else:
+            est_local[:N].copy_(rnd.alpha_hat)
+            est_local[N:].copy_(rnd.X)
+            dist.all_gather_into_tensor(est_all, est_local)
+            g = est_all.view(world, 2, N)
+            a_all.copy_(g[:, 0, :].reshape(-1))
+            X_all.copy_(g[:, 1, :].reshape(-1))
+            B.gs_schedule(X_all, a_all, C * world, S_all, s_min, s_max, rnd.d_status)
+            rnd.S_next.copy_(S_all[rank * N:(rank + 1) * N])
+
+    # ---- launches per step and a first (eager) run
+    reset_state()
+    c0 = B.gs_launch_count()
+    step()
+    torch.cuda.synchronize()
+    launches_per_step = B.gs_launch_count() - c0
+    assert int(rnd.d_status.item()) == 0, "device status after the first step"
+    first = {k: getattr(rnd, k).clone() for k in ("accepted", "out_tok", "n_out", "S_next")}
+
+    # ---- CUDA graph of one step (single GPU only)
+    graph = None
+    if world == 1 and not args.no_graph:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            step()
+        torch.cuda.current_stream().wait_stream(side)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            step()
+    run_step = graph.replay if graph is not None else step
+
+    # ---- timed region: W warm-up steps, then exactly K steps between barriers/synchronisations
+    for _ in range(args.warmup):
+        run_step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t_wall0 = time.time()
+    e0.record()
+    for _ in range(args.steps):
+        run_step()
+    e1.record()
+    torch.cuda.synchronize()
+    t_wall1 = time.time()
+    if world > 1:
+        dist.barrier()
+    ms_total = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+        g = torch.tensor([Gamma], dtype=torch.int64, device=dev)
+        dist.all_reduce(g)
+        gamma_all = int(g.item())
+    else:
+        gamma_all = Gamma
+    ms_step = ms_total / args.steps
+    clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
+
+    # ---- per-kernel durations (eager, CUDA events between the calls of the same step sequence)
+    n_k = min(args.steps, 30)
+    names = ("verify_attn", "lm_head_logits", "spec_accept", "gs_schedule")
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(n_k)]
+    for i in range(n_k):
+        evs[i][0].record()
+        rnd.attn(inp["Q"], inp["K"], inp["V"], inp["cu_q"], inp["cu_kv"]); evs[i][1].record()
+        rnd.head(inp["H"], inp["W"]); evs[i][2].record()
+        rnd.accept(inp["q_probs"], inp["draft_tok"], inp["cu_q"], inp["u_accept"], inp["u_sample"], inp["tau"])
+        evs[i][3].record()
+        rnd.schedule(s_min[:N], s_max[:N]); evs[i][4].record()
+    torch.cuda.synchronize()
+    k_us = {n: float(np.mean([evs[i][j].elapsed_time(evs[i][j + 1]) for i in range(n_k)])) * 1e3
+            for j, n in enumerate(names)}
+
+    if rank != 0:
+        return
+    # ---- rooflines
+    peak, peak_kind, peaks = _peaks()
+    d, V = cfg.d, cfg.V
+    es = 2 if cfg.dtype == "bf16" else 4
+    total_kv = int(inp["K"].shape[0])
+    bytes_head = d * V * es + Tq * V * 4 + Tq * d * es
+    bytes_attn = 2 * total_kv * cfg.Hkv * cfg.hd * es + 2 * Tq * cfg.Hq * cfg.hd * es
+    bytes_acc = Tq * V * 4 + N * V * 8
+    flops_head = 2.0 * Tq * d * V
+    ach = bytes_head / (k_us["lm_head_logits"] * 1e-6) / 1e9
+    khash = _kernel_hash()
+    roofline = {"kernel": "lm_head_tc_kernel", "bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s",
+                "frac": ach / peak, "peak_source": f"{peak_kind} (MEASURED_PEAKS.json hbm_gbs)" if peak_kind == "measured"
+                else "fallback 6650 GB/s", "traffic": NCU_TRAFFIC.get(khash, {}).get(cfg.name),
+                "algorithmic_bytes": bytes_head, "duration_us": k_us["lm_head_logits"],
+                "tensor_tflops": flops_head / (k_us["lm_head_logits"] * 1e-6) / 1e12}
+    kernels = {
+        "verify_attn": {"us": k_us["verify_attn"], "algorithmic_bytes": bytes_attn,
+                        "gbs": bytes_attn / k_us["verify_attn"] / 1e3, "frac_hbm": bytes_attn / k_us["verify_attn"] / 1e3 / peak},
+        "lm_head_logits": {"us": k_us["lm_head_logits"], "algorithmic_bytes": bytes_head, "gbs": ach, "frac_hbm": ach / peak},
+        "spec_accept": {"us": k_us["spec_accept"], "algorithmic_bytes": bytes_acc,
+                        "gbs": bytes_acc / k_us["spec_accept"] / 1e3, "frac_hbm": bytes_acc / k_us["spec_accept"] / 1e3 / peak},
+        "gs_schedule": {"us": k_us["gs_schedule"]},
+    }
+
+    # ---- end to end through the host-buffer entry point (pinned inputs, results read back each step)
+    e2e = None
+    if world == 1:
+        desc = B.RoundDesc(N=N, Tq=Tq, total_kv=total_kv, max_kv_len=rnd.max_kv_len, Hq=cfg.Hq, Hkv=cfg.Hkv,
+                           hd=cfg.hd, d=d, V=V, C=C, dt=B.GS_BF16 if cfg.dtype == "bf16" else B.GS_F32,
+                           scale=cfg.hd ** -0.5, temperature=float(inp["tau"]), eta=ETA, beta=BETA,
+                           alpha_min=1e-3, alpha_max=0.999)
+        ws = torch.empty(B.gs_verify_round_workspace(desc), dtype=torch.uint8, device=dev)
+        pin = {k: host[k].contiguous().pin_memory() for k in
+               ("Q", "H", "q_probs", "draft_tok", "u_accept", "u_sample", "cu_q", "cu_kv")}
+        outs = {k: torch.empty(n, dtype=torch.int32).pin_memory() for k, n in
+                (("accepted", N), ("out_tok", Tq), ("n_out", N), ("S_next", N), ("status", 1))}
+        h2d = sum(t.numel() * t.element_size() for t in pin.values())
+        d2h = sum(t.numel() * t.element_size() for t in outs.values())
+
+        def e2e_step():
+            B.gs_verify_round_host(desc, pin["Q"], pin["H"], pin["q_probs"], pin["draft_tok"], pin["u_accept"],
+                                   pin["u_sample"], pin["cu_q"], pin["cu_kv"], inp["K"], inp["V"], inp["W"],
+                                   rnd.alpha_hat, rnd.X, s_min, s_max, ws, outs["accepted"], outs["out_tok"],
+                                   outs["n_out"], outs["S_next"], outs["status"])
+            torch.cuda.current_stream().synchronize()
+
+        reset_state()
+        e2e_step()
+        e2e_ok = (int(outs["status"][0]) == 0 and torch.equal(outs["accepted"], first["accepted"].cpu())
+                  and torch.equal(outs["out_tok"], first["out_tok"].cpu()))
+        n_e = min(args.steps, 30)
+        for _ in range(3):
+            e2e_step()
+        t0 = time.time()
+        for _ in range(n_e):
+            e2e_step()
+        dt = (time.time() - t0) / n_e
+        e2e = {"value": Gamma / dt, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "ms_per_step": dt * 1e3, "matches_device_path": bool(e2e_ok)}
+
+    # ---- CPU baseline = the oracle on the host cores, and a parity check of this launch configuration
+    cpu = None
+    parity = None
+    if world == 1 and not args.skip_cpu_baseline:
+        import parity_utils as pu
+        t0 = time.time()
+        ref = oracle_round(host, N, C)
+        dt = time.time() - t0
+        cpu = {"value": Gamma / dt, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "seconds": dt,
+               "sample": f"the whole {cfg.name} step once ({Gamma} draft tokens, {Tq} verify positions)"}
+        got = {k: first[k].cpu().numpy() for k in ("accepted", "out_tok", "n_out")}
+        reset_state()
+        step()
+        torch.cuda.synchronize()
+        got.update(ratio=rnd.ratio.cpu().numpy(), p_tok=rnd.p_tok.cpu().numpy())
+        tau = float(np.float32(inp["tau"]))
+        try:
+            pu.assert_close_rel(rnd.O, ref["O"], "attention")
+            pu.assert_close_rel(rnd.logits, ref["logits"], "logits")
+            slack = pu.chain_slack(rnd.logits, ref["logits"], tau)
+            log = pu.compare_accept(got, ref, ref["logits"], host["q_probs"], host["cu_q"].numpy(),
+                                    host["u_sample"], tau, V, slack=slack)
+            parity = {"status": "ok", "accept_near_ties": len(log["accept_near_ties"]),
+                      "sample_near_ties": len(log["sample_near_ties"]), "sample_exact": log["sample_exact"]}
+        except AssertionError as ex:
+            parity = {"status": "FAILED", "detail": str(ex)[:300]}
+
+    goodput = float(first["n_out"].sum().item()) * world / (ms_step * 1e-3)
+    line = {
+        "metric": METRIC, "value": gamma_all / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+        "config": {"workload": cfg.name, "servers_per_gpu": N, "draft_tokens_per_gpu": Gamma, "verify_positions": Tq,
+                   "prefix": int(inp["prefix"][0]), "d": d, "V": V, "heads": f"{cfg.Hq}q/{cfg.Hkv}kv x {cfg.hd}",
+                   "temperature": float(inp["tau"]), "parallelism": f"dp{world} over draft servers",
+                   "l2": "inputs larger than L2: the 1.56 GB head weight streams through L2 every step and evicts the KV cache and logits",
+                   "launch": "CUDA graph replay of the four calls" if graph is not None else "eager, four calls per step"},
+        "goodput_tokens_per_s": goodput,
+        "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu, "e2e": e2e,
+        "gpu_launches": int(launches_per_step) * args.steps, "launches_per_step": int(launches_per_step),
+        "clocks": clocks, "parity_vs_oracle": parity, "kernel_source_hash": khash,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="cfg2", choices=["cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--skip-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    cfg = wl.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, cfg, rank, world)
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    try:
+        run_ours(args, cfg, rank, world, local_rank)
+    finally:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

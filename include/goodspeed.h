@@ -164,6 +164,46 @@ gs_status gs_schedule(const double* X, const double* alpha_hat, int N, int C,
                       const int32_t* s_min, const int32_t* s_max, int32_t* S_out,
                       int32_t* d_status, void* stream);
 
+/* --------------------------------------------------------------------------------------------
+ * gs_verify_round_host -- Algorithm 1, the verification-server steps of one round (batching,
+ * verification, estimator update, GoodSpeed-sched), for a caller whose per-round data is in HOST
+ * memory: what the draft servers sent (draft tokens, full draft distributions, Alg. 1 "Send
+ * s_i(t), q_{i,j}") plus the hidden states and queries of the new positions.  The KV caches, the
+ * head weight and the estimator state stay resident on the device.
+ *
+ *   h_*      host pointers (pinned memory lets the copies overlap); shapes as in the calls above
+ *   d_K,d_V  [total_kv, Hkv, hd], d_W [d, V]: device, resident; d_alpha_hat, d_X [N] fp64 device,
+ *            updated in place; d_s_min/d_s_max [N] int32 device, nullable
+ *   d_ws     device scratch of gs_verify_round_workspace() bytes, 256-aligned; it also holds the
+ *            attention output O and the logits of the round
+ *   outputs  h_accepted[N], h_out_tok[T_q], h_n_out[N], h_S_next[N], h_status[1] (device status)
+ * The call enqueues host->device copies, gs_verify_attn, gs_lm_head_logits, gs_spec_accept (with
+ * the estimator update), gs_schedule and the device->host copies on `stream` and returns; the host
+ * outputs are valid after the caller synchronises the stream.  Host buffers must stay untouched
+ * until then.  Errors: as the four calls; CUDA if a copy could not be enqueued.
+ */
+typedef struct gs_round_desc {
+  int N, Tq, total_kv, max_kv_len, Hq, Hkv, hd, d, V, C;
+  gs_dtype dt;
+  float scale, temperature;
+  double eta, beta, alpha_min, alpha_max;
+} gs_round_desc;
+
+size_t gs_verify_round_workspace(const gs_round_desc* r);
+gs_status gs_verify_round_host(const gs_round_desc* r,
+                               const void* h_Q, const void* h_H, const float* h_q_probs,
+                               const int32_t* h_draft_tok, const float* h_u_accept, const float* h_u_sample,
+                               const int32_t* h_cu_q, const int32_t* h_cu_kv,
+                               const void* d_K, const void* d_V, const void* d_W,
+                               double* d_alpha_hat, double* d_X,
+                               const int32_t* d_s_min, const int32_t* d_s_max,
+                               void* d_ws, size_t ws_bytes,
+                               int32_t* h_accepted, int32_t* h_out_tok, int32_t* h_n_out,
+                               int32_t* h_S_next, int32_t* h_status, void* stream);
+
+/* Number of CUDA kernels the library has launched so far in this process (host-side counter). */
+unsigned long long gs_launch_count(void);
+
 #ifdef __cplusplus
 }
 #endif

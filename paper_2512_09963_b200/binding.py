@@ -37,7 +37,17 @@ SIGNATURES = {
                             _vp, _vp, _vp, _vp, _vp, _vp,
                             _vp, _vp, _d, _d, _d, _d, _vp, _sz, _vp, _vp]),
     "gs_schedule": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp]),
+    "gs_verify_round_workspace": (_sz, [_vp]),
+    "gs_verify_round_host": (_i, [_vp] + [_vp] * 8 + [_vp] * 7 + [_vp, _sz] + [_vp] * 5 + [_vp]),
+    "gs_launch_count": (C.c_ulonglong, []),
 }
+
+
+class RoundDesc(C.Structure):
+    """Mirror of gs_round_desc."""
+    _fields_ = [("N", _i), ("Tq", _i), ("total_kv", _i), ("max_kv_len", _i), ("Hq", _i), ("Hkv", _i),
+                ("hd", _i), ("d", _i), ("V", _i), ("C", _i), ("dt", _i), ("scale", _f), ("temperature", _f),
+                ("eta", _d), ("beta", _d), ("alpha_min", _d), ("alpha_max", _d)]
 
 _lib = None
 
@@ -163,3 +173,31 @@ def gs_schedule(X, alpha_hat, C_budget, S_out, s_min=None, s_max=None, d_status=
     code = lib().gs_schedule(_ptr(X, f64), _ptr(alpha_hat, f64), N, int(C_budget), _ptr(s_min, i32),
                              _ptr(s_max, i32), _ptr(S_out, i32), _ptr(d_status, i32), _stream())
     _check("gs_schedule", code)
+
+
+def gs_launch_count() -> int:
+    return int(lib().gs_launch_count())
+
+
+def gs_verify_round_workspace(desc: RoundDesc) -> int:
+    return lib().gs_verify_round_workspace(C.byref(desc))
+
+
+def gs_verify_round_host(desc: RoundDesc, h_Q, h_H, h_q_probs, h_draft_tok, h_u_accept, h_u_sample,
+                         h_cu_q, h_cu_kv, d_K, d_V, d_W, d_alpha_hat, d_X, d_s_min, d_s_max, d_ws,
+                         h_accepted, h_out_tok, h_n_out, h_S_next, h_status):
+    """Host tensors (h_*) must be CPU tensors, ideally pinned; d_* are CUDA tensors."""
+    i32, f32, f64 = torch.int32, torch.float32, torch.float64
+    hp = lambda t, dt=None: _ptr(t, dt, cuda=False)
+    for t in (h_Q, h_H, h_q_probs, h_draft_tok, h_u_accept, h_u_sample, h_cu_q, h_cu_kv,
+              h_accepted, h_out_tok, h_n_out, h_S_next, h_status):
+        if t is not None and t.is_cuda:
+            raise ValueError("h_* tensors must live in host memory")
+    code = lib().gs_verify_round_host(
+        C.byref(desc), hp(h_Q), hp(h_H), hp(h_q_probs, f32), hp(h_draft_tok, i32), hp(h_u_accept, f32),
+        hp(h_u_sample, f32), hp(h_cu_q, i32), hp(h_cu_kv, i32),
+        _ptr(d_K), _ptr(d_V), _ptr(d_W), _ptr(d_alpha_hat, f64), _ptr(d_X, f64), _ptr(d_s_min, i32),
+        _ptr(d_s_max, i32), _ptr(d_ws), d_ws.numel() * d_ws.element_size(),
+        hp(h_accepted, i32), hp(h_out_tok, i32), hp(h_n_out, i32), hp(h_S_next, i32), hp(h_status, i32),
+        _stream())
+    _check("gs_verify_round_host", code)

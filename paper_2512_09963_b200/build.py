@@ -8,7 +8,7 @@ import sys
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libgoodspeed.so")
-SOURCES = ["api.cu", "spec_accept.cu", "schedule.cu", "verify_attn.cu", "lm_head.cu"]
+SOURCES = ["api.cu", "spec_accept.cu", "schedule.cu", "verify_attn.cu", "lm_head.cu", "round.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--expt-relaxed-constexpr", "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall"]
 

@@ -1,4 +1,12 @@
 #include "common.cuh"
+#include <atomic>
+
+namespace gs {
+static std::atomic<unsigned long long> g_launches{0};
+void count_launches(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+}  // namespace gs
+
+extern "C" unsigned long long gs_launch_count(void) { return gs::g_launches.load(std::memory_order_relaxed); }
 
 extern "C" const char* gs_status_str(gs_status s) {
   switch (s) {

@@ -113,6 +113,7 @@ inline gs_status launch_attn_generic(const void* Q, const void* K, const void* V
   attn_generic_kernel<T><<<grid, kGenAttnThreads, smem, st>>>(
       static_cast<const T*>(Q), static_cast<const T*>(K), static_cast<const T*>(V), static_cast<T*>(O),
       cu_q, cu_kv, N, Tq, total_kv, max_kv_len, Hq, Hkv, hd, scale, d_status);
+  count_launches(1);
   return launch_status();
 }
 

@@ -22,6 +22,9 @@ GS_DEVINL void set_status(int32_t* st, int code) {
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Number of kernels this library has launched (host-side count, all threads).
+void count_launches(int n);
+
 inline gs_status launch_status() {
   return cudaGetLastError() == cudaSuccess ? GS_OK : GS_ERR_CUDA;
 }

@@ -68,6 +68,7 @@ inline gs_status launch_lm_head_plain(const void* H, const void* W, float* logit
   dim3 grid((V + kHeadCols - 1) / kHeadCols, (T_ + kHeadRows - 1) / kHeadRows);
   lm_head_plain_kernel<T><<<grid, kHeadCols, 0, st>>>(static_cast<const T*>(H), static_cast<const T*>(W),
                                                      logits, T_, d, V);
+  count_launches(1);
   return launch_status();
 }
 
@@ -372,6 +373,7 @@ inline gs_status launch_lm_head_tc(const void* H, const void* W, float* logits, 
     const int grid = min(P.num_tiles, sms);
     kernels[kw == 16 ? 0 : (kw == 32 ? 1 : 2)][P.nt - 1]<<<grid, kTcThreads, smem, st>>>(tmapW, tmapH, P);
     if (cudaGetLastError() != cudaSuccess) return GS_ERR_CUDA;
+    count_launches(1);
   }
   return GS_OK;
 }

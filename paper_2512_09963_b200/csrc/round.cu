@@ -1,0 +1,121 @@
+// gs_verify_round_host: one whole verification round for a caller whose per-round data lives in
+// host memory (what the draft servers sent this round), with the model state resident on the GPU.
+// It stages the inputs with cudaMemcpyAsync, enqueues the four steps of the round on the same
+// stream and copies the small results back; nothing here computes.
+#include "common.cuh"
+
+namespace gs {
+
+struct RoundLayout {
+  size_t Q, H, q_probs, draft_tok, u_accept, u_sample, cu_q, cu_kv;     // staged inputs
+  size_t O, logits, accepted, out_tok, n_out, ratio, p_tok, S_next, status;
+  size_t ws_attn, ws_head, ws_acc;
+  size_t ws_attn_bytes, ws_head_bytes, ws_acc_bytes;
+  size_t total;
+};
+
+static size_t esize(gs_dtype dt) { return dt == GS_F32 ? 4 : 2; }
+
+static RoundLayout round_layout(const gs_round_desc& r) {
+  RoundLayout L;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + (bytes ? bytes : 1), 256); return o; };
+  const size_t Tq = (size_t)r.Tq, N = (size_t)r.N, Gamma = Tq - N, V = (size_t)r.V;
+  L.Q = take(Tq * r.Hq * r.hd * esize(r.dt));
+  L.H = take(Tq * r.d * esize(r.dt));
+  L.q_probs = take(Gamma * V * 4);
+  L.draft_tok = take(Gamma * 4);
+  L.u_accept = take(Gamma * 4);
+  L.u_sample = take(N * 4);
+  L.cu_q = take((N + 1) * 4);
+  L.cu_kv = take((N + 1) * 4);
+  L.O = take(Tq * r.Hq * r.hd * esize(r.dt));
+  L.logits = take(Tq * V * 4);
+  L.accepted = take(N * 4);
+  L.out_tok = take(Tq * 4);
+  L.n_out = take(N * 4);
+  L.ratio = take(Gamma * 4);
+  L.p_tok = take(Gamma * 4);
+  L.S_next = take(N * 4);
+  L.status = take(4);
+  L.ws_attn_bytes = gs_verify_attn_workspace(r.N, r.Tq, r.total_kv, r.max_kv_len, r.Hq, r.Hkv, r.hd, r.dt);
+  L.ws_head_bytes = gs_lm_head_workspace(r.Tq, r.d, r.V, r.dt);
+  L.ws_acc_bytes = gs_spec_accept_workspace(r.N, r.Tq, r.V);
+  L.ws_attn = take(L.ws_attn_bytes);
+  L.ws_head = take(L.ws_head_bytes);
+  L.ws_acc = take(L.ws_acc_bytes);
+  L.total = off;
+  return L;
+}
+
+static bool desc_ok(const gs_round_desc* r) {
+  return r != nullptr && r->N > 0 && r->Tq >= r->N && r->total_kv > 0 && r->max_kv_len > 0 && r->Hq > 0 &&
+         r->Hkv > 0 && r->hd > 0 && r->d > 0 && r->V > 0 && r->C >= 0 && (r->dt == GS_F32 || r->dt == GS_BF16);
+}
+
+}  // namespace gs
+
+extern "C" size_t gs_verify_round_workspace(const gs_round_desc* r) {
+  if (!gs::desc_ok(r)) return 0;
+  return gs::round_layout(*r).total;
+}
+
+extern "C" gs_status gs_verify_round_host(const gs_round_desc* r,
+                                          const void* h_Q, const void* h_H, const float* h_q_probs,
+                                          const int32_t* h_draft_tok, const float* h_u_accept,
+                                          const float* h_u_sample, const int32_t* h_cu_q, const int32_t* h_cu_kv,
+                                          const void* d_K, const void* d_V, const void* d_W,
+                                          double* d_alpha_hat, double* d_X,
+                                          const int32_t* d_s_min, const int32_t* d_s_max,
+                                          void* d_ws, size_t ws_bytes,
+                                          int32_t* h_accepted, int32_t* h_out_tok, int32_t* h_n_out,
+                                          int32_t* h_S_next, int32_t* h_status, void* stream) {
+  using namespace gs;
+  if (!desc_ok(r)) return GS_ERR_INVALID_ARG;
+  const size_t Gamma = (size_t)(r->Tq - r->N);
+  if (!h_Q || !h_H || !h_u_sample || !h_cu_q || !h_cu_kv || !d_K || !d_V || !d_W || !d_alpha_hat || !d_X ||
+      !h_accepted || !h_out_tok || !h_n_out || !h_S_next || !h_status)
+    return GS_ERR_INVALID_ARG;
+  if (Gamma > 0 && (!h_q_probs || !h_draft_tok || !h_u_accept)) return GS_ERR_INVALID_ARG;
+  if (d_ws == nullptr || (reinterpret_cast<uintptr_t>(d_ws) & 255u) != 0) return GS_ERR_WORKSPACE;
+  const RoundLayout L = round_layout(*r);
+  if (ws_bytes < L.total) return GS_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* w = static_cast<char*>(d_ws);
+  const size_t Tq = (size_t)r->Tq, N = (size_t)r->N, V = (size_t)r->V, es = esize(r->dt);
+  auto h2d = [&](size_t off, const void* src, size_t bytes) {
+    return bytes == 0 || cudaMemcpyAsync(w + off, src, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  };
+  auto d2h = [&](void* dst, size_t off, size_t bytes) {
+    return cudaMemcpyAsync(dst, w + off, bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  };
+  bool ok = h2d(L.Q, h_Q, Tq * r->Hq * r->hd * es) && h2d(L.H, h_H, Tq * r->d * es) &&
+            h2d(L.q_probs, h_q_probs, Gamma * V * 4) && h2d(L.draft_tok, h_draft_tok, Gamma * 4) &&
+            h2d(L.u_accept, h_u_accept, Gamma * 4) && h2d(L.u_sample, h_u_sample, N * 4) &&
+            h2d(L.cu_q, h_cu_q, (N + 1) * 4) && h2d(L.cu_kv, h_cu_kv, (N + 1) * 4);
+  if (!ok || cudaMemsetAsync(w + L.status, 0, 4, st) != cudaSuccess) return GS_ERR_CUDA;
+  int32_t* d_status = reinterpret_cast<int32_t*>(w + L.status);
+  const int32_t* cu_q = reinterpret_cast<const int32_t*>(w + L.cu_q);
+  const int32_t* cu_kv = reinterpret_cast<const int32_t*>(w + L.cu_kv);
+  gs_status s = gs_verify_attn(w + L.Q, d_K, d_V, w + L.O, cu_q, cu_kv, r->N, r->Tq, r->total_kv, r->max_kv_len,
+                               r->Hq, r->Hkv, r->hd, r->scale, r->dt, w + L.ws_attn, L.ws_attn_bytes, d_status, st);
+  if (s != GS_OK) return s;
+  s = gs_lm_head_logits(w + L.H, d_W, reinterpret_cast<float*>(w + L.logits), r->Tq, r->d, r->V, r->dt,
+                        w + L.ws_head, L.ws_head_bytes, d_status, st);
+  if (s != GS_OK) return s;
+  s = gs_spec_accept(reinterpret_cast<const float*>(w + L.logits), reinterpret_cast<const float*>(w + L.q_probs),
+                     reinterpret_cast<const int32_t*>(w + L.draft_tok), cu_q,
+                     reinterpret_cast<const float*>(w + L.u_accept), reinterpret_cast<const float*>(w + L.u_sample),
+                     r->temperature, r->N, r->Tq, r->V,
+                     reinterpret_cast<int32_t*>(w + L.accepted), reinterpret_cast<int32_t*>(w + L.out_tok),
+                     reinterpret_cast<int32_t*>(w + L.n_out), reinterpret_cast<float*>(w + L.ratio),
+                     reinterpret_cast<float*>(w + L.p_tok), nullptr, d_alpha_hat, d_X, r->eta, r->beta,
+                     r->alpha_min, r->alpha_max, w + L.ws_acc, L.ws_acc_bytes, d_status, st);
+  if (s != GS_OK) return s;
+  s = gs_schedule(d_X, d_alpha_hat, r->N, r->C, d_s_min, d_s_max, reinterpret_cast<int32_t*>(w + L.S_next),
+                  d_status, st);
+  if (s != GS_OK) return s;
+  ok = d2h(h_accepted, L.accepted, N * 4) && d2h(h_out_tok, L.out_tok, Tq * 4) && d2h(h_n_out, L.n_out, N * 4) &&
+       d2h(h_S_next, L.S_next, N * 4) && d2h(h_status, L.status, 4);
+  return ok ? GS_OK : GS_ERR_CUDA;
+}

@@ -97,5 +97,6 @@ extern "C" gs_status gs_schedule(const double* X, const double* alpha_hat, int N
   const int threads = (N + 31) / 32 * 32;
   gs::schedule_kernel<<<1, threads, 0, static_cast<cudaStream_t>(stream)>>>(
       X, alpha_hat, N, C, s_min, s_max, S_out, d_status);
+  gs::count_launches(1);
   return gs::launch_status();
 }

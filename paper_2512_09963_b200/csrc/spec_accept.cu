@@ -474,5 +474,6 @@ extern "C" gs_status gs_spec_accept(const float* logits, const float* q_probs, c
   S.N = N; S.V = V; S.n_chunk = n_chunk; S.Gamma = Gamma; S.k2 = k2;
   S.sel = w.sel; S.mass = w.mass; S.out_tok = out_tok; S.margin = margin;
   sa_sample<<<N, kSaThreads, 0, st>>>(S);
+  count_launches(k2 > 0.f ? 4 : 3);
   return launch_status();
 }
