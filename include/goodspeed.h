@@ -71,8 +71,11 @@ int gs_version(void);
  *   dt: GS_F32 (fp32 in/out) or GS_BF16 (bf16 in/out); scores, softmax and accumulation fp32.
  *   max_kv_len: an upper bound on any server's cu_kv[i+1]-cu_kv[i] (sizes the split-KV scratch).
  *   scale: multiplies q.k (pass 1/sqrt(hd)).
- * Errors: INVALID_ARG (null/negative), SHAPE (Hq % Hkv != 0), UNSUPPORTED (hd > 256 for
- * GS_F32; for GS_BF16 hd must be 64 or 128 and Hq/Hkv <= 16), WORKSPACE.
+ * GS_BF16 with hd = 128 and a group size Hq/Hkv that divides 128 runs on the tensor cores
+ * (tcgen05, split over the KV length, partial results merged from the workspace); every other
+ * shape runs a plain kernel.
+ * Errors: INVALID_ARG (null/negative), SHAPE (Hq % Hkv != 0), UNSUPPORTED (hd > 256, T_q > 65535),
+ * WORKSPACE.
  * Device status: GS_ERR_SHAPE if a server has fewer keys than new positions, more keys than
  * max_kv_len, or offsets that decrease; that server's rows are then left unwritten.
  */

@@ -1,11 +1,15 @@
-// gs_verify_attn: dispatch between the tensor-core split-KV kernel (bf16) and the plain kernel.
+// gs_verify_attn: dispatch between the tensor-core split-KV kernel (bf16, head size 128) and the
+// plain kernel (fp32, other head sizes).
 #include "common.cuh"
 #include "attn_generic.cuh"
+#include "attn_tc.cuh"
 
 extern "C" size_t gs_verify_attn_workspace(int N, int Tq, int total_kv, int max_kv_len, int Hq, int Hkv,
                                            int hd, gs_dtype dt) {
-  (void)N; (void)Tq; (void)total_kv; (void)max_kv_len; (void)Hq; (void)Hkv; (void)hd; (void)dt;
-  return 256;
+  using namespace gs;
+  if (N <= 0 || Tq <= 0 || total_kv <= 0 || max_kv_len <= 0 || Hq <= 0 || Hkv <= 0) return 256;
+  if (!attn_tc_supported(Hq, Hkv, hd, dt)) return 256;
+  return align_up(attn_tc_plan(N, Tq, total_kv, max_kv_len, Hq, Hkv).ws_bytes, 256);
 }
 
 extern "C" gs_status gs_verify_attn(const void* Q, const void* K, const void* V, void* O,
@@ -28,6 +32,10 @@ extern "C" gs_status gs_verify_attn(const void* Q, const void* K, const void* V,
   if (dt == GS_F32)
     return launch_attn_generic<float>(Q, K, V, O, cu_q, cu_kv, N, Tq, total_kv, max_kv_len, Hq, Hkv, hd,
                                       scale, d_status, st);
+  const bool aligned = (reinterpret_cast<uintptr_t>(Q) % 16 == 0) && (reinterpret_cast<uintptr_t>(K) % 16 == 0) &&
+                       (reinterpret_cast<uintptr_t>(V) % 16 == 0) && (reinterpret_cast<uintptr_t>(ws) % 256 == 0);
+  if (attn_tc_supported(Hq, Hkv, hd, dt) && aligned && total_kv > 0 && max_kv_len > 0)
+    return launch_attn_tc(Q, K, V, O, cu_q, cu_kv, N, Tq, total_kv, max_kv_len, Hq, Hkv, scale, ws, d_status, st);
   return launch_attn_generic<__nv_bfloat16>(Q, K, V, O, cu_q, cu_kv, N, Tq, total_kv, max_kv_len, Hq, Hkv,
                                             hd, scale, d_status, st);
 }
