@@ -28,13 +28,13 @@ constexpr uint32_t kAtPBytes = kAtRows * kAtTile * 2;          // 16 KB
 constexpr uint32_t kAtKvBytes = 2 * kAtTile * kAtHd * 2;       // K + V of one tile: 32 KB
 constexpr uint32_t kAtSmem = kAtQBytes + kAtPBytes + kAtStages * kAtKvBytes + 256;
 constexpr uint32_t kAtTmemCols = 256;    // S: columns 0..63, O: columns 64..191
-constexpr int kAtPartStride = kAtHd + 2; // floats per partial row: O[128], m, l
+constexpr int kAtPartStride = kAtHd + 4; // floats per partial row: O[128], m, l, 2 pad (rows stay 16-byte aligned)
 constexpr float kAtLog2e = 1.4426950408889634f;
 
 struct AttnTcParams {
   const int32_t* cu_q;
   const int32_t* cu_kv;
-  float* part;              // [items][128][130]
+  float* part;              // [items][128][132]
   int32_t* d_status;
   int N, Tq, total_kv, max_kv_len, Hq, Hkv, G, TB;   // TB = 128 / G query positions per item
   int tiles_per_chunk;      // KV tiles per split (upper bound; splits of a server are balanced)
