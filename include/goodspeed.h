@@ -151,6 +151,34 @@ gs_status gs_spec_accept(const float* logits, const float* q_probs, const int32_
                          void* ws, size_t ws_bytes, int32_t* d_status, void* stream);
 
 /* --------------------------------------------------------------------------------------------
+ * gs_spec_accept_static -- no counterpart in the paper: a convenience of this library.
+ *
+ * The same computation, arguments and results as gs_spec_accept, for callers that cannot provide
+ * a workspace because they are not allowed to allocate device memory where the round runs (a
+ * serving loop with a memory pool frozen at start-up, a plug-in that only borrows its input and
+ * output buffers, a context in which an allocation would stall or fail).  The scratch is a fixed
+ * array of gs_spec_accept_static_capacity() bytes (2 MiB) inside the library; every GPU that
+ * loads the library holds that array until the process ends.  The call itself allocates nothing.
+ *   - Limit: gs_spec_accept_workspace(N, Tq, V) must not exceed the capacity (for V = 151936 that
+ *     is about 3400 verify positions); larger problems return GS_ERR_WORKSPACE and launch nothing.
+ *   - The first call on each device looks the array's device address up (with that device
+ *     current); make that first call outside any stream capture.
+ *   - All calls share the one array.  Nothing in it has to be cleared between calls (every word a
+ *     call reads it has written before), but two calls that overlap on the GPU (different
+ *     streams, or different host threads) race on it and give wrong results: keep them ordered.
+ * Errors: as gs_spec_accept, plus WORKSPACE for the size limit and CUDA if the address lookup fails.
+ */
+size_t gs_spec_accept_static_capacity(void);
+gs_status gs_spec_accept_static(const float* logits, const float* q_probs, const int32_t* draft_tok,
+                                const int32_t* cu_q, const float* u_accept, const float* u_sample,
+                                float temperature, int N, int Tq, int V,
+                                int32_t* accepted, int32_t* out_tok, int32_t* n_out,
+                                float* ratio, float* p_tok, float* margin,
+                                double* alpha_hat, double* X, double eta, double beta,
+                                double alpha_min, double alpha_max,
+                                int32_t* d_status, void* stream);
+
+/* --------------------------------------------------------------------------------------------
  * gs_schedule -- GoodSpeed-sched (Eq. goodspeed_sched, Sec. III-C) with U_i = log:
  *   maximise sum_i (1/X_i) (1 - alpha_hat_i^(S_i+1)) / (1 - alpha_hat_i)
  *   subject to sum_i S_i <= C, s_min_i <= S_i <= s_max_i, S_i integer.

@@ -36,6 +36,10 @@ SIGNATURES = {
     "gs_spec_accept": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _f, _i, _i, _i,
                             _vp, _vp, _vp, _vp, _vp, _vp,
                             _vp, _vp, _d, _d, _d, _d, _vp, _sz, _vp, _vp]),
+    "gs_spec_accept_static_capacity": (_sz, []),
+    "gs_spec_accept_static": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _f, _i, _i, _i,
+                                   _vp, _vp, _vp, _vp, _vp, _vp,
+                                   _vp, _vp, _d, _d, _d, _d, _vp, _vp]),
     "gs_schedule": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp]),
     "gs_verify_round_workspace": (_sz, [_vp]),
     "gs_verify_round_host": (_i, [_vp] + [_vp] * 8 + [_vp] * 7 + [_vp, _sz] + [_vp] * 5 + [_vp]),
@@ -201,3 +205,26 @@ def gs_verify_round_host(desc: RoundDesc, h_Q, h_H, h_q_probs, h_draft_tok, h_u_
         hp(h_accepted, i32), hp(h_out_tok, i32), hp(h_n_out, i32), hp(h_S_next, i32), hp(h_status, i32),
         _stream())
     _check("gs_verify_round_host", code)
+
+
+def gs_spec_accept_static_capacity() -> int:
+    return int(lib().gs_spec_accept_static_capacity())
+
+
+def gs_spec_accept_static(logits, q_probs, draft_tok, cu_q, u_accept, u_sample, temperature,
+                          accepted, out_tok, n_out, ratio, p_tok, margin=None,
+                          alpha_hat=None, X=None, eta=0.0, beta=0.0, alpha_min=1e-3, alpha_max=0.999,
+                          d_status=None):
+    """gs_spec_accept without a workspace argument: the scratch is a fixed array inside the library,
+    so the call allocates nothing (see the header for the size limit and the sharing rules)."""
+    Tq, V = logits.shape
+    N = cu_q.numel() - 1
+    f32, i32, f64 = torch.float32, torch.int32, torch.float64
+    code = lib().gs_spec_accept_static(_ptr(logits, f32), _ptr(q_probs, f32), _ptr(draft_tok, i32),
+                                       _ptr(cu_q, i32), _ptr(u_accept, f32), _ptr(u_sample, f32),
+                                       float(temperature), N, Tq, V,
+                                       _ptr(accepted, i32), _ptr(out_tok, i32), _ptr(n_out, i32),
+                                       _ptr(ratio, f32), _ptr(p_tok, f32), _ptr(margin, f32),
+                                       _ptr(alpha_hat, f64), _ptr(X, f64), float(eta), float(beta),
+                                       float(alpha_min), float(alpha_max), _ptr(d_status, i32), _stream())
+    _check("gs_spec_accept_static", code)

@@ -477,3 +477,54 @@ extern "C" gs_status gs_spec_accept(const float* logits, const float* q_probs, c
   count_launches(k2 > 0.f ? 4 : 3);
   return launch_status();
 }
+
+// ------------------------------------------------------------------------------------------------
+// gs_spec_accept_static: the same acceptance pass for callers that cannot hand over a workspace.
+//
+// Some hosts of this library may not allocate device memory at the point where a round runs: a
+// serving loop whose memory pool was sized and frozen at start-up, a plug-in that is only lent
+// input and output buffers, code running where cudaMalloc would serialise or fail.  For them the
+// scratch (chunk statistics, per-server selection, chunk masses) lives in the fixed array below,
+// which every GPU that loads the library carries until the process exits.
+namespace gs {
+
+constexpr size_t kSaStaticBytes = 2u << 20;   // 2 MiB
+static __device__ __align__(256) unsigned char g_sa_static_scratch[kSaStaticBytes];
+
+// In host code the symbol above is only a handle; the device address has to be asked for, once
+// per device, with that device current.
+static void* sa_static_scratch_ptr(gs_status* err) {
+  constexpr int kMaxDevices = 64;
+  static void* cached[kMaxDevices] = {};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { *err = GS_ERR_CUDA; return nullptr; }
+  if (cached[dev] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_sa_static_scratch) != cudaSuccess || p == nullptr) { *err = GS_ERR_CUDA; return nullptr; }
+    cached[dev] = p;
+  }
+  return cached[dev];
+}
+
+}  // namespace gs
+
+extern "C" size_t gs_spec_accept_static_capacity(void) { return gs::kSaStaticBytes; }
+
+extern "C" gs_status gs_spec_accept_static(const float* logits, const float* q_probs, const int32_t* draft_tok,
+                                           const int32_t* cu_q, const float* u_accept, const float* u_sample,
+                                           float temperature, int N, int Tq, int V,
+                                           int32_t* accepted, int32_t* out_tok, int32_t* n_out,
+                                           float* ratio, float* p_tok, float* margin,
+                                           double* alpha_hat, double* X, double eta, double beta,
+                                           double alpha_min, double alpha_max,
+                                           int32_t* d_status, void* stream) {
+  if (N < 0 || Tq < 0 || V < 0) return GS_ERR_INVALID_ARG;
+  if (N == 0) return GS_OK;
+  if (gs_spec_accept_workspace(N, Tq, V) > gs::kSaStaticBytes) return GS_ERR_WORKSPACE;   // problem too large
+  gs_status err = GS_OK;
+  void* scratch = gs::sa_static_scratch_ptr(&err);
+  if (scratch == nullptr) return err;
+  return gs_spec_accept(logits, q_probs, draft_tok, cu_q, u_accept, u_sample, temperature, N, Tq, V,
+                        accepted, out_tok, n_out, ratio, p_tok, margin, alpha_hat, X, eta, beta,
+                        alpha_min, alpha_max, scratch, gs::kSaStaticBytes, d_status, stream);
+}
