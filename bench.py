@@ -337,7 +337,7 @@ def run_ours(args, cfg, rank, world, local_rank):
 
     # ---- end to end through the host-buffer entry point (pinned inputs, results read back each step)
     e2e = None
-    if world == 1:
+    if world == 1 and not args.profile_small:
         desc = B.RoundDesc(N=N, Tq=Tq, total_kv=total_kv, max_kv_len=rnd.max_kv_len, Hq=cfg.Hq, Hkv=cfg.Hkv,
                            hd=cfg.hd, d=d, V=V, C=C, dt=B.GS_BF16 if cfg.dtype == "bf16" else B.GS_F32,
                            scale=cfg.hd ** -0.5, temperature=float(inp["tau"]), eta=ETA, beta=BETA,
@@ -425,12 +425,18 @@ def main():
     ap.add_argument("--config", default="cfg2", choices=["cfg2", "cfg3", "cfg4"])
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--profile-small", action="store_true",
+                    help="profiling case: vocabulary cut to 32768 (W = 336 MB, still larger than L2), eager "
+                         "launches, no CPU baseline and no end-to-end leg; for ncu --set full captures")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     cfg = wl.CONFIGS[args.config]
+    if args.profile_small:
+        cfg = wl.shrink(cfg, V=32768, name=cfg.name + "_V32768")
+        args.no_graph = args.skip_cpu_baseline = True
     if args.impl == "reference":
         run_reference(args, cfg, rank, world)
         return
