@@ -9,8 +9,10 @@
 //                        max/sum, bf16 P written to shared memory in the swizzled operand layout
 //     O += P V           tcgen05.mma  M=128, N=128, K=64    (V read as an MN-major operand)
 // K/V tiles arrive by TMA through a 2-stage ring.  Two CTAs share an SM, so one CTA's softmax
-// overlaps the other's MMAs and loads.  Each item writes an unnormalised partial (m, l, O) to the
-// workspace; a second kernel merges the splits.  CTAs are persistent and stride over the items.
+// overlaps the other's MMAs and loads.  An item whose server needs a single KV split normalises and
+// stores its rows directly; otherwise it writes an unnormalised partial (m, l, O) to the workspace
+// and takes a ticket, and the last split of a (server, position block, KV head) to finish merges
+// them (nobody waits).  CTAs are persistent and stride over the items.
 #pragma once
 #include "common.cuh"
 #include "sm100_ptx.cuh"
@@ -35,6 +37,8 @@ struct AttnTcParams {
   const int32_t* cu_q;
   const int32_t* cu_kv;
   float* part;              // [items][128][132]
+  int* tickets;             // [groups][4] splits of a (server, position block, KV head) done, per 32-row quadrant
+  __nv_bfloat16* O;
   int32_t* d_status;
   int N, Tq, total_kv, max_kv_len, Hq, Hkv, G, TB;   // TB = 128 / G query positions per item
   int tiles_per_chunk;      // KV tiles per split (upper bound; splits of a server are balanced)
@@ -48,6 +52,8 @@ struct AttnItem {
   int n_t;                         // positions in the block
   int kv0, Lkv, L;                 // first key row (global), keys of the server, prefix length
   int tile0, n_tiles;              // tiles [tile0, tile0 + n_tiles) of the server
+  int item_base, nsplit, n_used;   // first item of the server, its splits, splits that see any key
+  int group;                       // index of (server, position block, KV head) over the whole batch
   int valid;
 };
 
@@ -62,13 +68,13 @@ GS_DEVINL int attn_nsplit(int Lkv, int tiles_per_chunk) {
 GS_DEVINL AttnItem attn_find_item(const AttnTcParams& P, int id) {
   AttnItem it;
   it.valid = 0;
-  int base = 0;
+  int base = 0, gbase = 0;
   for (int i = 0; i < P.N; ++i) {
     const int q0 = P.cu_q[i], n_new = P.cu_q[i + 1] - q0;
     const int k0 = P.cu_kv[i], Lkv = P.cu_kv[i + 1] - k0;
     if (n_new <= 0 || Lkv < n_new || Lkv > P.max_kv_len || k0 < 0 || k0 + Lkv > P.total_kv || q0 < 0 ||
         q0 + n_new > P.Tq)
-      continue;   // flagged by the combine kernel
+      continue;   // flagged by the checking kernel
     const int tgs = (n_new + P.TB - 1) / P.TB;
     const int nsplit = attn_nsplit(Lkv, P.tiles_per_chunk);
     const int cnt = tgs * nsplit * P.Hkv;
@@ -77,6 +83,8 @@ GS_DEVINL AttnItem attn_find_item(const AttnTcParams& P, int id) {
       it.g = rem % P.Hkv; rem /= P.Hkv;
       it.split = rem % nsplit; it.tg = rem / nsplit;
       it.server = i;
+      it.item_base = base; it.nsplit = nsplit;
+      it.group = gbase + it.tg * P.Hkv + it.g;
       it.q_row0 = q0 + it.tg * P.TB;
       it.n_t = min(P.TB, n_new - it.tg * P.TB);
       it.kv0 = k0; it.Lkv = Lkv; it.L = Lkv - n_new;
@@ -88,10 +96,14 @@ GS_DEVINL AttnItem attn_find_item(const AttnTcParams& P, int id) {
       const int last_key = it.L + it.tg * P.TB + it.n_t - 1;
       const int last_tile = last_key / kAtTile;
       if (it.tile0 + it.n_tiles - 1 > last_tile) it.n_tiles = max(0, last_tile - it.tile0 + 1);
+      it.n_used = 0;
+      for (int sp = 0; sp < nsplit; ++sp)
+        if (sp * tb + min(sp, tr) <= last_tile) it.n_used = sp + 1;
       it.valid = 1;
       return it;
     }
     base += cnt;
+    gbase += tgs * P.Hkv;
   }
   return it;
 }
@@ -108,7 +120,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant_
   uint8_t* tail = smem_raw + (bars - base) + 8 * (5 + 2 * kAtStages);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 4);
-  volatile int* s_item = reinterpret_cast<volatile int*>(tail + 8);   // AttnItem broadcast (11 ints)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if ((base & 1023u) != 0) {                     // the operand layouts need a 1024-byte aligned base
@@ -251,10 +262,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant_
           sv[c] = __float_as_uint(s);
           tmax = fmaxf(tmax, s);
         }
-        const float m_new = fmaxf(m_run, tmax);
+        // The reference maximum only moves when the tile maximum exceeds it by more than 2^8:
+        // P stays below 256, the final O/l is unchanged, and O in TMEM is rescaled rarely.
+        const float m_new = (tmax > m_run + 8.f) ? tmax : m_run;
         const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
         const float corr = (m_run == -INFINITY) ? 0.f : fast_exp2(m_run - m_use);
-        // Rescale O when this warp has a row whose maximum moved (never for the first tile, whose
+        // Rescale O when this warp has a row whose reference moved (never for the first tile, whose
         // P V product overwrites O).  All earlier MMAs have completed: S of this tile was
         // committed after them.
         const bool need = row_ok && j > 0 && (m_new > m_run);
@@ -299,26 +312,91 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant_
         if (lane == 0) mbar_arrive(bar(3));
       }
       if (!ok) break;
-      // epilogue: unnormalised partial (O, m, l) of this item
+      // epilogue
       if (!mbar_wait(bar(4), (uint32_t)n_item & 1u, abort_flag)) { ok = false; break; }
       tc_fence_after();
-      float* out = P.part + ((size_t)id * kAtRows + r) * kAtPartStride;
+      float o[kAtHd];
 #pragma unroll
       for (int c0 = 0; c0 < kAtHd; c0 += 16) {
-        uint32_t o[16];
-        tmem_ld16(tmem_O + lane_addr + c0, o);
+        uint32_t t16[16];
+        tmem_ld16(tmem_O + lane_addr + c0, t16);
         tmem_ld_wait();
-        if (row_ok) {
 #pragma unroll
-          for (int c = 0; c < 16; c += 4)
-            *reinterpret_cast<float4*>(out + c0 + c) = make_float4(__uint_as_float(o[c]), __uint_as_float(o[c + 1]),
-                                                                   __uint_as_float(o[c + 2]), __uint_as_float(o[c + 3]));
-        }
+        for (int c = 0; c < 16; ++c) o[c0 + c] = __uint_as_float(t16[c]);
       }
-      if (row_ok) { out[kAtHd] = m_run; out[kAtHd + 1] = l_run; }
+      // TMEM and the Q buffer are free again: the next item may start while this one is stored
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(1));
+      __nv_bfloat16* orow = P.O + ((size_t)(it.q_row0 + r / P.G) * P.Hq + it.g * P.G + (r % P.G)) * kAtHd;
+      if (it.n_used == 1) {
+        // the only split of its group: normalise and store
+        if (row_ok) {
+          const float inv = 1.f / l_run;
+#pragma unroll
+          for (int c = 0; c < kAtHd; c += 8) {
+            uint4 pk;
+            __nv_bfloat162 b0 = __floats2bfloat162_rn(o[c] * inv, o[c + 1] * inv);
+            __nv_bfloat162 b1 = __floats2bfloat162_rn(o[c + 2] * inv, o[c + 3] * inv);
+            __nv_bfloat162 b2 = __floats2bfloat162_rn(o[c + 4] * inv, o[c + 5] * inv);
+            __nv_bfloat162 b3 = __floats2bfloat162_rn(o[c + 6] * inv, o[c + 7] * inv);
+            pk.x = *reinterpret_cast<uint32_t*>(&b0); pk.y = *reinterpret_cast<uint32_t*>(&b1);
+            pk.z = *reinterpret_cast<uint32_t*>(&b2); pk.w = *reinterpret_cast<uint32_t*>(&b3);
+            *reinterpret_cast<uint4*>(orow + c) = pk;
+          }
+        }
+      } else {
+        // unnormalised partial (O, m, l), then a ticket; the last split of the group merges
+        float* out = P.part + ((size_t)id * kAtRows + r) * kAtPartStride;
+        if (row_ok) {
+#pragma unroll
+          for (int c = 0; c < kAtHd; c += 4) *reinterpret_cast<float4*>(out + c) = make_float4(o[c], o[c + 1], o[c + 2], o[c + 3]);
+          out[kAtHd] = m_run; out[kAtHd + 1] = l_run;
+        }
+        // One ticket per (group, 32-row quadrant): the warp that takes the last one finds the other
+        // splits' rows of its quadrant complete (their writers fenced before taking theirs).
+        __threadfence();
+        __syncwarp();
+        int tk = 0;
+        if (lane == 0) tk = atomicAdd(&P.tickets[it.group * 4 + q], 1);
+        tk = __shfl_sync(0xffffffffu, tk, 0);
+        const bool last = (tk == it.n_used - 1);
+        if (last && row_ok) {
+          __threadfence();
+          float M = -INFINITY;
+          for (int sp = 0; sp < it.n_used; ++sp) {
+            const float* p = P.part + ((size_t)(it.item_base + (it.tg * it.nsplit + sp) * P.Hkv + it.g) * kAtRows + r) * kAtPartStride;
+            M = fmaxf(M, __ldcg(p + kAtHd));
+          }
+          float L = 0.f;
+#pragma unroll
+          for (int c = 0; c < kAtHd; ++c) o[c] = 0.f;
+          for (int sp = 0; sp < it.n_used; ++sp) {
+            const float* p = P.part + ((size_t)(it.item_base + (it.tg * it.nsplit + sp) * P.Hkv + it.g) * kAtRows + r) * kAtPartStride;
+            const float ms = __ldcg(p + kAtHd);
+            if (ms == -INFINITY) continue;
+            const float w = fast_exp2(ms - M);
+            L += __ldcg(p + kAtHd + 1) * w;
+#pragma unroll
+            for (int c = 0; c < kAtHd; c += 4) {
+              const float4 v = __ldcg(reinterpret_cast<const float4*>(p + c));
+              o[c] += v.x * w; o[c + 1] += v.y * w; o[c + 2] += v.z * w; o[c + 3] += v.w * w;
+            }
+          }
+          const float inv = 1.f / L;
+#pragma unroll
+          for (int c = 0; c < kAtHd; c += 8) {
+            uint4 pk;
+            __nv_bfloat162 b0 = __floats2bfloat162_rn(o[c] * inv, o[c + 1] * inv);
+            __nv_bfloat162 b1 = __floats2bfloat162_rn(o[c + 2] * inv, o[c + 3] * inv);
+            __nv_bfloat162 b2 = __floats2bfloat162_rn(o[c + 4] * inv, o[c + 5] * inv);
+            __nv_bfloat162 b3 = __floats2bfloat162_rn(o[c + 6] * inv, o[c + 7] * inv);
+            pk.x = *reinterpret_cast<uint32_t*>(&b0); pk.y = *reinterpret_cast<uint32_t*>(&b1);
+            pk.z = *reinterpret_cast<uint32_t*>(&b2); pk.w = *reinterpret_cast<uint32_t*>(&b3);
+            *reinterpret_cast<uint4*>(orow + c) = pk;
+          }
+        }
+      }
       ++n_item;
     }
   }
@@ -331,55 +409,22 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant_
   }
 }
 
-// Merges the splits of one (query row, query head): O = sum_s O_s 2^(m_s - M) / sum_s l_s 2^(m_s - M).
-__global__ void __launch_bounds__(128)
-attn_combine_kernel(const AttnTcParams P, __nv_bfloat16* __restrict__ O) {
-  const int h = blockIdx.x, row = blockIdx.y, c = threadIdx.x;      // 128 threads = 128 head dims
-  if (row >= P.cu_q[P.N]) return;
-  const int i = find_server(P.cu_q, P.N, row);
-  const int q0 = P.cu_q[i], n_new = P.cu_q[i + 1] - q0;
-  const int k0 = P.cu_kv[i], Lkv = P.cu_kv[i + 1] - k0;
-  if (n_new <= 0 || Lkv < n_new || Lkv > P.max_kv_len || k0 < 0 || k0 + Lkv > P.total_kv) {
-    if (c == 0) set_status(P.d_status, GS_ERR_SHAPE);
-    return;
+// Offsets the device has to vouch for: a server with fewer keys than new positions, more keys than
+// max_kv_len, or offsets outside the tensors is skipped by the main kernel and flagged here.
+__global__ void attn_check_kernel(const AttnTcParams P) {
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < P.N; i += gridDim.x * blockDim.x) {
+    const int q0 = P.cu_q[i], n_new = P.cu_q[i + 1] - q0;
+    const int k0 = P.cu_kv[i], Lkv = P.cu_kv[i + 1] - k0;
+    if (n_new <= 0 || Lkv < n_new || Lkv > P.max_kv_len || k0 < 0 || k0 + Lkv > P.total_kv || q0 < 0 ||
+        q0 + n_new > P.Tq)
+      set_status(P.d_status, GS_ERR_SHAPE);
   }
-  // first item of server i
-  int base = 0;
-  for (int s = 0; s < i; ++s) {
-    const int nn = P.cu_q[s + 1] - P.cu_q[s], lk = P.cu_kv[s + 1] - P.cu_kv[s];
-    if (nn <= 0 || lk < nn || lk > P.max_kv_len || P.cu_kv[s] < 0 || P.cu_kv[s] + lk > P.total_kv) continue;
-    base += ((nn + P.TB - 1) / P.TB) * attn_nsplit(lk, P.tiles_per_chunk) * P.Hkv;
-  }
-  const int t = row - q0, tg = t / P.TB, g = h / P.G;
-  const int r = (t - tg * P.TB) * P.G + (h - g * P.G);
-  const int nsplit = attn_nsplit(Lkv, P.tiles_per_chunk);
-  const int tiles = (Lkv + kAtTile - 1) / kAtTile, tb = tiles / nsplit, tr = tiles % nsplit;
-  const int last_tile = (Lkv - n_new + min(tg * P.TB + P.TB, n_new) - 1) / kAtTile;
-  float M = -INFINITY;
-  int used = 0;
-  for (int s = 0; s < nsplit; ++s) {
-    const int tile0 = s * tb + min(s, tr);
-    if (tile0 > last_tile) break;            // this split saw nothing for the block: no partial written
-    used = s + 1;
-    const float* p = P.part + ((size_t)(base + (tg * nsplit + s) * P.Hkv + g) * kAtRows + r) * kAtPartStride;
-    M = fmaxf(M, p[kAtHd]);
-  }
-  float acc = 0.f, L = 0.f;
-  for (int s = 0; s < used; ++s) {
-    const float* p = P.part + ((size_t)(base + (tg * nsplit + s) * P.Hkv + g) * kAtRows + r) * kAtPartStride;
-    const float ms = p[kAtHd];
-    if (ms == -INFINITY) continue;
-    const float w = fast_exp2(ms - M);
-    L += p[kAtHd + 1] * w;
-    acc += p[c] * w;
-  }
-  O[((size_t)row * P.Hq + h) * kAtHd + c] = __float2bfloat16_rn(acc / L);
 }
 
 // ------------------------------------------------------------------ host side
 struct AttnTcPlan {
-  int TB, tiles_per_chunk, max_items, grid;
-  size_t ws_bytes;
+  int TB, tiles_per_chunk, max_items, max_groups, grid;
+  size_t ticket_bytes, ws_bytes;
 };
 
 inline bool attn_tc_supported(int Hq, int Hkv, int hd, gs_dtype dt) {
@@ -402,7 +447,9 @@ inline AttnTcPlan attn_tc_plan(int N, int Tq, int total_kv, int max_kv_len, int 
   const long long items = (long long)Hkv * blocks * ((max_tiles + pl.tiles_per_chunk - 1) / pl.tiles_per_chunk);
   pl.max_items = (int)min(items, (long long)INT_MAX / 2);
   pl.grid = min(pl.max_items, slots);
-  pl.ws_bytes = (size_t)pl.max_items * kAtRows * kAtPartStride * sizeof(float);
+  pl.max_groups = (int)min((long long)Hkv * blocks, (long long)INT_MAX / 2);
+  pl.ticket_bytes = align_up((size_t)pl.max_groups * 4 * sizeof(int), 256);
+  pl.ws_bytes = pl.ticket_bytes + (size_t)pl.max_items * kAtRows * kAtPartStride * sizeof(float);
   return pl;
 }
 
@@ -417,7 +464,10 @@ inline gs_status launch_attn_tc(const void* Q, const void* K, const void* V, voi
   }
   const AttnTcPlan pl = attn_tc_plan(N, Tq, total_kv, max_kv_len, Hq, Hkv);
   AttnTcParams P;
-  P.cu_q = cu_q; P.cu_kv = cu_kv; P.part = static_cast<float*>(ws); P.d_status = d_status;
+  P.cu_q = cu_q; P.cu_kv = cu_kv; P.d_status = d_status;
+  P.tickets = static_cast<int*>(ws);
+  P.part = reinterpret_cast<float*>(static_cast<char*>(ws) + pl.ticket_bytes);
+  P.O = static_cast<__nv_bfloat16*>(O);
   P.N = N; P.Tq = Tq; P.total_kv = total_kv; P.max_kv_len = max_kv_len; P.Hq = Hq; P.Hkv = Hkv;
   P.G = Hq / Hkv; P.TB = pl.TB; P.tiles_per_chunk = pl.tiles_per_chunk; P.max_items = pl.max_items;
   P.scale_log2 = scale * kAtLog2e;
@@ -438,11 +488,11 @@ inline gs_status launch_attn_tc(const void* Q, const void* K, const void* V, voi
   if (!make_tmap_bf16_2d(&tmK, K, (uint64_t)total_kv, (uint64_t)Hkv * kAtHd, (uint64_t)Hkv * kAtHd, kAtTile, 64) ||
       !make_tmap_bf16_2d(&tmV, V, (uint64_t)total_kv, (uint64_t)Hkv * kAtHd, (uint64_t)Hkv * kAtHd, kAtTile, 64))
     return GS_ERR_CUDA;
+  if (cudaMemsetAsync(P.tickets, 0, pl.ticket_bytes, st) != cudaSuccess) return GS_ERR_CUDA;
   attn_tc_kernel<<<pl.grid, kAtThreads, kAtSmem, st>>>(tmQ, tmK, tmV, P);
   if (cudaGetLastError() != cudaSuccess) return GS_ERR_CUDA;
-  dim3 cgrid(Hq, Tq);
-  attn_combine_kernel<<<cgrid, 128, 0, st>>>(P, static_cast<__nv_bfloat16*>(O));
-  count_launches(2);
+  if (d_status != nullptr) attn_check_kernel<<<1, 128, 0, st>>>(P);
+  count_launches(d_status != nullptr ? 2 : 1);
   return launch_status();
 }
 

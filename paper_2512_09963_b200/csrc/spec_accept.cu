@@ -1,16 +1,18 @@
 // gs_spec_accept: temperature softmax statistics, sequential accept/reject, correction or bonus
 // token by inverse CDF, and the estimator updates (Sec. II-A2; Eq. updatealpha, Eq. updateX).
 //
-// Four launches on one stream:
+// Two launches on one stream:
 //   1. sa_row_stats   every logit row is cut into chunks of 4096 floats; one CTA per (chunk,row)
 //                     streams its chunk once with 16-byte loads and writes (max, argmax, sum exp).
-//   2. sa_decide      one CTA per server merges the chunk statistics of its rows in chunk order,
-//                     evaluates p(s_j), q(s_j), the ratios, the accepted count, the estimators,
-//                     and selects the one row the last token is drawn from.
-//   3. sa_mass        one CTA per (chunk, server) sums the mass of the selected row's chunk:
-//                     max(0, p - q) after a rejection, p for the bonus row.
-//   4. sa_sample      one CTA per server scans the chunk masses in order, finds the chunk that
-//                     holds u * total, and does an ordered prefix scan inside that chunk.
+//   2. sa_finish      one CTA per (chunk, server).  Every CTA of a server first repeats the small
+//                     "decide" step (a warp per row merges that row's chunk statistics, evaluates
+//                     p(s_j), q(s_j), the ratio; one thread scans for the first rejection), which
+//                     selects the one row the last token is drawn from; the CTA then sums the mass
+//                     of its chunk of that row (max(0, p - q) after a rejection, p for the bonus
+//                     row).  The last CTA of a server to finish (an atomic ticket, nobody waits)
+//                     scans the chunk masses in order, finds the chunk that holds u * total and
+//                     does an ordered prefix scan inside it.  CTA (0, server) writes the outputs
+//                     and the estimator update.
 // Only one row per server is read a second time.  All cross-thread sums are fp64 in a fixed
 // order, so two runs give identical bits.
 #include "common.cuh"
@@ -28,19 +30,9 @@ struct ChunkStat {   // 16 bytes
   double z;
 };
 
-struct ServerSel {   // what sa_mass / sa_sample need about a server
-  int row;           // logits row the last token is drawn from
-  int qrow;          // q_probs row to subtract, or -1 for the bonus row
-  float M;           // row max
-  int arg;           // row argmax
-  double invZ;       // 1 / sum exp
-  int valid;
-  int pad;
-};
-
 struct SaWorkspace {
   ChunkStat* stats;   // [Tq * n_chunk]
-  ServerSel* sel;     // [N]
+  int* tickets;       // [N] CTAs of a server that have delivered their chunk mass
   double* mass;       // [N * n_chunk]
 };
 
@@ -48,11 +40,11 @@ static size_t sa_layout(int N, int Tq, int V, SaWorkspace* w, char* base) {
   size_t n_chunk = (size_t)(V + kSaChunk - 1) / kSaChunk;
   size_t off = 0;
   size_t stats = off; off = align_up(off + sizeof(ChunkStat) * n_chunk * (size_t)Tq, 256);
-  size_t sel = off;   off = align_up(off + sizeof(ServerSel) * (size_t)N, 256);
+  size_t sel = off;   off = align_up(off + sizeof(int) * (size_t)N, 256);
   size_t mass = off;  off = align_up(off + sizeof(double) * n_chunk * (size_t)N, 256);
   if (w != nullptr) {
     w->stats = reinterpret_cast<ChunkStat*>(base + stats);
-    w->sel = reinterpret_cast<ServerSel*>(base + sel);
+    w->tickets = reinterpret_cast<int*>(base + sel);
     w->mass = reinterpret_cast<double*>(base + mass);
   }
   return off;
@@ -97,12 +89,15 @@ GS_DEVINL double block_sum_f64(double v, double* smem8) {
 
 template <bool VEC>
 __global__ void __launch_bounds__(kSaThreads)
-sa_row_stats(const float* __restrict__ logits, int V, int n_chunk, float k2, ChunkStat* __restrict__ stats) {
+sa_row_stats(const float* __restrict__ logits, int V, int n_chunk, float k2, ChunkStat* __restrict__ stats,
+             int* __restrict__ tickets, int N) {
   __shared__ float s_m[kSaThreads / 32];
   __shared__ int s_a[kSaThreads / 32];
   __shared__ double s_z[kSaThreads / 32];
   __shared__ float s_bm;
   const int tid = threadIdx.x, c = blockIdx.x, r = blockIdx.y;
+  if (c == 0 && r == 0)
+    for (int i = tid; i < N; i += kSaThreads) tickets[i] = 0;     // for the next kernel
   const float* row = logits + (size_t)r * V;
   const int base = c * kSaChunk;
   float v[kSaPerThread];
@@ -138,117 +133,17 @@ sa_row_stats(const float* __restrict__ logits, int V, int n_chunk, float k2, Chu
   }
 }
 
-struct SaDecideArgs {
+struct SaFinishArgs {
   const float* logits; const float* q_probs; const int32_t* draft_tok; const int32_t* cu_q;
-  const float* u_accept;
-  int N, Tq, V, n_chunk;
-  float tau;
+  const float* u_accept; const float* u_sample;
+  int N, Tq, V, n_chunk, Gamma;
+  float tau, k2;
   int32_t* accepted; int32_t* out_tok; int32_t* n_out;
   float* ratio; float* p_tok; float* margin;
   double* alpha_hat; double* X; double eta, beta, alpha_min, alpha_max;
-  const ChunkStat* stats; ServerSel* sel;
+  const ChunkStat* stats; int* tickets; double* mass;
   int32_t* d_status;
 };
-
-constexpr int kDecideThreads = 128;
-
-// Merges the chunk statistics of row r in chunk order.
-GS_DEVINL void merge_row(const ChunkStat* __restrict__ st, int n_chunk, float tau, float& M, int& arg, double& Z) {
-  M = st[0].m; arg = st[0].arg;
-  for (int c = 1; c < n_chunk; ++c) argmax_merge(M, arg, st[c].m, st[c].arg);
-  Z = 0.0;
-  if (tau > 0.f) {
-    const double inv_tau = 1.0 / (double)tau;
-    for (int c = 0; c < n_chunk; ++c) {
-      if (st[c].m > -INFINITY) Z += st[c].z * exp(((double)st[c].m - (double)M) * inv_tau);
-    }
-  }
-}
-
-__global__ void __launch_bounds__(kDecideThreads) sa_decide(SaDecideArgs A) {
-  extern __shared__ unsigned char smem_raw[];
-  const int i = blockIdx.x, tid = threadIdx.x;
-  const int r0 = A.cu_q[i], r1 = A.cu_q[i + 1];
-  const int gamma = r1 - r0 - 1;
-  if (r0 < 0 || gamma < 0 || r1 > A.Tq) {
-    if (tid == 0) {
-      set_status(A.d_status, GS_ERR_SHAPE);
-      A.sel[i].valid = 0;
-      A.accepted[i] = 0; A.n_out[i] = 0;
-    }
-    return;
-  }
-  const int g0 = r0 - i;
-  // per-row merged statistics, rows j = 0..gamma
-  float* sM = reinterpret_cast<float*>(smem_raw);                // [gamma+1]
-  int* sArg = reinterpret_cast<int*>(sM + (gamma + 1));          // [gamma+1]
-  int* sRej = sArg + (gamma + 1);                                // [gamma+1] 1 = would be rejected
-  size_t off = (size_t)(3 * (gamma + 1)) * 4;
-  off = (off + 7) / 8 * 8;
-  double* sZ = reinterpret_cast<double*>(smem_raw + off);        // [gamma+1]
-  double* sRatio = sZ + (gamma + 1);                             // [gamma+1] clipped ratios
-
-  for (int j = tid; j <= gamma; j += kDecideThreads) {
-    float M; int arg; double Z;
-    merge_row(A.stats + (size_t)(r0 + j) * A.n_chunk, A.n_chunk, A.tau, M, arg, Z);
-    sM[j] = M; sArg[j] = arg; sZ[j] = Z;
-    if (j < gamma) {
-      const int s = A.draft_tok[g0 + j];
-      double p = 0.0, q = 0.0, rho = 0.0;
-      if (s < 0 || s >= A.V) {
-        set_status(A.d_status, GS_ERR_INVALID_ARG);
-      } else {
-        const float l = A.logits[(size_t)(r0 + j) * A.V + s];
-        if (A.tau > 0.f) p = (Z > 0.0) ? exp(((double)l - (double)M) / (double)A.tau) / Z : 0.0;
-        else p = (s == arg) ? 1.0 : 0.0;
-        q = (double)A.q_probs[(size_t)(g0 + j) * A.V + s];
-        if (q > 0.0) rho = p / q;
-        else rho = (p > 0.0) ? (double)INFINITY : 0.0;
-      }
-      const double u = (double)A.u_accept[g0 + j];
-      sRej[j] = (u > rho) ? 1 : 0;
-      const double clipped = rho < 1.0 ? rho : 1.0;
-      sRatio[j] = clipped;
-      A.ratio[g0 + j] = (float)clipped;
-      A.p_tok[g0 + j] = (float)p;
-      if (A.margin != nullptr) A.margin[g0 + j] = (float)(u - rho);
-    }
-  }
-  __syncthreads();
-  __shared__ int s_acc;
-  if (tid == 0) {
-    int a = gamma;
-    for (int j = 0; j < gamma; ++j) {
-      if (sRej[j]) { a = j; break; }
-    }
-    s_acc = a;
-    A.accepted[i] = a;
-    A.n_out[i] = a + 1;
-    ServerSel sel;
-    sel.row = r0 + a;
-    sel.qrow = (a < gamma) ? (g0 + a) : -1;
-    sel.M = sM[a]; sel.arg = sArg[a];
-    sel.invZ = (sZ[a] > 0.0) ? 1.0 / sZ[a] : 0.0;
-    sel.valid = 1; sel.pad = 0;
-    A.sel[i] = sel;
-    if (A.alpha_hat != nullptr && A.X != nullptr) {
-      if (gamma > 0) {
-        double sum = 0.0;
-        for (int j = 0; j < gamma; ++j) sum += sRatio[j];
-        const double obs = sum / (double)gamma;
-        double ah = (1.0 - A.eta) * A.alpha_hat[i] + A.eta * obs;
-        ah = ah < A.alpha_min ? A.alpha_min : ah;
-        ah = ah > A.alpha_max ? A.alpha_max : ah;
-        A.alpha_hat[i] = ah;
-      }
-      A.X[i] = (1.0 - A.beta) * A.X[i] + A.beta * (double)(a + 1);
-    }
-  }
-  __syncthreads();
-  const int a = s_acc;
-  for (int j = tid; j <= gamma; j += kDecideThreads)
-    A.out_tok[r0 + j] = (j < a) ? A.draft_tok[g0 + j] : -1;
-}
 
 // Mass of element v of the selected row: max(0, p - q) or p, in fp64 from an fp32 exponential.
 GS_DEVINL double elem_mass(float l, float M, float k2, double invZ, bool resid, float q) {
@@ -256,34 +151,6 @@ GS_DEVINL double elem_mass(float l, float M, float k2, double invZ, bool resid, 
   if (resid) { p -= (double)q; p = p > 0.0 ? p : 0.0; }
   return p;
 }
-
-template <bool VEC>
-__global__ void __launch_bounds__(kSaThreads)
-sa_mass(const float* __restrict__ logits, const float* __restrict__ q_probs, int V, int n_chunk, float k2,
-        const ServerSel* __restrict__ sel, double* __restrict__ mass) {
-  __shared__ double s_z[kSaThreads / 32];
-  const int tid = threadIdx.x, c = blockIdx.x, i = blockIdx.y;
-  const ServerSel s = sel[i];
-  if (!s.valid) return;
-  const int base = c * kSaChunk;
-  float l[kSaPerThread], q[kSaPerThread];
-  load_chunk<VEC>(logits + (size_t)s.row * V, base, V, tid, l);
-  const bool resid = s.qrow >= 0;
-  if (resid) load_chunk<VEC>(q_probs + (size_t)s.qrow * V, base, V, tid, q, 0.f);
-  double acc = 0.0;
-#pragma unroll
-  for (int e = 0; e < kSaPerThread; ++e) acc += elem_mass(l[e], s.M, k2, s.invZ, resid, resid ? q[e] : 0.f);
-  double tot = block_sum_f64(acc, s_z);
-  if (tid == 0) mass[(size_t)i * n_chunk + c] = tot;
-}
-
-struct SaSampleArgs {
-  const float* logits; const float* q_probs; const float* u_sample; const int32_t* cu_q;
-  int N, V, n_chunk, Gamma;
-  float k2;
-  const ServerSel* sel; const double* mass;
-  int32_t* out_tok; float* margin;
-};
 
 // Ordered scan of one chunk: thread t owns the 16 consecutive elements base + 16 t .. +15.
 // Returns through s_tok the smallest index whose inclusive prefix (offset by `before`) exceeds
@@ -335,61 +202,176 @@ GS_DEVINL void scan_chunk(const float* __restrict__ lrow, const float* __restric
   __syncthreads();
 }
 
-__global__ void __launch_bounds__(kSaThreads) sa_sample(SaSampleArgs A) {
-  __shared__ int s_chunk, s_tok, s_last;
+template <bool VEC>
+__global__ void __launch_bounds__(kSaThreads) sa_finish(SaFinishArgs A) {
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ int s_acc, s_is_last, s_chunk, s_tok, s_last;
   __shared__ double s_before, s_thr, s_total, s_lo, s_hi;
   __shared__ double s_warp[kSaThreads / 32];
-  const int i = blockIdx.x, tid = threadIdx.x;
-  const ServerSel s = A.sel[i];
-  if (!s.valid) return;
+  const int c = blockIdx.x, i = blockIdx.y, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const bool writer = (c == 0);           // one CTA per server owns the outputs
+  const int r0 = A.cu_q[i], r1 = A.cu_q[i + 1];
+  const int gamma = r1 - r0 - 1;
+  if (r0 < 0 || gamma < 0 || r1 > A.Tq) {
+    if (writer && tid == 0) {
+      set_status(A.d_status, GS_ERR_SHAPE);
+      A.accepted[i] = 0; A.n_out[i] = 0;
+    }
+    return;
+  }
+  const int g0 = r0 - i;
+  // per-row merged statistics, rows j = 0..gamma
+  float* sM = reinterpret_cast<float*>(smem_raw);                // [gamma+1]
+  int* sArg = reinterpret_cast<int*>(sM + (gamma + 1));          // [gamma+1]
+  int* sRej = sArg + (gamma + 1);                                // [gamma+1] 1 = would be rejected
+  size_t off = (size_t)(3 * (gamma + 1)) * 4;
+  off = (off + 7) / 8 * 8;
+  double* sZ = reinterpret_cast<double*>(smem_raw + off);        // [gamma+1]
+  double* sRatio = sZ + (gamma + 1);                             // [gamma+1] clipped ratios
+
+  // ---- decide: a warp per row, lanes over the row's chunks
+  const double inv_tau = A.tau > 0.f ? 1.0 / (double)A.tau : 0.0;
+  for (int j = wid; j <= gamma; j += kSaThreads / 32) {
+    const ChunkStat* st = A.stats + (size_t)(r0 + j) * A.n_chunk;
+    float M = -INFINITY; int arg = INT_MAX;
+    for (int cc = lane; cc < A.n_chunk; cc += 32) argmax_merge(M, arg, st[cc].m, st[cc].arg);
+    warp_argmax(M, arg);
+    double z = 0.0;
+    if (A.tau > 0.f)
+      for (int cc = lane; cc < A.n_chunk; cc += 32)
+        if (st[cc].m > -INFINITY) z += st[cc].z * exp(((double)st[cc].m - (double)M) * inv_tau);
+    const double Z = warp_sum_f64(z);
+    if (lane == 0) {
+      sM[j] = M; sArg[j] = arg; sZ[j] = Z;
+      if (j < gamma) {
+        const int s = A.draft_tok[g0 + j];
+        double p = 0.0, q = 0.0, rho = 0.0;
+        if (s < 0 || s >= A.V) {
+          if (writer) set_status(A.d_status, GS_ERR_INVALID_ARG);
+        } else {
+          const float l = A.logits[(size_t)(r0 + j) * A.V + s];
+          if (A.tau > 0.f) p = (Z > 0.0) ? exp(((double)l - (double)M) * inv_tau) / Z : 0.0;
+          else p = (s == arg) ? 1.0 : 0.0;
+          q = (double)A.q_probs[(size_t)(g0 + j) * A.V + s];
+          if (q > 0.0) rho = p / q;
+          else rho = (p > 0.0) ? (double)INFINITY : 0.0;
+        }
+        const double u = (double)A.u_accept[g0 + j];
+        sRej[j] = (u > rho) ? 1 : 0;
+        const double clipped = rho < 1.0 ? rho : 1.0;
+        sRatio[j] = clipped;
+        if (writer) {
+          A.ratio[g0 + j] = (float)clipped;
+          A.p_tok[g0 + j] = (float)p;
+          if (A.margin != nullptr) A.margin[g0 + j] = (float)(u - rho);
+        }
+      }
+    }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int a = gamma;
+    for (int j = 0; j < gamma; ++j) {
+      if (sRej[j]) { a = j; break; }
+    }
+    s_acc = a;
+    if (writer) {
+      A.accepted[i] = a;
+      A.n_out[i] = a + 1;
+      if (A.alpha_hat != nullptr && A.X != nullptr) {
+        if (gamma > 0) {
+          double sum = 0.0;
+          for (int j = 0; j < gamma; ++j) sum += sRatio[j];
+          const double obs = sum / (double)gamma;
+          double ah = (1.0 - A.eta) * A.alpha_hat[i] + A.eta * obs;
+          ah = ah < A.alpha_min ? A.alpha_min : ah;
+          ah = ah > A.alpha_max ? A.alpha_max : ah;
+          A.alpha_hat[i] = ah;
+        }
+        A.X[i] = (1.0 - A.beta) * A.X[i] + A.beta * (double)(a + 1);
+      }
+    }
+  }
+  __syncthreads();
+  const int a = s_acc;
+  const int row = r0 + a;                                  // the row the last token is drawn from
+  const bool resid = a < gamma;                            // correction (max(0,p-q)) or bonus (p)
+  const float selM = sM[a];
+  const int selArg = sArg[a];
+  const double invZ = (sZ[a] > 0.0) ? 1.0 / sZ[a] : 0.0;
+  if (writer)
+    for (int j = tid; j <= gamma; j += kSaThreads)
+      if (j != a) A.out_tok[r0 + j] = (j < a) ? A.draft_tok[g0 + j] : -1;
   if (A.k2 <= 0.f) {   // greedy target: the one-hot (and its residual) sits on the argmax
-    if (tid == 0) {
-      A.out_tok[s.row] = s.arg;
+    if (writer && tid == 0) {
+      A.out_tok[row] = selArg;
       if (A.margin != nullptr) A.margin[A.Gamma + i] = 1.0f;
     }
     return;
   }
-  const float* lrow = A.logits + (size_t)s.row * A.V;
-  const float* qrow = s.qrow >= 0 ? A.q_probs + (size_t)s.qrow * A.V : nullptr;
+  const float* lrow = A.logits + (size_t)row * A.V;
+  const float* qrow = resid ? A.q_probs + (size_t)(g0 + a) * A.V : nullptr;
+
+  // ---- mass of this CTA's chunk of the selected row
+  {
+    const int base = c * kSaChunk;
+    float l[kSaPerThread], q[kSaPerThread];
+    load_chunk<VEC>(lrow, base, A.V, tid, l);
+    if (resid) load_chunk<VEC>(qrow, base, A.V, tid, q, 0.f);
+    double acc = 0.0;
+#pragma unroll
+    for (int e = 0; e < kSaPerThread; ++e) acc += elem_mass(l[e], selM, A.k2, invZ, resid, resid ? q[e] : 0.f);
+    const double tot = block_sum_f64(acc, s_warp);
+    if (tid == 0) {
+      A.mass[(size_t)i * A.n_chunk + c] = tot;
+      __threadfence();
+      const int ticket = atomicAdd(&A.tickets[i], 1);
+      s_is_last = (ticket == A.n_chunk - 1) ? 1 : 0;
+    }
+  }
+  __syncthreads();
+  if (!s_is_last) return;
+  __threadfence();
+
+  // ---- the server's last CTA draws the token
   const double u = (double)A.u_sample[i];
   if (tid == 0) {
     const double* m = A.mass + (size_t)i * A.n_chunk;
     double total = 0.0;
-    for (int c = 0; c < A.n_chunk; ++c) total += m[c];
+    for (int cc = 0; cc < A.n_chunk; ++cc) total += __ldcg(m + cc);
     const double thr = u * total;
     double run = 0.0, before = 0.0;
     int pick = -1, last_pos = -1;
-    for (int c = 0; c < A.n_chunk; ++c) {
-      if (m[c] > 0.0) last_pos = c;
-      if (run + m[c] > thr) { pick = c; before = run; break; }
-      run += m[c];
+    for (int cc = 0; cc < A.n_chunk; ++cc) {
+      const double mc = __ldcg(m + cc);
+      if (mc > 0.0) last_pos = cc;
+      if (run + mc > thr) { pick = cc; before = run; break; }
+      run += mc;
     }
     if (pick < 0 && last_pos >= 0) {   // rounding left no chunk: last chunk that has mass
       pick = last_pos;
       before = 0.0;
-      for (int c = 0; c < pick; ++c) before += m[c];
+      for (int cc = 0; cc < pick; ++cc) before += __ldcg(m + cc);
     }
     s_chunk = pick; s_before = before; s_thr = thr; s_total = total;
     s_tok = INT_MAX; s_last = -1; s_lo = 0.0; s_hi = 0.0;
   }
   __syncthreads();
   if (s_chunk >= 0) {
-    scan_chunk(lrow, qrow, s_chunk * kSaChunk, A.V, s.M, A.k2, s.invZ, s_before, s_thr,
+    scan_chunk(lrow, qrow, s_chunk * kSaChunk, A.V, selM, A.k2, invZ, s_before, s_thr,
                &s_tok, &s_last, &s_lo, &s_hi, s_warp);
   } else {
     // max(0, p - q) has no mass at all: draw from p itself, scanning the whole row in order.
-    qrow = nullptr;
     double before = 0.0;   // total of p is 1 by construction of invZ
     const double thr = u;
     if (tid == 0) { s_thr = thr; s_total = 1.0; }
-    for (int c = 0; c < A.n_chunk; ++c) {
+    for (int cc = 0; cc < A.n_chunk; ++cc) {
       __syncthreads();
       if (tid == 0) s_before = before;
       __syncthreads();
-      scan_chunk(lrow, nullptr, c * kSaChunk, A.V, s.M, A.k2, s.invZ, s_before, thr,
+      scan_chunk(lrow, nullptr, cc * kSaChunk, A.V, selM, A.k2, invZ, s_before, thr,
                  &s_tok, &s_last, &s_lo, &s_hi, s_warp);
       if (s_tok != INT_MAX) break;
-      // advance `before` by this chunk's mass (recomputed in the same order by every thread 0)
       double part = 0.0;
       for (int k = 0; k < kSaThreads / 32; ++k) part += s_warp[k];
       before += part;
@@ -399,12 +381,12 @@ __global__ void __launch_bounds__(kSaThreads) sa_sample(SaSampleArgs A) {
     int tok = s_tok;
     float marg = 0.f;
     if (tok == INT_MAX) {
-      tok = s_last >= 0 ? s_last : s.arg;
+      tok = s_last >= 0 ? s_last : selArg;
     } else if (s_total > 0.0) {
-      const double a = s_thr - s_lo, b = s_hi - s_thr;
-      marg = (float)((a < b ? a : b) / s_total);
+      const double x = s_thr - s_lo, y = s_hi - s_thr;
+      marg = (float)((x < y ? x : y) / s_total);
     }
-    A.out_tok[s.row] = tok;
+    A.out_tok[row] = tok;
     if (A.margin != nullptr) A.margin[A.Gamma + i] = marg;
   }
 }
@@ -444,37 +426,30 @@ extern "C" gs_status gs_spec_accept(const float* logits, const float* q_probs, c
                    (q_probs == nullptr || reinterpret_cast<uintptr_t>(q_probs) % 16 == 0);
 
   dim3 g1(n_chunk, Tq);
-  if (vec) sa_row_stats<true><<<g1, kSaThreads, 0, st>>>(logits, V, n_chunk, k2, w.stats);
-  else sa_row_stats<false><<<g1, kSaThreads, 0, st>>>(logits, V, n_chunk, k2, w.stats);
+  if (vec) sa_row_stats<true><<<g1, kSaThreads, 0, st>>>(logits, V, n_chunk, k2, w.stats, w.tickets, N);
+  else sa_row_stats<false><<<g1, kSaThreads, 0, st>>>(logits, V, n_chunk, k2, w.stats, w.tickets, N);
 
-  SaDecideArgs A;
+  SaFinishArgs A;
   A.logits = logits; A.q_probs = q_probs; A.draft_tok = draft_tok; A.cu_q = cu_q; A.u_accept = u_accept;
-  A.N = N; A.Tq = Tq; A.V = V; A.n_chunk = n_chunk; A.tau = temperature;
+  A.u_sample = u_sample;
+  A.N = N; A.Tq = Tq; A.V = V; A.n_chunk = n_chunk; A.Gamma = Gamma; A.tau = temperature; A.k2 = k2;
   A.accepted = accepted; A.out_tok = out_tok; A.n_out = n_out;
   A.ratio = ratio; A.p_tok = p_tok; A.margin = margin;
   A.alpha_hat = alpha_hat; A.X = X; A.eta = eta; A.beta = beta; A.alpha_min = alpha_min; A.alpha_max = alpha_max;
-  A.stats = w.stats; A.sel = w.sel; A.d_status = d_status;
+  A.stats = w.stats; A.tickets = w.tickets; A.mass = w.mass; A.d_status = d_status;
   // rows of one server are bounded by Tq - (N-1); size the dynamic shared memory for that
   const size_t max_rows = (size_t)(Tq - N + 1);
   const size_t smem = align_up(3 * max_rows * 4, 8) + 2 * max_rows * 8;
-  if (smem > 200 * 1024) return GS_ERR_UNSUPPORTED;
-  if (smem > 48 * 1024) {
-    if (cudaFuncSetAttribute(sa_decide, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+  if (smem > 160 * 1024) return GS_ERR_UNSUPPORTED;
+  if (smem > 40 * 1024) {
+    if (cudaFuncSetAttribute(sa_finish<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+        cudaFuncSetAttribute(sa_finish<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return GS_ERR_CUDA;
   }
-  sa_decide<<<N, kDecideThreads, smem, st>>>(A);
-
-  if (k2 > 0.f) {
-    dim3 g3(n_chunk, N);
-    if (vec) sa_mass<true><<<g3, kSaThreads, 0, st>>>(logits, q_probs, V, n_chunk, k2, w.sel, w.mass);
-    else sa_mass<false><<<g3, kSaThreads, 0, st>>>(logits, q_probs, V, n_chunk, k2, w.sel, w.mass);
-  }
-  SaSampleArgs S;
-  S.logits = logits; S.q_probs = q_probs; S.u_sample = u_sample; S.cu_q = cu_q;
-  S.N = N; S.V = V; S.n_chunk = n_chunk; S.Gamma = Gamma; S.k2 = k2;
-  S.sel = w.sel; S.mass = w.mass; S.out_tok = out_tok; S.margin = margin;
-  sa_sample<<<N, kSaThreads, 0, st>>>(S);
-  count_launches(k2 > 0.f ? 4 : 3);
+  dim3 g2(k2 > 0.f ? n_chunk : 1, N);
+  if (vec) sa_finish<true><<<g2, kSaThreads, smem, st>>>(A);
+  else sa_finish<false><<<g2, kSaThreads, smem, st>>>(A);
+  count_launches(2);
   return launch_status();
 }
 

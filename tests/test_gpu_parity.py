@@ -238,6 +238,7 @@ def run_attn(inp):
 
 
 ATTN_CASES = [
+    ("long-split", wl.shrink(wl.CONFIGS["cfg2"], prefix_scale=1.0, N=2, name="attn_long")),  # 2 servers x 2048: many KV splits
     ("cfg2-shaped", wl.shrink(wl.CONFIGS["cfg2"], prefix_scale=0.15, name="attn2")),       # 307-key prefixes
     ("cfg3-shaped", wl.shrink(wl.CONFIGS["cfg3"], prefix_scale=0.08, name="attn3")),       # ragged 10..655
     ("cfg4-shaped", wl.shrink(wl.CONFIGS["cfg4"], prefix_scale=0.07, N=5, name="attn4")),
