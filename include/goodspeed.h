@@ -160,7 +160,7 @@ gs_status gs_spec_accept(const float* logits, const float* q_probs, const int32_
  * array of gs_spec_accept_static_capacity() bytes (2 MiB) inside the library; every GPU that
  * loads the library holds that array until the process ends.  The call itself allocates nothing.
  *   - Limit: gs_spec_accept_workspace(N, Tq, V) must not exceed the capacity (for V = 151936 that
- *     is about 3400 verify positions); larger problems return GS_ERR_WORKSPACE and launch nothing.
+ *     is about 6800 verify positions); larger problems return GS_ERR_WORKSPACE and launch nothing.
  *   - The first call on each device looks the array's device address up (with that device
  *     current); make that first call outside any stream capture.
  *   - All calls share the one array.  Nothing in it has to be cleared between calls (every word a

@@ -2,7 +2,7 @@
 // token by inverse CDF, and the estimator updates (Sec. II-A2; Eq. updatealpha, Eq. updateX).
 //
 // Two launches on one stream:
-//   1. sa_row_stats   every logit row is cut into chunks of 4096 floats; one CTA per (chunk,row)
+//   1. sa_row_stats   every logit row is cut into chunks of 8192 floats; one CTA per (chunk,row)
 //                     streams its chunk once with 16-byte loads and writes (max, argmax, sum exp).
 //   2. sa_finish      one CTA per (chunk, server).  Every CTA of a server first repeats the small
 //                     "decide" step (a warp per row merges that row's chunk statistics, evaluates
@@ -20,8 +20,8 @@
 namespace gs {
 
 constexpr int kSaThreads = 256;
-constexpr int kSaChunk = 4096;                   // floats per CTA
-constexpr int kSaPerThread = kSaChunk / kSaThreads;  // 16
+constexpr int kSaChunk = 8192;                   // floats per CTA
+constexpr int kSaPerThread = kSaChunk / kSaThreads;  // 32
 constexpr float kLog2e = 1.4426950408889634f;
 
 struct ChunkStat {   // 16 bytes
@@ -50,13 +50,13 @@ static size_t sa_layout(int N, int Tq, int V, SaWorkspace* w, char* base) {
   return off;
 }
 
-// Loads the 16 floats a thread owns in a chunk: element (k*256 + tid)*4 + j, k,j in 0..3.
+// Loads the 32 floats a thread owns in a chunk: element (k*256 + tid)*4 + j, k in 0..7, j in 0..3.
 // Out-of-range elements read as `fill`.
 template <bool VEC>
 GS_DEVINL void load_chunk(const float* __restrict__ row, int base, int V, int tid, float (&v)[kSaPerThread],
                           float fill = -INFINITY) {
 #pragma unroll
-  for (int k = 0; k < 4; ++k) {
+  for (int k = 0; k < kSaPerThread / 4; ++k) {
     int idx = base + (k * kSaThreads + tid) * 4;
     if (VEC && idx + 3 < V) {
       float4 t = __ldg(reinterpret_cast<const float4*>(row + idx));
@@ -143,6 +143,7 @@ struct SaFinishArgs {
   double* alpha_hat; double* X; double eta, beta, alpha_min, alpha_max;
   const ChunkStat* stats; int* tickets; double* mass;
   int32_t* d_status;
+  int smem_bytes;
 };
 
 // Mass of element v of the selected row: max(0, p - q) or p, in fp64 from an fp32 exponential.
@@ -152,7 +153,7 @@ GS_DEVINL double elem_mass(float l, float M, float k2, double invZ, bool resid, 
   return p;
 }
 
-// Ordered scan of one chunk: thread t owns the 16 consecutive elements base + 16 t .. +15.
+// Ordered scan of one chunk: thread t owns the 32 consecutive elements base + 32 t .. +31.
 // Returns through s_tok the smallest index whose inclusive prefix (offset by `before`) exceeds
 // thr, or INT_MAX; s_last = largest index with positive mass.
 GS_DEVINL void scan_chunk(const float* __restrict__ lrow, const float* __restrict__ qrow, int base, int V,
@@ -229,34 +230,62 @@ __global__ void __launch_bounds__(kSaThreads) sa_finish(SaFinishArgs A) {
   double* sZ = reinterpret_cast<double*>(smem_raw + off);        // [gamma+1]
   double* sRatio = sZ + (gamma + 1);                             // [gamma+1] clipped ratios
 
-  // ---- decide: a warp per row, lanes over the row's chunks
+  // ---- decide.  First every draft position's scalars are fetched in parallel (token -> logit and
+  // draft probability are dependent loads), then a warp per row merges that row's chunk statistics.
+  float* sL = reinterpret_cast<float*>(sRatio + (gamma + 1));    // [gamma] logit of the draft token
+  float* sQ = sL + (gamma + 1);                                  // [gamma] q of the draft token
+  float* sU = sQ + (gamma + 1);                                  // [gamma] uniform
+  int* sTok = reinterpret_cast<int*>(sU + (gamma + 1));          // [gamma] token, -1 if out of range
+  for (int j = tid; j < gamma; j += kSaThreads) {
+    const int s = A.draft_tok[g0 + j];
+    const bool in = (s >= 0 && s < A.V);
+    sTok[j] = in ? s : -1;
+    sL[j] = in ? A.logits[(size_t)(r0 + j) * A.V + s] : 0.f;
+    sQ[j] = in ? A.q_probs[(size_t)(g0 + j) * A.V + s] : 0.f;
+    sU[j] = A.u_accept[g0 + j];
+    if (!in && writer) set_status(A.d_status, GS_ERR_INVALID_ARG);
+  }
+  __syncthreads();
   const double inv_tau = A.tau > 0.f ? 1.0 / (double)A.tau : 0.0;
   for (int j = wid; j <= gamma; j += kSaThreads / 32) {
     const ChunkStat* st = A.stats + (size_t)(r0 + j) * A.n_chunk;
     float M = -INFINITY; int arg = INT_MAX;
-    for (int cc = lane; cc < A.n_chunk; cc += 32) argmax_merge(M, arg, st[cc].m, st[cc].arg);
-    warp_argmax(M, arg);
     double z = 0.0;
-    if (A.tau > 0.f)
-      for (int cc = lane; cc < A.n_chunk; cc += 32)
-        if (st[cc].m > -INFINITY) z += st[cc].z * exp(((double)st[cc].m - (double)M) * inv_tau);
+    if (A.n_chunk <= 64) {
+      // at most two chunks per lane: read them once
+      ChunkStat c0s, c1s;
+      c0s.m = -INFINITY; c0s.arg = INT_MAX; c0s.z = 0.0; c1s = c0s;
+      if (lane < A.n_chunk) c0s = st[lane];
+      if (lane + 32 < A.n_chunk) c1s = st[lane + 32];
+      argmax_merge(M, arg, c0s.m, c0s.arg);
+      argmax_merge(M, arg, c1s.m, c1s.arg);
+      warp_argmax(M, arg);
+      if (A.tau > 0.f) {
+        if (c0s.m > -INFINITY) z += c0s.z * exp(((double)c0s.m - (double)M) * inv_tau);
+        if (c1s.m > -INFINITY) z += c1s.z * exp(((double)c1s.m - (double)M) * inv_tau);
+      }
+    } else {
+      for (int cc = lane; cc < A.n_chunk; cc += 32) argmax_merge(M, arg, st[cc].m, st[cc].arg);
+      warp_argmax(M, arg);
+      if (A.tau > 0.f)
+        for (int cc = lane; cc < A.n_chunk; cc += 32)
+          if (st[cc].m > -INFINITY) z += st[cc].z * exp(((double)st[cc].m - (double)M) * inv_tau);
+    }
     const double Z = warp_sum_f64(z);
     if (lane == 0) {
       sM[j] = M; sArg[j] = arg; sZ[j] = Z;
       if (j < gamma) {
-        const int s = A.draft_tok[g0 + j];
+        const int s = sTok[j];
         double p = 0.0, q = 0.0, rho = 0.0;
-        if (s < 0 || s >= A.V) {
-          if (writer) set_status(A.d_status, GS_ERR_INVALID_ARG);
-        } else {
-          const float l = A.logits[(size_t)(r0 + j) * A.V + s];
+        if (s >= 0) {
+          const float l = sL[j];
           if (A.tau > 0.f) p = (Z > 0.0) ? exp(((double)l - (double)M) * inv_tau) / Z : 0.0;
           else p = (s == arg) ? 1.0 : 0.0;
-          q = (double)A.q_probs[(size_t)(g0 + j) * A.V + s];
+          q = (double)sQ[j];
           if (q > 0.0) rho = p / q;
           else rho = (p > 0.0) ? (double)INFINITY : 0.0;
         }
-        const double u = (double)A.u_accept[g0 + j];
+        const double u = (double)sU[j];
         sRej[j] = (u > rho) ? 1 : 0;
         const double clipped = rho < 1.0 ? rho : 1.0;
         sRatio[j] = clipped;
@@ -335,15 +364,21 @@ __global__ void __launch_bounds__(kSaThreads) sa_finish(SaFinishArgs A) {
 
   // ---- the server's last CTA draws the token
   const double u = (double)A.u_sample[i];
+  double* sMass = reinterpret_cast<double*>(smem_raw);           // the decide arrays are dead now
+  const bool mass_in_smem = (size_t)A.n_chunk * sizeof(double) <= (size_t)A.smem_bytes;
+  if (mass_in_smem)
+    for (int cc = tid; cc < A.n_chunk; cc += kSaThreads) sMass[cc] = __ldcg(A.mass + (size_t)i * A.n_chunk + cc);
+  __syncthreads();
   if (tid == 0) {
-    const double* m = A.mass + (size_t)i * A.n_chunk;
+    const double* gm = A.mass + (size_t)i * A.n_chunk;
+    auto mass_at = [&](int cc) { return mass_in_smem ? sMass[cc] : __ldcg(gm + cc); };
     double total = 0.0;
-    for (int cc = 0; cc < A.n_chunk; ++cc) total += __ldcg(m + cc);
+    for (int cc = 0; cc < A.n_chunk; ++cc) total += mass_at(cc);
     const double thr = u * total;
     double run = 0.0, before = 0.0;
     int pick = -1, last_pos = -1;
     for (int cc = 0; cc < A.n_chunk; ++cc) {
-      const double mc = __ldcg(m + cc);
+      const double mc = mass_at(cc);
       if (mc > 0.0) last_pos = cc;
       if (run + mc > thr) { pick = cc; before = run; break; }
       run += mc;
@@ -351,7 +386,7 @@ __global__ void __launch_bounds__(kSaThreads) sa_finish(SaFinishArgs A) {
     if (pick < 0 && last_pos >= 0) {   // rounding left no chunk: last chunk that has mass
       pick = last_pos;
       before = 0.0;
-      for (int cc = 0; cc < pick; ++cc) before += __ldcg(m + cc);
+      for (int cc = 0; cc < pick; ++cc) before += mass_at(cc);
     }
     s_chunk = pick; s_before = before; s_thr = thr; s_total = total;
     s_tok = INT_MAX; s_last = -1; s_lo = 0.0; s_hi = 0.0;
@@ -439,8 +474,9 @@ extern "C" gs_status gs_spec_accept(const float* logits, const float* q_probs, c
   A.stats = w.stats; A.tickets = w.tickets; A.mass = w.mass; A.d_status = d_status;
   // rows of one server are bounded by Tq - (N-1); size the dynamic shared memory for that
   const size_t max_rows = (size_t)(Tq - N + 1);
-  const size_t smem = align_up(3 * max_rows * 4, 8) + 2 * max_rows * 8;
+  const size_t smem = align_up(3 * max_rows * 4, 8) + 2 * max_rows * 8 + 4 * max_rows * 4;
   if (smem > 160 * 1024) return GS_ERR_UNSUPPORTED;
+  A.smem_bytes = (int)smem;
   if (smem > 40 * 1024) {
     if (cudaFuncSetAttribute(sa_finish<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
         cudaFuncSetAttribute(sa_finish<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
