@@ -156,6 +156,7 @@ GS_DEVINL double elem_mass(float l, float M, float k2, double invZ, bool resid, 
 // Ordered scan of one chunk: thread t owns the 32 consecutive elements base + 32 t .. +31.
 // Returns through s_tok the smallest index whose inclusive prefix (offset by `before`) exceeds
 // thr, or INT_MAX; s_last = largest index with positive mass.
+template <bool VEC>
 GS_DEVINL void scan_chunk(const float* __restrict__ lrow, const float* __restrict__ qrow, int base, int V,
                           float M, float k2, double invZ, double before, double thr,
                           int* s_tok, int* s_last, double* s_lo, double* s_hi, double* s_warp) {
@@ -164,11 +165,35 @@ GS_DEVINL void scan_chunk(const float* __restrict__ lrow, const float* __restric
   double w[kSaPerThread];
   double run = 0.0;
   int last_pos = -1;
+  // the thread's 32 consecutive elements: 16-byte loads when the row allows it
+  float lv[kSaPerThread], qv[kSaPerThread];
+  const bool vec_ok = VEC && first + kSaPerThread <= V;
+  if (vec_ok) {
+#pragma unroll
+    for (int e = 0; e < kSaPerThread; e += 4) {
+      const float4 t = __ldg(reinterpret_cast<const float4*>(lrow + first + e));
+      lv[e] = t.x; lv[e + 1] = t.y; lv[e + 2] = t.z; lv[e + 3] = t.w;
+    }
+    if (qrow != nullptr) {
+#pragma unroll
+      for (int e = 0; e < kSaPerThread; e += 4) {
+        const float4 t = __ldg(reinterpret_cast<const float4*>(qrow + first + e));
+        qv[e] = t.x; qv[e + 1] = t.y; qv[e + 2] = t.z; qv[e + 3] = t.w;
+      }
+    }
+  } else {
+#pragma unroll
+    for (int e = 0; e < kSaPerThread; ++e) {
+      const int idx = first + e;
+      lv[e] = idx < V ? lrow[idx] : -INFINITY;
+      qv[e] = (idx < V && qrow != nullptr) ? qrow[idx] : 0.f;
+    }
+  }
 #pragma unroll
   for (int e = 0; e < kSaPerThread; ++e) {
     const int idx = first + e;
     double x = 0.0;
-    if (idx < V) x = elem_mass(lrow[idx], M, k2, invZ, qrow != nullptr, qrow != nullptr ? qrow[idx] : 0.f);
+    if (idx < V) x = elem_mass(lv[e], M, k2, invZ, qrow != nullptr, qrow != nullptr ? qv[e] : 0.f);
     if (x > 0.0) last_pos = idx;
     run += x;
     w[e] = run;   // inclusive prefix inside the thread
@@ -393,7 +418,7 @@ __global__ void __launch_bounds__(kSaThreads) sa_finish(SaFinishArgs A) {
   }
   __syncthreads();
   if (s_chunk >= 0) {
-    scan_chunk(lrow, qrow, s_chunk * kSaChunk, A.V, selM, A.k2, invZ, s_before, s_thr,
+    scan_chunk<VEC>(lrow, qrow, s_chunk * kSaChunk, A.V, selM, A.k2, invZ, s_before, s_thr,
                &s_tok, &s_last, &s_lo, &s_hi, s_warp);
   } else {
     // max(0, p - q) has no mass at all: draw from p itself, scanning the whole row in order.
@@ -404,7 +429,7 @@ __global__ void __launch_bounds__(kSaThreads) sa_finish(SaFinishArgs A) {
       __syncthreads();
       if (tid == 0) s_before = before;
       __syncthreads();
-      scan_chunk(lrow, nullptr, cc * kSaChunk, A.V, selM, A.k2, invZ, s_before, thr,
+      scan_chunk<VEC>(lrow, nullptr, cc * kSaChunk, A.V, selM, A.k2, invZ, s_before, thr,
                  &s_tok, &s_last, &s_lo, &s_hi, s_warp);
       if (s_tok != INT_MAX) break;
       double part = 0.0;
