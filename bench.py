@@ -461,7 +461,8 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="cfg2", choices=["cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--config", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--rounds", type=int, default=1000, help="rounds of the closed loop (--config cfg5)")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--profile-small", action="store_true",
@@ -482,6 +483,20 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
     torch.cuda.set_device(local_rank)
+    if args.config == "cfg5":
+        # closed-loop scheduling: Algorithm 1 for --rounds rounds with gs_schedule in the loop
+        if rank == 0:
+            from paper_2512_09963_b200 import build as gs_build
+            from paper_2512_09963_b200.closed_loop import run_closed_loop
+            gs_build.build()
+            rep = run_closed_loop(cfg, args.rounds, device=f"cuda:{local_rank}")
+            rep.update(metric=METRIC, unit=UNIT, value=rep["verified_tokens_per_s"], n_gpus=1, dtype=cfg.dtype,
+                       data="synthetic", config={"workload": "cfg5", "servers": cfg.N, "budget_C": cfg.C,
+                                                 "drift": "true alpha ~ Beta(4,2) redrawn every 100 rounds",
+                                                 "timing": "GPU time of the four library calls per round (CUDA events); "
+                                                           "input generation between rounds is untimed"})
+            print(json.dumps(rep), flush=True)
+        return
     if world > 1:
         import torch.distributed as dist
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")

@@ -1,0 +1,152 @@
+"""Closed-loop harness: Algorithm 1 run round after round with the scheduler in the loop.
+
+The draft servers are simulated (workloads.py): each has a true acceptance rate alpha_i that is
+redrawn every `epoch` rounds, and draft noise calibrated to it.  Every round the harness builds the
+inputs for the allocation S(t) the scheduler produced in the previous round (gamma_i = S_i(t)),
+runs the library's round on the GPU, and feeds S(t+1) back.  It holds no verification arithmetic:
+the GPU does the round; the harness only generates inputs and keeps running sums for the report.
+"""
+from __future__ import annotations
+
+import dataclasses
+import math
+
+import numpy as np
+import torch
+
+from . import binding as B
+from . import workloads as wl
+
+
+class ClosedLoop:
+    def __init__(self, cfg: wl.VerifyConfig, device="cuda", epoch=100, eta=0.1, beta=0.5, s_min=0):
+        self.cfg, self.dev, self.epoch = cfg, torch.device(device), epoch
+        self.eta, self.beta = eta, beta
+        N, C = cfg.N, cfg.C
+        self.N, self.C = N, C
+        self.max_new = C + 1                                   # a single server can get the whole budget
+        self.prefix = int(cfg.prefix_lo)
+        dt = wl.torch_dtype(cfg)
+        self.W = wl.make_layer(cfg, self.dev)["W"]
+        per = self.prefix + self.max_new
+        self.K_pool = wl._normal(cfg, "K_pool", 0, (N, per, cfg.Hkv, cfg.hd), 1.0, dt, self.dev)
+        self.V_pool = wl._normal(cfg, "V_pool", 0, (N, per, cfg.Hkv, cfg.hd), 1.0, dt, self.dev)
+        self.s_min = torch.full((N,), int(s_min), dtype=torch.int32, device=self.dev)
+        self.s_max = torch.full((N,), C, dtype=torch.int32, device=self.dev)
+        self.S = np.full(N, C // N, dtype=np.int64)            # S_i(0) = floor(C/N)
+        self._sigma_epoch = -1
+        # device state and output buffers sized for the largest round
+        Tq_max = C + N
+        f32, i32, f64 = torch.float32, torch.int32, torch.float64
+        self.alpha_hat = torch.full((N,), 0.5, dtype=f64, device=self.dev)
+        self.X = torch.ones(N, dtype=f64, device=self.dev)
+        self.O = torch.empty((Tq_max, cfg.Hq, cfg.hd), dtype=dt, device=self.dev)
+        self.logits = torch.empty((Tq_max * cfg.V,), dtype=f32, device=self.dev)
+        self.accepted = torch.empty(N, dtype=i32, device=self.dev)
+        self.out_tok = torch.empty(Tq_max, dtype=i32, device=self.dev)
+        self.n_out = torch.empty(N, dtype=i32, device=self.dev)
+        self.ratio = torch.empty(max(C, 1), dtype=f32, device=self.dev)
+        self.p_tok = torch.empty(max(C, 1), dtype=f32, device=self.dev)
+        self.S_next = torch.empty(N, dtype=i32, device=self.dev)
+        self.d_status = torch.zeros(1, dtype=i32, device=self.dev)
+        gsdt = B.GS_F32 if dt == torch.float32 else B.GS_BF16
+        total_kv_max = N * self.prefix + Tq_max
+        self.max_kv_len = self.prefix + self.max_new
+        ws = lambda n: torch.empty(max(int(n), 256), dtype=torch.uint8, device=self.dev)
+        self.ws_attn = ws(B.gs_verify_attn_workspace(N, Tq_max, total_kv_max, self.max_kv_len, cfg.Hq, cfg.Hkv,
+                                                     cfg.hd, gsdt))
+        self.ws_head = ws(B.gs_lm_head_workspace(Tq_max, cfg.d, cfg.V, gsdt))
+        self.ws_acc = ws(B.gs_spec_accept_workspace(N, Tq_max, cfg.V))
+
+    # ---------------------------------------------------------------- inputs of round t
+    def true_alpha(self, t):
+        return wl.draw_true_alpha(self.cfg, t // self.epoch)
+
+    def sigma(self, t):
+        e = t // self.epoch
+        if e != self._sigma_epoch:
+            self._sigma = wl.calibrate_sigma(self.true_alpha(t), self.cfg.V, self.cfg.tau)
+            self._sigma_epoch = e
+        return self._sigma
+
+    def make_inputs(self, t, gamma):
+        cfg = self.cfg
+        gamma = np.asarray(gamma, np.int64)
+        n_new = gamma + 1
+        cu_q = np.concatenate([[0], np.cumsum(n_new)]).astype(np.int32)
+        cu_kv = np.concatenate([[0], np.cumsum(self.prefix + n_new)]).astype(np.int32)
+        Tq = int(cu_q[-1])
+        dt = wl.torch_dtype(cfg)
+        inp = {
+            "Q": wl._normal(cfg, "Q", t, (Tq, cfg.Hq, cfg.hd), 1.0, dt, self.dev),
+            "K": torch.cat([self.K_pool[i, :self.prefix + int(n_new[i])] for i in range(self.N)]).contiguous(),
+            "V": torch.cat([self.V_pool[i, :self.prefix + int(n_new[i])] for i in range(self.N)]).contiguous(),
+            "cu_q": torch.from_numpy(cu_q).to(self.dev), "cu_kv": torch.from_numpy(cu_kv).to(self.dev),
+            "H": wl.make_hidden(cfg, Tq, t, self.dev), "W": self.W, "tau": float(cfg.tau),
+            "gamma": gamma,
+        }
+        logits = wl.library_logits(inp["H"], self.W)
+        inp["q_probs"], inp["draft_tok"] = wl.simulate_drafts(cfg, logits, inp["cu_q"], self.sigma(t), cfg.tau, t)
+        G = int(gamma.sum())
+        inp["u_accept"] = torch.from_numpy(wl.open_uniform(wl._rng(cfg, "u_accept", t), G)).to(self.dev)
+        inp["u_sample"] = torch.from_numpy(wl.open_uniform(wl._rng(cfg, "u_sample", t), self.N)).to(self.dev)
+        return inp
+
+    # ---------------------------------------------------------------- one round on the GPU
+    def gpu_round(self, inp):
+        cfg = self.cfg
+        Tq = inp["Q"].shape[0]
+        G = Tq - self.N
+        O = self.O[:Tq]
+        logits = self.logits[:Tq * cfg.V].view(Tq, cfg.V)
+        B.gs_verify_attn(inp["Q"], inp["K"], inp["V"], O, inp["cu_q"], inp["cu_kv"], self.max_kv_len,
+                         1.0 / math.sqrt(cfg.hd), self.ws_attn, self.d_status)
+        B.gs_lm_head_logits(inp["H"], inp["W"], logits, self.ws_head, self.d_status)
+        B.gs_spec_accept(logits, inp["q_probs"], inp["draft_tok"], inp["cu_q"], inp["u_accept"], inp["u_sample"],
+                         inp["tau"], self.accepted, self.out_tok[:Tq], self.n_out, self.ratio[:G], self.p_tok[:G],
+                         None, self.alpha_hat, self.X, self.eta, self.beta, ws=self.ws_acc, d_status=self.d_status)
+        B.gs_schedule(self.X, self.alpha_hat, self.C, self.S_next, self.s_min, self.s_max, self.d_status)
+        return O, logits
+
+
+def jain(x):
+    x = np.asarray(x, dtype=np.float64)
+    return float(x.sum() ** 2 / (len(x) * (x * x).sum()))
+
+
+def run_closed_loop(cfg: wl.VerifyConfig, rounds: int, device="cuda", on_round=None):
+    """Runs `rounds` rounds; returns the report dict.  on_round(t, loop, inp, O, logits) is called after
+    each round is enqueued and synchronised (tests use it to compare with the oracle in lock-step)."""
+    loop = ClosedLoop(cfg, device)
+    N = cfg.N
+    tot = np.zeros(N)
+    x_hist, X_hist = [], []
+    gpu_ms = 0.0
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    drafted = 0
+    for t in range(rounds):
+        inp = loop.make_inputs(t, loop.S)
+        e0.record()
+        O, logits = loop.gpu_round(inp)
+        e1.record()
+        torch.cuda.synchronize()
+        gpu_ms += e0.elapsed_time(e1)
+        assert int(loop.d_status.item()) == 0, "device status"
+        if on_round is not None:
+            on_round(t, loop, inp, O, logits)
+        x = loop.n_out.cpu().numpy().astype(np.float64)
+        tot += x
+        drafted += int(loop.S.sum())
+        x_hist.append(x)
+        X_hist.append(loop.X.cpu().numpy().copy())
+        loop.S = loop.S_next.cpu().numpy().astype(np.int64)
+    xbar = tot / rounds
+    xh, Xh = np.asarray(x_hist), np.asarray(X_hist)
+    ma = lambda a: np.convolve(a, np.ones(10) / 10, mode="valid") if len(a) >= 10 else a
+    est_err = float(np.mean(np.abs(ma(xh.sum(1)) - ma(Xh.sum(1))))) if rounds >= 10 else None
+    return {"rounds": rounds, "goodput_per_server": [float(v) for v in xbar], "jain": jain(xbar),
+            "utility_sum_log": float(np.log(xbar).sum()), "gpu_ms_per_round": gpu_ms / rounds,
+            "verified_tokens_per_s": drafted / (gpu_ms * 1e-3), "goodput_tokens_per_s": float(tot.sum()) / (gpu_ms * 1e-3),
+            "estimated_vs_realised_goodput_ma10_abs_err": est_err,
+            "final_alpha_hat": [float(v) for v in loop.alpha_hat.cpu().numpy()],
+            "true_alpha_last_epoch": [float(v) for v in loop.true_alpha(rounds - 1)]}
