@@ -8,8 +8,9 @@
 //     P = 2^(S*c - m)    four softmax warps, one thread per row: tcgen05.ld, causal mask, online
 //                        max/sum, bf16 P written to shared memory in the swizzled operand layout
 //     O += P V           tcgen05.mma  M=128, N=128, K=64    (V read as an MN-major operand)
-// K/V tiles arrive by TMA through a 2-stage ring.  Two CTAs share an SM, so one CTA's softmax
-// overlaps the other's MMAs and loads.  An item whose server needs a single KV split normalises and
+// K/V tiles arrive by TMA through a 4-stage ring (one CTA per SM).  S and P are double-buffered and
+// the MMA thread issues S of tile j+1 before it waits for P of tile j, so the tensor core, the
+// softmax warps and the loads of later tiles overlap.  An item whose server needs a single KV split normalises and
 // stores its rows directly; otherwise it writes an unnormalised partial (m, l, O) to the workspace
 // and takes a ticket, and the last split of a (server, position block, KV head) to finish merges
 // them (nobody waits).  CTAs are persistent and stride over the items.
@@ -25,12 +26,12 @@ constexpr int kAtThreads = 192;          // warp 0 TMA, warp 1 MMA, warps 2-5 so
 constexpr int kAtTile = 64;              // keys per tile
 constexpr int kAtHd = 128;
 constexpr int kAtRows = 128;
-constexpr int kAtStages = 2;
+constexpr int kAtStages = 4;
 constexpr uint32_t kAtQBytes = kAtRows * kAtHd * 2;            // 32 KB: two halves of 64 columns
 constexpr uint32_t kAtPBytes = kAtRows * kAtTile * 2;          // 16 KB
 constexpr uint32_t kAtKvBytes = 2 * kAtTile * kAtHd * 2;       // K + V of one tile: 32 KB
-constexpr uint32_t kAtSmem = kAtQBytes + kAtPBytes + kAtStages * kAtKvBytes + 256;
-constexpr uint32_t kAtTmemCols = 256;    // S: columns 0..63, O: columns 64..191
+constexpr uint32_t kAtSmem = kAtQBytes + 2 * kAtPBytes + kAtStages * kAtKvBytes + 256;   // 192.25 KB: one CTA per SM
+constexpr uint32_t kAtTmemCols = 256;    // S: two buffers, columns 0..63 and 64..127; O: columns 128..255
 constexpr int kAtPartStride = kAtHd + 4; // floats per partial row: O[128], m, l, 2 pad (rows stay 16-byte aligned)
 constexpr float kAtLog2e = 1.4426950408889634f;
 
@@ -109,18 +110,20 @@ GS_DEVINL AttnItem attn_find_item(const AttnTcParams& P, int id) {
   return it;
 }
 
-__global__ void __launch_bounds__(kAtThreads, 2)
+__global__ void __launch_bounds__(kAtThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant__ CUtensorMap tmapK,
                const __grid_constant__ CUtensorMap tmapV, const AttnTcParams P) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = smem_u32(smem_raw);
-  const uint32_t q_base = base, p_base = base + kAtQBytes, kv_base = p_base + kAtPBytes;
+  const uint32_t q_base = base, p_base = base + kAtQBytes, kv_base = p_base + 2 * kAtPBytes;
   const uint32_t bars = kv_base + kAtStages * kAtKvBytes;
-  // barriers: 0 q_full, 1 item_done, 2 s_full, 3 p_full, 4 o_full, 5.. kv_full[S], kv_empty[S],
-  //           then epi_a, epi_b (the 128 softmax threads meet twice per item that took a ticket)
+  // barriers: 0 q_full, 1 item_done, 2-3 s_full[2], 4-5 p_full[2], 6 o_full, 7 pv_done,
+  //           8.. kv_full[S], kv_empty[S], then epi_a, epi_b (the 128 softmax threads meet twice
+  //           per item that took a ticket)
   auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
-  constexpr int kEpiA = 5 + 2 * kAtStages, kEpiB = kEpiA + 1;
-  uint8_t* tail = smem_raw + (bars - base) + 8 * (7 + 2 * kAtStages);
+  constexpr int kSFull = 2, kPFull = 4, kOFull = 6, kPvDone = 7, kKvFull = 8, kKvEmpty = 8 + kAtStages;
+  constexpr int kEpiA = 8 + 2 * kAtStages, kEpiB = kEpiA + 1;
+  uint8_t* tail = smem_raw + (bars - base) + 8 * (10 + 2 * kAtStages);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 4);
   volatile int* s_last = reinterpret_cast<volatile int*>(tail + 8);
@@ -131,8 +134,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant_
     return;
   }
   if (threadIdx.x == 0) {
-    mbar_init(bar(0), 1); mbar_init(bar(1), 4); mbar_init(bar(2), 1); mbar_init(bar(3), 4); mbar_init(bar(4), 1);
-    for (int s = 0; s < kAtStages; ++s) { mbar_init(bar(5 + s), 1); mbar_init(bar(5 + kAtStages + s), 1); }
+    mbar_init(bar(0), 1); mbar_init(bar(1), 4);
+    mbar_init(bar(kSFull), 1); mbar_init(bar(kSFull + 1), 1);
+    mbar_init(bar(kPFull), 4); mbar_init(bar(kPFull + 1), 4);
+    mbar_init(bar(kOFull), 1); mbar_init(bar(kPvDone), 1);
+    for (int s = 0; s < kAtStages; ++s) { mbar_init(bar(kKvFull + s), 1); mbar_init(bar(kKvEmpty + s), 1); }
     mbar_init(bar(kEpiA), 128); mbar_init(bar(kEpiB), 128);
     *abort_flag = 0;
     fence_barrier_init();
@@ -147,7 +153,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_S = tmem_base, tmem_O = tmem_base + 64u;
+  const uint32_t tmem_S = tmem_base, tmem_O = tmem_base + 128u;     // S buffer b at tmem_S + 64 b
 
   // Every role walks the same item sequence and recomputes the item from the offsets.
   if (warp == 0) {
@@ -176,15 +182,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant_
         tma_load_3d(q_base, &tmapQ, 0, it.g * P.G, it.q_row0, bar(0));
         tma_load_3d(q_base + kAtQBytes / 2, &tmapQ, 64, it.g * P.G, it.q_row0, bar(0));
         for (int j = 0; j < it.n_tiles; ++j) {
-          if (!mbar_wait(bar(5 + kAtStages + st), ph ^ 1u, abort_flag)) { ok = false; break; }
-          mbar_arrive_expect_tx(bar(5 + st), kAtKvBytes);
+          if (!mbar_wait(bar(kKvEmpty + st), ph ^ 1u, abort_flag)) { ok = false; break; }
+          mbar_arrive_expect_tx(bar(kKvFull + st), kAtKvBytes);
           const uint32_t dst = kv_base + st * kAtKvBytes;
           const int key = it.kv0 + (it.tile0 + j) * kAtTile;
           const int col = it.g * kAtHd;
-          tma_load_2d(dst, &tmapK, col, key, bar(5 + st));
-          tma_load_2d(dst + 8192u, &tmapK, col + 64, key, bar(5 + st));
-          tma_load_2d(dst + 16384u, &tmapV, col, key, bar(5 + st));
-          tma_load_2d(dst + 24576u, &tmapV, col + 64, key, bar(5 + st));
+          tma_load_2d(dst, &tmapK, col, key, bar(kKvFull + st));
+          tma_load_2d(dst + 8192u, &tmapK, col + 64, key, bar(kKvFull + st));
+          tma_load_2d(dst + 16384u, &tmapV, col, key, bar(kKvFull + st));
+          tma_load_2d(dst + 24576u, &tmapV, col + 64, key, bar(kKvFull + st));
           if (++st == kAtStages) { st = 0; ph ^= 1u; }
         }
         ++n_item;
@@ -201,9 +207,22 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant_
       const uint64_t dp = smem_desc_sw128(p_base, 16u, 1024u);
       const uint64_t dk0 = smem_desc_sw128(kv_base, 16u, 1024u);
       const uint64_t dv0 = smem_desc_sw128(kv_base + 16384u, 8192u, 1024u); // 64-column blocks 8 KB apart
-      uint32_t st = 0, ph = 0;
+      // Two cursors walk the K/V ring: S = Q K^T runs one tile ahead of O += P V, so the tensor core
+      // computes the next tile's scores while the softmax warps work on the current tile.
+      uint32_t st_s = 0, ph_s = 0, st_v = 0;
       int n_item = 0, n_tile_total = 0;
       bool ok = true;
+      auto issue_S = [&](uint32_t stage, int n) {
+        const uint64_t dk = dk0 + (uint64_t)(stage * (kAtKvBytes >> 4));
+        const uint32_t d = tmem_S + (uint32_t)(n & 1) * 64u;
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {     // 128 head dims = 8 x 16; second half 16 KB (Q) / 8 KB (K) further
+          const uint64_t a = dq + (uint64_t)((kk >> 2) * (16384 >> 4) + (kk & 3) * 2);
+          const uint64_t b = dk + (uint64_t)((kk >> 2) * (8192 >> 4) + (kk & 3) * 2);
+          umma_bf16(d, a, b, idesc_s, kk > 0 ? 1u : 0u);
+        }
+        umma_commit(bar(kSFull + (n & 1)));                                  // S of tile n ready
+      };
       for (int id = blockIdx.x; id < P.max_items && ok; id += gridDim.x) {
         const AttnItem it = attn_find_item(P, id);
         if (!it.valid) break;
@@ -211,30 +230,34 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant_
         if (!mbar_wait(bar(0), (uint32_t)n_item & 1u, abort_flag)) { ok = false; break; }      // Q landed
         if (n_item > 0 && !mbar_wait(bar(1), (uint32_t)(n_item - 1) & 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
+        if (!mbar_wait(bar(kKvFull + st_s), ph_s, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        issue_S(st_s, n_tile_total);
+        if (++st_s == kAtStages) { st_s = 0; ph_s ^= 1u; }
         for (int j = 0; j < it.n_tiles; ++j, ++n_tile_total) {
-          if (!mbar_wait(bar(5 + st), ph, abort_flag)) { ok = false; break; }
-          tc_fence_after();
-          const uint64_t dk = dk0 + (uint64_t)(st * (kAtKvBytes >> 4));
-          const uint64_t dv = dv0 + (uint64_t)(st * (kAtKvBytes >> 4));
-#pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {     // 128 head dims = 8 x 16; second half 16 KB (Q) / 8 KB (K) further
-            const uint64_t a = dq + (uint64_t)((kk >> 2) * (16384 >> 4) + (kk & 3) * 2);
-            const uint64_t b = dk + (uint64_t)((kk >> 2) * (8192 >> 4) + (kk & 3) * 2);
-            umma_bf16(tmem_S, a, b, idesc_s, kk > 0 ? 1u : 0u);
+          const int n = n_tile_total;
+          if (j + 1 < it.n_tiles) {
+            // The S buffer of tile n+1 was last read for tile n-1, whose P has been consumed below.
+            if (!mbar_wait(bar(kKvFull + st_s), ph_s, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            issue_S(st_s, n + 1);
+            if (++st_s == kAtStages) { st_s = 0; ph_s ^= 1u; }
           }
-          umma_commit(bar(2));                                               // S ready
-          if (!mbar_wait(bar(3), (uint32_t)n_tile_total & 1u, abort_flag)) { ok = false; break; }   // P ready
+          if (!mbar_wait(bar(kPFull + (n & 1)), (uint32_t)(n >> 1) & 1u, abort_flag)) { ok = false; break; }   // P ready
           tc_fence_after();
+          const uint64_t dv = dv0 + (uint64_t)(st_v * (kAtKvBytes >> 4));
+          const uint64_t dpn = dp + (uint64_t)((n & 1) * (kAtPBytes >> 4));
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk) {     // 64 keys = 4 x 16: P +32 bytes, V +2 groups of 8 keys
-            const uint64_t a = dp + (uint64_t)(kk * 2);
+            const uint64_t a = dpn + (uint64_t)(kk * 2);
             const uint64_t b = dv + (uint64_t)(kk * (2048 >> 4));
             umma_bf16(tmem_O, a, b, idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
           }
-          umma_commit(bar(5 + kAtStages + st));                              // K/V stage free
-          if (++st == kAtStages) { st = 0; ph ^= 1u; }
+          umma_commit(bar(kKvEmpty + st_v));                                 // K/V stage free
+          umma_commit(bar(kPvDone));                                         // O holds tiles <= n
+          if (++st_v == kAtStages) st_v = 0;
         }
-        if (ok) umma_commit(bar(4));                                         // O complete
+        if (ok) umma_commit(bar(kOFull));                                    // O complete
         ++n_item;
       }
       if (!ok) { const uint64_t t0 = global_timer_ns(); while (global_timer_ns() - t0 < 200000ull) { } }
@@ -255,38 +278,44 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant_
       const bool row_ok = r < R;
       const int t = it.tg * P.TB + r / P.G;              // position index inside the server
       const int last_visible = it.L + t;                 // keys 0..L+t
-      float m_run = -INFINITY, l_run = 0.f;
+      float m_run = -INFINITY, l_run = 0.f;     // reference maximum (scaled, log2 units) and running sum
+      const int first_visible_end = it.L + it.tg * P.TB;      // last key the block's FIRST position sees
       for (int j = 0; j < it.n_tiles; ++j, ++n_tile_total) {
-        if (!mbar_wait(bar(2), (uint32_t)n_tile_total & 1u, abort_flag)) { ok = false; break; }
+        const int n = n_tile_total;
+        if (!mbar_wait(bar(kSFull + (n & 1)), (uint32_t)(n >> 1) & 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
-        uint32_t sv[64];
+        float sv[64];
         {
           uint32_t (*s4)[16] = reinterpret_cast<uint32_t (*)[16]>(sv);
-          tmem_ld16(tmem_S + lane_addr + 0, s4[0]);
-          tmem_ld16(tmem_S + lane_addr + 16, s4[1]);
-          tmem_ld16(tmem_S + lane_addr + 32, s4[2]);
-          tmem_ld16(tmem_S + lane_addr + 48, s4[3]);
+          const uint32_t src = tmem_S + (uint32_t)(n & 1) * 64u + lane_addr;
+          tmem_ld16(src + 0, s4[0]);
+          tmem_ld16(src + 16, s4[1]);
+          tmem_ld16(src + 32, s4[2]);
+          tmem_ld16(src + 48, s4[3]);
           tmem_ld_wait();
         }
         const int key0 = (it.tile0 + j) * kAtTile;       // key index inside the server
+        // Only tiles that reach past what the block's first position sees need the causal mask.
+        if (key0 + kAtTile - 1 > first_visible_end) {
+#pragma unroll
+          for (int c = 0; c < 64; ++c) sv[c] = (key0 + c <= last_visible) ? sv[c] : -INFINITY;
+        }
         float tmax = -INFINITY;
 #pragma unroll
-        for (int c = 0; c < 64; ++c) {
-          float s = __uint_as_float(sv[c]) * P.scale_log2;
-          s = (key0 + c <= last_visible) ? s : -INFINITY;
-          sv[c] = __float_as_uint(s);
-          tmax = fmaxf(tmax, s);
-        }
+        for (int c = 0; c < 64; ++c) tmax = fmaxf(tmax, sv[c]);
+        tmax *= P.scale_log2;                            // the scale is positive
         // The reference maximum only moves when the tile maximum exceeds it by more than 2^8:
         // P stays below 256, the final O/l is unchanged, and O in TMEM is rescaled rarely.
         const float m_new = (tmax > m_run + 8.f) ? tmax : m_run;
         const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
         const float corr = (m_run == -INFINITY) ? 0.f : fast_exp2(m_run - m_use);
         // Rescale O when this warp has a row whose reference moved (never for the first tile, whose
-        // P V product overwrites O).  All earlier MMAs have completed: S of this tile was
-        // committed after them.
+        // P V product overwrites O).  S runs a tile ahead, so the product of the previous tile
+        // may still be in flight: wait for it first.  The next product waits for this tile's P.
         const bool need = row_ok && j > 0 && (m_new > m_run);
         if (__any_sync(0xffffffffu, need)) {
+          if (!mbar_wait(bar(kPvDone), (uint32_t)(n - 1) & 1u, abort_flag)) { ok = false; break; }
+          tc_fence_after();
           const float f = need ? corr : 1.f;
 #pragma unroll
           for (int c0 = 0; c0 < kAtHd; c0 += 16) {
@@ -304,14 +333,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant_
           tmem_st_wait();
         }
         float lsum = 0.f;
-        const uint32_t prow = p_base + (uint32_t)r * 128u;
+        const uint32_t prow = p_base + (uint32_t)(n & 1) * kAtPBytes + (uint32_t)r * 128u;
+        const float neg_m = -m_use;
 #pragma unroll
         for (int ch = 0; ch < 8; ++ch) {               // 8 keys = 16 bytes per chunk
           uint32_t pk[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            const float p0 = fast_exp2(__uint_as_float(sv[ch * 8 + 2 * e]) - m_use);
-            const float p1 = fast_exp2(__uint_as_float(sv[ch * 8 + 2 * e + 1]) - m_use);
+            const float p0 = fast_exp2(fmaf(sv[ch * 8 + 2 * e], P.scale_log2, neg_m));
+            const float p1 = fast_exp2(fmaf(sv[ch * 8 + 2 * e + 1], P.scale_log2, neg_m));
             lsum += p0 + p1;
             __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
             pk[e] = *reinterpret_cast<uint32_t*>(&b);
@@ -324,11 +354,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant_
         fence_proxy_async();          // generic-proxy writes of P -> visible to the tensor core
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(bar(3));
+        if (lane == 0) mbar_arrive(bar(kPFull + (n & 1)));
       }
       if (!ok) break;
       // epilogue
-      if (!mbar_wait(bar(4), (uint32_t)n_item & 1u, abort_flag)) { ok = false; break; }
+      if (!mbar_wait(bar(kOFull), (uint32_t)n_item & 1u, abort_flag)) { ok = false; break; }
       tc_fence_after();
       __nv_bfloat16* orow = P.O + ((size_t)(it.q_row0 + r / P.G) * P.Hq + it.g * P.G + (r % P.G)) * kAtHd;
       float* out = P.part + ((size_t)id * kAtRows + r) * kAtPartStride;
@@ -484,7 +514,7 @@ inline AttnTcPlan attn_tc_plan(int N, int Tq, int total_kv, int max_kv_len, int 
   AttnTcPlan pl;
   const int G = Hq / Hkv;
   pl.TB = 128 / G;
-  const int slots = 2 * sm_count();
+  const int slots = sm_count();                        // one CTA per SM
   const int heads_total = max(1, N * Hkv);
   const int tiles_avg = max(1, (total_kv / max(1, N) + kAtTile - 1) / kAtTile);
   const int nsplit_target = max(1, slots / heads_total);
