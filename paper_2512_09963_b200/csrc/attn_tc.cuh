@@ -4,11 +4,13 @@
 // up to 128/G positions are packed into the 128 rows of one MMA tile (row = position * G + head in
 // group), so K and V of a KV head are read once for the whole group and all positions.  Per tile
 // of 64 keys:
-//     S = Q K^T          tcgen05.mma  M=128, N=64,  K=128   (Q, K from shared memory, S in TMEM)
+//     S = Q K^T          tcgen05.mma  M=128, N=64,  K=128   (Q from tensor memory, K from shared memory)
 //     P = 2^(S*c - m)    four softmax warps, one thread per row: tcgen05.ld, causal mask, online
-//                        max/sum, bf16 P written to shared memory in the swizzled operand layout
-//     O += P V           tcgen05.mma  M=128, N=128, K=64    (V read as an MN-major operand)
-// K/V tiles arrive by TMA through a 4-stage ring (one CTA per SM).  S and P are double-buffered and
+//                        max/sum, bf16 P stored back to tensor memory (tcgen05.st)
+//     O += P V           tcgen05.mma  M=128, N=128, K=64    (P from tensor memory, V an MN-major operand)
+// Shared memory carries only K and V: with Q and P as shared-memory operands the tensor core's
+// operand reads (Q again for every tile) plus the TMA writes exceeded the 128 B/clk of an SM.
+// K/V tiles arrive by TMA through a 6-stage ring (one CTA per SM).  S and P are double-buffered and
 // the MMA thread issues S of tile j+1 before it waits for P of tile j, so the tensor core, the
 // softmax warps and the loads of later tiles overlap.  An item whose server needs a single KV split normalises and
 // stores its rows directly; otherwise it writes an unnormalised partial (m, l, O) to the workspace
@@ -26,12 +28,14 @@ constexpr int kAtThreads = 192;          // warp 0 TMA, warp 1 MMA, warps 2-5 so
 constexpr int kAtTile = 64;              // keys per tile
 constexpr int kAtHd = 128;
 constexpr int kAtRows = 128;
-constexpr int kAtStages = 4;
-constexpr uint32_t kAtQBytes = kAtRows * kAtHd * 2;            // 32 KB: two halves of 64 columns
-constexpr uint32_t kAtPBytes = kAtRows * kAtTile * 2;          // 16 KB
+constexpr int kAtStages = 6;
 constexpr uint32_t kAtKvBytes = 2 * kAtTile * kAtHd * 2;       // K + V of one tile: 32 KB
-constexpr uint32_t kAtSmem = kAtQBytes + 2 * kAtPBytes + kAtStages * kAtKvBytes + 256;   // 192.25 KB: one CTA per SM
-constexpr uint32_t kAtTmemCols = 256;    // S: two buffers, columns 0..63 and 64..127; O: columns 128..255
+constexpr uint32_t kAtSmem = kAtStages * kAtKvBytes + 256;     // 192.25 KB: one CTA per SM
+// Tensor memory (512 columns): S two buffers 0..63 / 64..127, O 128..255, Q (bf16 pairs) 256..319,
+// P (bf16 pairs) two buffers 320..351 / 352..383.  Q and P are A operands read from tensor memory,
+// so shared memory carries only K and V.
+constexpr uint32_t kAtTmemCols = 512;
+constexpr uint32_t kAtColS = 0, kAtColO = 128, kAtColQ = 256, kAtColP = 320;
 constexpr int kAtPartStride = kAtHd + 4; // floats per partial row: O[128], m, l, 2 pad (rows stay 16-byte aligned)
 constexpr float kAtLog2e = 1.4426950408889634f;
 
@@ -41,6 +45,7 @@ struct AttnTcParams {
   float* part;              // [items][128][132]
   int* tickets;             // [groups] splits of a (server, position block, KV head) that are done
   __nv_bfloat16* O;
+  const __nv_bfloat16* Q;
   int32_t* d_status;
   int N, Tq, total_kv, max_kv_len, Hq, Hkv, G, TB;   // TB = 128 / G query positions per item
   int tiles_per_chunk;      // KV tiles per split (upper bound; splits of a server are balanced)
@@ -111,11 +116,11 @@ GS_DEVINL AttnItem attn_find_item(const AttnTcParams& P, int id) {
 }
 
 __global__ void __launch_bounds__(kAtThreads, 1)
-attn_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant__ CUtensorMap tmapK,
-               const __grid_constant__ CUtensorMap tmapV, const AttnTcParams P) {
+attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant__ CUtensorMap tmapV,
+               const AttnTcParams P) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = smem_u32(smem_raw);
-  const uint32_t q_base = base, p_base = base + kAtQBytes, kv_base = p_base + 2 * kAtPBytes;
+  const uint32_t kv_base = base;
   const uint32_t bars = kv_base + kAtStages * kAtKvBytes;
   // barriers: 0 q_full, 1 item_done, 2-3 s_full[2], 4-5 p_full[2], 6 o_full, 7 pv_done,
   //           8.. kv_full[S], kv_empty[S], then epi_a, epi_b (the 128 softmax threads meet twice
@@ -134,7 +139,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant_
     return;
   }
   if (threadIdx.x == 0) {
-    mbar_init(bar(0), 1); mbar_init(bar(1), 4);
+    mbar_init(bar(0), 4); mbar_init(bar(1), 4);
     mbar_init(bar(kSFull), 1); mbar_init(bar(kSFull + 1), 1);
     mbar_init(bar(kPFull), 4); mbar_init(bar(kPFull + 1), 4);
     mbar_init(bar(kOFull), 1); mbar_init(bar(kPvDone), 1);
@@ -143,7 +148,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant_
     *abort_flag = 0;
     fence_barrier_init();
     fence_proxy_async();
-    tma_prefetch_desc(&tmapQ); tma_prefetch_desc(&tmapK); tma_prefetch_desc(&tmapV);
+    tma_prefetch_desc(&tmapK); tma_prefetch_desc(&tmapV);
   }
   if (warp == 1) {
     tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kAtTmemCols);
@@ -153,7 +158,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_S = tmem_base, tmem_O = tmem_base + 128u;     // S buffer b at tmem_S + 64 b
+  const uint32_t tmem_S = tmem_base + kAtColS, tmem_O = tmem_base + kAtColO;     // S buffer b at tmem_S + 64 b
+  const uint32_t tmem_Q = tmem_base + kAtColQ, tmem_P = tmem_base + kAtColP;     // P buffer b at tmem_P + 32 b
 
   // Every role walks the same item sequence and recomputes the item from the offsets.
   if (warp == 0) {
@@ -176,11 +182,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant_
         const AttnItem it = attn_find_item(P, id);
         if (!it.valid) break;
         if (it.n_tiles == 0) continue;
-        // Q may be overwritten once the previous item is completely done
-        if (n_item > 0 && !mbar_wait(bar(1), (uint32_t)(n_item - 1) & 1u, abort_flag)) { ok = false; break; }
-        mbar_arrive_expect_tx(bar(0), kAtQBytes);
-        tma_load_3d(q_base, &tmapQ, 0, it.g * P.G, it.q_row0, bar(0));
-        tma_load_3d(q_base + kAtQBytes / 2, &tmapQ, 64, it.g * P.G, it.q_row0, bar(0));
         for (int j = 0; j < it.n_tiles; ++j) {
           if (!mbar_wait(bar(kKvEmpty + st), ph ^ 1u, abort_flag)) { ok = false; break; }
           mbar_arrive_expect_tx(bar(kKvFull + st), kAtKvBytes);
@@ -203,8 +204,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant_
     if (lane == 0) {
       const uint32_t idesc_s = idesc_bf16(128, kAtTile, false, false);     // S = Q K^T, both K-major
       const uint32_t idesc_o = idesc_bf16(128, kAtHd, false, true);        // O = P V, V is MN-major
-      const uint64_t dq = smem_desc_sw128(q_base, 16u, 1024u);
-      const uint64_t dp = smem_desc_sw128(p_base, 16u, 1024u);
       const uint64_t dk0 = smem_desc_sw128(kv_base, 16u, 1024u);
       const uint64_t dv0 = smem_desc_sw128(kv_base + 16384u, 8192u, 1024u); // 64-column blocks 8 KB apart
       // Two cursors walk the K/V ring: S = Q K^T runs one tile ahead of O += P V, so the tensor core
@@ -216,10 +215,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant_
         const uint64_t dk = dk0 + (uint64_t)(stage * (kAtKvBytes >> 4));
         const uint32_t d = tmem_S + (uint32_t)(n & 1) * 64u;
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {     // 128 head dims = 8 x 16; second half 16 KB (Q) / 8 KB (K) further
-          const uint64_t a = dq + (uint64_t)((kk >> 2) * (16384 >> 4) + (kk & 3) * 2);
+        for (int kk = 0; kk < 8; ++kk) {     // 128 head dims = 8 x 16: Q +8 TMEM columns, K +32 bytes / second half 8 KB further
           const uint64_t b = dk + (uint64_t)((kk >> 2) * (8192 >> 4) + (kk & 3) * 2);
-          umma_bf16(d, a, b, idesc_s, kk > 0 ? 1u : 0u);
+          umma_bf16_ts(d, tmem_Q + (uint32_t)(kk * 8), b, idesc_s, kk > 0 ? 1u : 0u);
         }
         umma_commit(bar(kSFull + (n & 1)));                                  // S of tile n ready
       };
@@ -227,8 +225,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant_
         const AttnItem it = attn_find_item(P, id);
         if (!it.valid) break;
         if (it.n_tiles == 0) continue;
-        if (!mbar_wait(bar(0), (uint32_t)n_item & 1u, abort_flag)) { ok = false; break; }      // Q landed
-        if (n_item > 0 && !mbar_wait(bar(1), (uint32_t)(n_item - 1) & 1u, abort_flag)) { ok = false; break; }
+        // Q of this item sits in tensor memory (written by the softmax warps after they have
+        // drained O of the previous item)
+        if (!mbar_wait(bar(0), (uint32_t)n_item & 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         if (!mbar_wait(bar(kKvFull + st_s), ph_s, abort_flag)) { ok = false; break; }
         tc_fence_after();
@@ -246,12 +245,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant_
           if (!mbar_wait(bar(kPFull + (n & 1)), (uint32_t)(n >> 1) & 1u, abort_flag)) { ok = false; break; }   // P ready
           tc_fence_after();
           const uint64_t dv = dv0 + (uint64_t)(st_v * (kAtKvBytes >> 4));
-          const uint64_t dpn = dp + (uint64_t)((n & 1) * (kAtPBytes >> 4));
+          const uint32_t pn = tmem_P + (uint32_t)(n & 1) * 32u;
 #pragma unroll
-          for (int kk = 0; kk < 4; ++kk) {     // 64 keys = 4 x 16: P +32 bytes, V +2 groups of 8 keys
-            const uint64_t a = dpn + (uint64_t)(kk * 2);
+          for (int kk = 0; kk < 4; ++kk) {     // 64 keys = 4 x 16: P +8 TMEM columns, V +2 groups of 8 keys
             const uint64_t b = dv + (uint64_t)(kk * (2048 >> 4));
-            umma_bf16(tmem_O, a, b, idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
+            umma_bf16_ts(tmem_O, pn + (uint32_t)(kk * 8), b, idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
           }
           umma_commit(bar(kKvEmpty + st_v));                                 // K/V stage free
           umma_commit(bar(kPvDone));                                         // O holds tiles <= n
@@ -278,6 +276,27 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant_
       const bool row_ok = r < R;
       const int t = it.tg * P.TB + r / P.G;              // position index inside the server
       const int last_visible = it.L + t;                 // keys 0..L+t
+      // This thread's query row goes to tensor memory as packed bf16 pairs (the A operand of
+      // S = Q K^T).  The previous item's MMAs are finished: its O was drained above.
+      {
+        const uint4* qrow = reinterpret_cast<const uint4*>(
+            P.Q + ((size_t)(it.q_row0 + r / P.G) * P.Hq + it.g * P.G + (r % P.G)) * kAtHd);
+#pragma unroll
+        for (int c0 = 0; c0 < 64; c0 += 16) {            // 16 columns = 32 head dims = 4 x 16 bytes
+          uint32_t w[16];
+#pragma unroll
+          for (int v4 = 0; v4 < 4; ++v4) {
+            uint4 x = make_uint4(0u, 0u, 0u, 0u);
+            if (row_ok) x = __ldg(qrow + c0 / 4 + v4);
+            w[4 * v4] = x.x; w[4 * v4 + 1] = x.y; w[4 * v4 + 2] = x.z; w[4 * v4 + 3] = x.w;
+          }
+          tmem_st16(tmem_Q + lane_addr + c0, w);
+        }
+        tmem_st_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(0));
+      }
       float m_run = -INFINITY, l_run = 0.f;     // reference maximum (scaled, log2 units) and running sum
       const int first_visible_end = it.L + it.tg * P.TB;      // last key the block's FIRST position sees
       for (int j = 0; j < it.n_tiles; ++j, ++n_tile_total) {
@@ -333,25 +352,24 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant_
           tmem_st_wait();
         }
         float lsum = 0.f;
-        const uint32_t prow = p_base + (uint32_t)(n & 1) * kAtPBytes + (uint32_t)r * 128u;
         const float neg_m = -m_use;
+        const uint32_t pdst = tmem_P + (uint32_t)(n & 1) * 32u + lane_addr;
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {               // 8 keys = 16 bytes per chunk
-          uint32_t pk[4];
+        for (int h = 0; h < 2; ++h) {                  // 32 keys = 16 columns of bf16 pairs per store
+          uint32_t pk[16];
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float p0 = fast_exp2(fmaf(sv[ch * 8 + 2 * e], P.scale_log2, neg_m));
-            const float p1 = fast_exp2(fmaf(sv[ch * 8 + 2 * e + 1], P.scale_log2, neg_m));
+          for (int e = 0; e < 16; ++e) {
+            const float p0 = fast_exp2(fmaf(sv[h * 32 + 2 * e], P.scale_log2, neg_m));
+            const float p1 = fast_exp2(fmaf(sv[h * 32 + 2 * e + 1], P.scale_log2, neg_m));
             lsum += p0 + p1;
             __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
             pk[e] = *reinterpret_cast<uint32_t*>(&b);
           }
-          const uint32_t addr = prow + (uint32_t)((ch ^ (r & 7)) << 4);   // 128-byte swizzle
-          asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
+          tmem_st16(pdst + (uint32_t)h * 16u, pk);
         }
+        tmem_st_wait();
         l_run = l_run * corr + lsum;
         m_run = m_new;
-        fence_proxy_async();          // generic-proxy writes of P -> visible to the tensor core
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(kPFull + (n & 1)));
@@ -390,10 +408,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant_
           }
         }
       }
-      // TMEM and the Q buffer are free again: the next item may start while the splits are merged
       tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(1));
       if (!single) {
         if (row_ok) { out[kAtHd] = m_run; out[kAtHd + 1] = l_run; }
         // One ticket per group: the CTA that takes the last one finds the other splits' rows
@@ -545,28 +560,19 @@ inline gs_status launch_attn_tc(const void* Q, const void* K, const void* V, voi
   P.tickets = static_cast<int*>(ws);
   P.part = reinterpret_cast<float*>(static_cast<char*>(ws) + pl.ticket_bytes);
   P.O = static_cast<__nv_bfloat16*>(O);
+  P.Q = static_cast<const __nv_bfloat16*>(Q);
   P.N = N; P.Tq = Tq; P.total_kv = total_kv; P.max_kv_len = max_kv_len; P.Hq = Hq; P.Hkv = Hkv;
   P.G = Hq / Hkv; P.TB = pl.TB; P.tiles_per_chunk = pl.tiles_per_chunk; P.max_items = pl.max_items;
   P.scale_log2 = scale * kAtLog2e;
   auto enc = tensor_map_encoder();
   if (enc == nullptr) return GS_ERR_CUDA;
-  CUtensorMap tmQ, tmK, tmV;
-  {  // Q [Tq][Hq][hd]: box = 64 columns x G heads x TB positions -> rows (position, head in group)
-    cuuint64_t dims[3] = {(cuuint64_t)kAtHd, (cuuint64_t)Hq, (cuuint64_t)Tq};
-    cuuint64_t strides[2] = {(cuuint64_t)kAtHd * 2, (cuuint64_t)Hq * kAtHd * 2};
-    cuuint32_t box[3] = {64, (cuuint32_t)P.G, (cuuint32_t)P.TB};
-    cuuint32_t es[3] = {1, 1, 1};
-    if (enc(&tmQ, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(Q), dims, strides, box, es,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return GS_ERR_CUDA;
-  }
+  CUtensorMap tmK, tmV;
   // K, V [total_kv][Hkv*hd]: box = 64 columns x 64 keys
   if (!make_tmap_bf16_2d(&tmK, K, (uint64_t)total_kv, (uint64_t)Hkv * kAtHd, (uint64_t)Hkv * kAtHd, kAtTile, 64) ||
       !make_tmap_bf16_2d(&tmV, V, (uint64_t)total_kv, (uint64_t)Hkv * kAtHd, (uint64_t)Hkv * kAtHd, kAtTile, 64))
     return GS_ERR_CUDA;
   if (cudaMemsetAsync(P.tickets, 0, pl.ticket_bytes, st) != cudaSuccess) return GS_ERR_CUDA;
-  attn_tc_kernel<<<pl.grid, kAtThreads, kAtSmem, st>>>(tmQ, tmK, tmV, P);
+  attn_tc_kernel<<<pl.grid, kAtThreads, kAtSmem, st>>>(tmK, tmV, P);
   if (cudaGetLastError() != cudaSuccess) return GS_ERR_CUDA;
   count_launches(1);
   return launch_status();
