@@ -3,14 +3,14 @@
 // Work item = (server, block of query positions, KV head, KV split).  The GQA group's queries of
 // up to 128/G positions are packed into the 128 rows of one MMA tile (row = position * G + head in
 // group), so K and V of a KV head are read once for the whole group and all positions.  Per tile
-// of 64 keys:
-//     S = Q K^T          tcgen05.mma  M=128, N=64,  K=128   (Q from tensor memory, K from shared memory)
+// of 128 keys:
+//     S = Q K^T          tcgen05.mma  M=128, N=128, K=128   (Q from tensor memory, K from shared memory)
 //     P = 2^(S*c - m)    four softmax warps, one thread per row: tcgen05.ld, causal mask, online
 //                        max/sum, bf16 P stored back to tensor memory (tcgen05.st)
-//     O += P V           tcgen05.mma  M=128, N=128, K=64    (P from tensor memory, V an MN-major operand)
+//     O += P V           tcgen05.mma  M=128, N=128, K=128   (P from tensor memory, V an MN-major operand)
 // Shared memory carries only K and V: with Q and P as shared-memory operands the tensor core's
 // operand reads (Q again for every tile) plus the TMA writes exceeded the 128 B/clk of an SM.
-// K/V tiles arrive by TMA through a 6-stage ring (one CTA per SM).  S and P are double-buffered and
+// K/V tiles (128 keys) arrive by TMA through a 3-stage ring (one CTA per SM).  S and P are double-buffered and
 // the MMA thread issues S of tile j+1 before it waits for P of tile j, so the tensor core, the
 // softmax warps and the loads of later tiles overlap.  An item whose server needs a single KV split normalises and
 // stores its rows directly; otherwise it writes an unnormalised partial (m, l, O) to the workspace
@@ -25,17 +25,18 @@
 namespace gs {
 
 constexpr int kAtThreads = 192;          // warp 0 TMA, warp 1 MMA, warps 2-5 softmax/epilogue
-constexpr int kAtTile = 64;              // keys per tile
+constexpr int kAtTile = 128;             // keys per tile
 constexpr int kAtHd = 128;
 constexpr int kAtRows = 128;
-constexpr int kAtStages = 6;
-constexpr uint32_t kAtKvBytes = 2 * kAtTile * kAtHd * 2;       // K + V of one tile: 32 KB
+constexpr int kAtStages = 3;
+constexpr uint32_t kAtKvBytes = 2 * kAtTile * kAtHd * 2;       // K + V of one tile: 64 KB
 constexpr uint32_t kAtSmem = kAtStages * kAtKvBytes + 256;     // 192.25 KB: one CTA per SM
-// Tensor memory (512 columns): S two buffers 0..63 / 64..127, O 128..255, Q (bf16 pairs) 256..319,
-// P (bf16 pairs) two buffers 320..351 / 352..383.  Q and P are A operands read from tensor memory,
-// so shared memory carries only K and V.
+// Tensor memory (512 columns): S two buffers 0..127 / 128..255 (P, as bf16 pairs, overwrites the first
+// 64 columns of its S buffer once the thread has read its scores), O 256..383, Q (bf16 pairs) 384..447.
+// Q and P are A operands read from tensor memory, so shared memory carries only K and V.
 constexpr uint32_t kAtTmemCols = 512;
-constexpr uint32_t kAtColS = 0, kAtColO = 128, kAtColQ = 256, kAtColP = 320;
+constexpr uint32_t kAtColS = 0, kAtColO = 256, kAtColQ = 384;
+constexpr uint32_t kAtHalfBytes = kAtTile * 128u;              // one 64-column half of a K or V tile
 constexpr int kAtPartStride = kAtHd + 4; // floats per partial row: O[128], m, l, 2 pad (rows stay 16-byte aligned)
 constexpr float kAtLog2e = 1.4426950408889634f;
 
@@ -158,8 +159,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_S = tmem_base + kAtColS, tmem_O = tmem_base + kAtColO;     // S buffer b at tmem_S + 64 b
-  const uint32_t tmem_Q = tmem_base + kAtColQ, tmem_P = tmem_base + kAtColP;     // P buffer b at tmem_P + 32 b
+  const uint32_t tmem_S = tmem_base + kAtColS, tmem_O = tmem_base + kAtColO;     // S buffer b at tmem_S + 128 b
+  const uint32_t tmem_Q = tmem_base + kAtColQ;
 
   // Every role walks the same item sequence and recomputes the item from the offsets.
   if (warp == 0) {
@@ -189,9 +190,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
           const int key = it.kv0 + (it.tile0 + j) * kAtTile;
           const int col = it.g * kAtHd;
           tma_load_2d(dst, &tmapK, col, key, bar(kKvFull + st));
-          tma_load_2d(dst + 8192u, &tmapK, col + 64, key, bar(kKvFull + st));
-          tma_load_2d(dst + 16384u, &tmapV, col, key, bar(kKvFull + st));
-          tma_load_2d(dst + 24576u, &tmapV, col + 64, key, bar(kKvFull + st));
+          tma_load_2d(dst + kAtHalfBytes, &tmapK, col + 64, key, bar(kKvFull + st));
+          tma_load_2d(dst + 2 * kAtHalfBytes, &tmapV, col, key, bar(kKvFull + st));
+          tma_load_2d(dst + 3 * kAtHalfBytes, &tmapV, col + 64, key, bar(kKvFull + st));
           if (++st == kAtStages) { st = 0; ph ^= 1u; }
         }
         ++n_item;
@@ -205,7 +206,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
       const uint32_t idesc_s = idesc_bf16(128, kAtTile, false, false);     // S = Q K^T, both K-major
       const uint32_t idesc_o = idesc_bf16(128, kAtHd, false, true);        // O = P V, V is MN-major
       const uint64_t dk0 = smem_desc_sw128(kv_base, 16u, 1024u);
-      const uint64_t dv0 = smem_desc_sw128(kv_base + 16384u, 8192u, 1024u); // 64-column blocks 8 KB apart
+      const uint64_t dv0 = smem_desc_sw128(kv_base + 2 * kAtHalfBytes, kAtHalfBytes, 1024u); // 64-column blocks one half apart
       // Two cursors walk the K/V ring: S = Q K^T runs one tile ahead of O += P V, so the tensor core
       // computes the next tile's scores while the softmax warps work on the current tile.
       uint32_t st_s = 0, ph_s = 0, st_v = 0;
@@ -213,10 +214,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
       bool ok = true;
       auto issue_S = [&](uint32_t stage, int n) {
         const uint64_t dk = dk0 + (uint64_t)(stage * (kAtKvBytes >> 4));
-        const uint32_t d = tmem_S + (uint32_t)(n & 1) * 64u;
+        const uint32_t d = tmem_S + (uint32_t)(n & 1) * 128u;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {     // 128 head dims = 8 x 16: Q +8 TMEM columns, K +32 bytes / second half 8 KB further
-          const uint64_t b = dk + (uint64_t)((kk >> 2) * (8192 >> 4) + (kk & 3) * 2);
+          const uint64_t b = dk + (uint64_t)((kk >> 2) * (kAtHalfBytes >> 4) + (kk & 3) * 2);
           umma_bf16_ts(d, tmem_Q + (uint32_t)(kk * 8), b, idesc_s, kk > 0 ? 1u : 0u);
         }
         umma_commit(bar(kSFull + (n & 1)));                                  // S of tile n ready
@@ -245,9 +246,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
           if (!mbar_wait(bar(kPFull + (n & 1)), (uint32_t)(n >> 1) & 1u, abort_flag)) { ok = false; break; }   // P ready
           tc_fence_after();
           const uint64_t dv = dv0 + (uint64_t)(st_v * (kAtKvBytes >> 4));
-          const uint32_t pn = tmem_P + (uint32_t)(n & 1) * 32u;
+          const uint32_t pn = tmem_S + (uint32_t)(n & 1) * 128u;       // P sits where the scores were
 #pragma unroll
-          for (int kk = 0; kk < 4; ++kk) {     // 64 keys = 4 x 16: P +8 TMEM columns, V +2 groups of 8 keys
+          for (int kk = 0; kk < kAtTile / 16; ++kk) {     // 16 keys per step: P +8 TMEM columns, V +2 groups of 8 keys
             const uint64_t b = dv + (uint64_t)(kk * (2048 >> 4));
             umma_bf16_ts(tmem_O, pn + (uint32_t)(kk * 8), b, idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
           }
@@ -303,25 +304,23 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
         const int n = n_tile_total;
         if (!mbar_wait(bar(kSFull + (n & 1)), (uint32_t)(n >> 1) & 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
-        float sv[64];
+        float sv[kAtTile];
         {
           uint32_t (*s4)[16] = reinterpret_cast<uint32_t (*)[16]>(sv);
-          const uint32_t src = tmem_S + (uint32_t)(n & 1) * 64u + lane_addr;
-          tmem_ld16(src + 0, s4[0]);
-          tmem_ld16(src + 16, s4[1]);
-          tmem_ld16(src + 32, s4[2]);
-          tmem_ld16(src + 48, s4[3]);
+          const uint32_t src = tmem_S + (uint32_t)(n & 1) * 128u + lane_addr;
+#pragma unroll
+          for (int c0 = 0; c0 < kAtTile / 16; ++c0) tmem_ld16(src + 16 * c0, s4[c0]);
           tmem_ld_wait();
         }
         const int key0 = (it.tile0 + j) * kAtTile;       // key index inside the server
         // Only tiles that reach past what the block's first position sees need the causal mask.
         if (key0 + kAtTile - 1 > first_visible_end) {
 #pragma unroll
-          for (int c = 0; c < 64; ++c) sv[c] = (key0 + c <= last_visible) ? sv[c] : -INFINITY;
+          for (int c = 0; c < kAtTile; ++c) sv[c] = (key0 + c <= last_visible) ? sv[c] : -INFINITY;
         }
         float tmax = -INFINITY;
 #pragma unroll
-        for (int c = 0; c < 64; ++c) tmax = fmaxf(tmax, sv[c]);
+        for (int c = 0; c < kAtTile; ++c) tmax = fmaxf(tmax, sv[c]);
         tmax *= P.scale_log2;                            // the scale is positive
         // The reference maximum only moves when the tile maximum exceeds it by more than 2^8:
         // P stays below 256, the final O/l is unchanged, and O in TMEM is rescaled rarely.
@@ -353,9 +352,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
         }
         float lsum = 0.f;
         const float neg_m = -m_use;
-        const uint32_t pdst = tmem_P + (uint32_t)(n & 1) * 32u + lane_addr;
+        const uint32_t pdst = tmem_S + (uint32_t)(n & 1) * 128u + lane_addr;   // over this thread's own scores
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {                  // 32 keys = 16 columns of bf16 pairs per store
+        for (int h = 0; h < kAtTile / 32; ++h) {       // 32 keys = 16 columns of bf16 pairs per store
           uint32_t pk[16];
 #pragma unroll
           for (int e = 0; e < 16; ++e) {
@@ -567,7 +566,7 @@ inline gs_status launch_attn_tc(const void* Q, const void* K, const void* V, voi
   auto enc = tensor_map_encoder();
   if (enc == nullptr) return GS_ERR_CUDA;
   CUtensorMap tmK, tmV;
-  // K, V [total_kv][Hkv*hd]: box = 64 columns x 64 keys
+  // K, V [total_kv][Hkv*hd]: box = 64 columns x 128 keys
   if (!make_tmap_bf16_2d(&tmK, K, (uint64_t)total_kv, (uint64_t)Hkv * kAtHd, (uint64_t)Hkv * kAtHd, kAtTile, 64) ||
       !make_tmap_bf16_2d(&tmV, V, (uint64_t)total_kv, (uint64_t)Hkv * kAtHd, (uint64_t)Hkv * kAtHd, kAtTile, 64))
     return GS_ERR_CUDA;
