@@ -116,6 +116,26 @@ GS_DEVINL AttnItem attn_find_item(const AttnTcParams& P, int id) {
   return it;
 }
 
+// 2^x on the FMA pipe (x <= 127): floor by the 1.5*2^23 trick, a cubic for 2^f on [0,1] (relative
+// error 9e-5, far below bf16 resolution) and an integer add to the exponent.  One softmax thread
+// needs 128 exponentials per tile and the special-function unit delivers 4 per clock per SM
+// quarter, so every fourth exponential is evaluated here instead.
+GS_DEVINL float poly_exp2(float x) {
+  x = fmaxf(x, -126.f);
+  const float t = (x - 0.5f) + 12582912.f;
+  const float n = t - 12582912.f;                       // floor(x) (x itself on exact integers + 0.5 ties)
+  const float f = x - n;
+  const float p = fmaf(f, fmaf(f, fmaf(f, 0.07706156f, 0.22765097f), 0.69511545f), 1.0f);
+  const int e = __float_as_int(t) - 0x4B400000;         // floor(x) as an integer
+  return __int_as_float(__float_as_int(p) + (e << 23));
+}
+
+// Two non-negative floats to a packed bf16 pair (round half up on the dropped bits) with integer
+// ops only: the conversion instruction shares the special-function pipe with the exponentials.
+GS_DEVINL uint32_t pack_bf16_pos(float lo, float hi) {
+  return __byte_perm(__float_as_uint(lo) + 0x8000u, __float_as_uint(hi) + 0x8000u, 0x7632);
+}
+
 __global__ void __launch_bounds__(kAtThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant__ CUtensorMap tmapV,
                const AttnTcParams P) {
@@ -304,23 +324,31 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
         const int n = n_tile_total;
         if (!mbar_wait(bar(kSFull + (n & 1)), (uint32_t)(n >> 1) & 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
-        float sv[kAtTile];
-        {
-          uint32_t (*s4)[16] = reinterpret_cast<uint32_t (*)[16]>(sv);
-          const uint32_t src = tmem_S + (uint32_t)(n & 1) * 128u + lane_addr;
-#pragma unroll
-          for (int c0 = 0; c0 < kAtTile / 16; ++c0) tmem_ld16(src + 16 * c0, s4[c0]);
-          tmem_ld_wait();
-        }
+        // The tile is walked twice in chunks of 32 columns (rolled loops: one softmax warp per
+        // scheduler executes straight from the instruction cache, and a fully unrolled 128-column
+        // body does not fit it): first the row maximum, then exponentials and P.
+        const uint32_t s_src = tmem_S + (uint32_t)(n & 1) * 128u + lane_addr;
         const int key0 = (it.tile0 + j) * kAtTile;       // key index inside the server
         // Only tiles that reach past what the block's first position sees need the causal mask.
-        if (key0 + kAtTile - 1 > first_visible_end) {
+        const bool masked = key0 + kAtTile - 1 > first_visible_end;
+        float tm[8];
 #pragma unroll
-          for (int c = 0; c < kAtTile; ++c) sv[c] = (key0 + c <= last_visible) ? sv[c] : -INFINITY;
+        for (int c = 0; c < 8; ++c) tm[c] = -INFINITY;
+#pragma unroll 1
+        for (int c4 = 0; c4 < kAtTile / 32; ++c4) {
+          float sv[32];
+          uint32_t (*s4)[16] = reinterpret_cast<uint32_t (*)[16]>(sv);
+          tmem_ld16(s_src + 32 * c4, s4[0]);
+          tmem_ld16(s_src + 32 * c4 + 16, s4[1]);
+          tmem_ld_wait();
+          if (masked) {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) sv[c] = (key0 + 32 * c4 + c <= last_visible) ? sv[c] : -INFINITY;
+          }
+#pragma unroll
+          for (int c = 0; c < 32; ++c) tm[c & 7] = fmaxf(tm[c & 7], sv[c]);
         }
-        float tmax = -INFINITY;
-#pragma unroll
-        for (int c = 0; c < kAtTile; ++c) tmax = fmaxf(tmax, sv[c]);
+        float tmax = fmaxf(fmaxf(fmaxf(tm[0], tm[1]), fmaxf(tm[2], tm[3])), fmaxf(fmaxf(tm[4], tm[5]), fmaxf(tm[6], tm[7])));
         tmax *= P.scale_log2;                            // the scale is positive
         // The reference maximum only moves when the tile maximum exceeds it by more than 2^8:
         // P stays below 256, the final O/l is unchanged, and O in TMEM is rescaled rarely.
@@ -350,24 +378,34 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
           }
           tmem_st_wait();
         }
-        float lsum = 0.f;
+        float ls[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
         const float neg_m = -m_use;
-        const uint32_t pdst = tmem_S + (uint32_t)(n & 1) * 128u + lane_addr;   // over this thread's own scores
+        // P (bf16 pairs, 16 columns per chunk) overwrites score columns this thread has already read.
+#pragma unroll 1
+        for (int c4 = 0; c4 < kAtTile / 32; ++c4) {
+          float sv[32];
+          uint32_t (*s4)[16] = reinterpret_cast<uint32_t (*)[16]>(sv);
+          tmem_ld16(s_src + 32 * c4, s4[0]);
+          tmem_ld16(s_src + 32 * c4 + 16, s4[1]);
+          tmem_ld_wait();
+          if (masked) {
 #pragma unroll
-        for (int h = 0; h < kAtTile / 32; ++h) {       // 32 keys = 16 columns of bf16 pairs per store
+            for (int c = 0; c < 32; ++c) sv[c] = (key0 + 32 * c4 + c <= last_visible) ? sv[c] : -INFINITY;
+          }
           uint32_t pk[16];
 #pragma unroll
           for (int e = 0; e < 16; ++e) {
-            const float p0 = fast_exp2(fmaf(sv[h * 32 + 2 * e], P.scale_log2, neg_m));
-            const float p1 = fast_exp2(fmaf(sv[h * 32 + 2 * e + 1], P.scale_log2, neg_m));
-            lsum += p0 + p1;
-            __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
-            pk[e] = *reinterpret_cast<uint32_t*>(&b);
+            const float x0 = fmaf(sv[2 * e], P.scale_log2, neg_m);
+            const float x1 = fmaf(sv[2 * e + 1], P.scale_log2, neg_m);
+            const float p0 = fast_exp2(x0);
+            const float p1 = (e & 1) ? poly_exp2(x1) : fast_exp2(x1);       // every fourth on the FMA pipe
+            ls[e & 7] += p0 + p1;
+            pk[e] = pack_bf16_pos(p0, p1);
           }
-          tmem_st16(pdst + (uint32_t)h * 16u, pk);
+          tmem_st16(s_src + 16 * c4, pk);
         }
         tmem_st_wait();
-        l_run = l_run * corr + lsum;
+        l_run = l_run * corr + (((ls[0] + ls[1]) + (ls[2] + ls[3])) + ((ls[4] + ls[5]) + (ls[6] + ls[7])));
         m_run = m_new;
         tc_fence_before();
         __syncwarp();
