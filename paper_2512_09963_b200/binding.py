@@ -31,6 +31,7 @@ SIGNATURES = {
                             _vp, _sz, _vp, _vp]),
     "gs_lm_head_workspace": (_sz, [_i, _i, _i, _i]),
     "gs_lm_head_configure": (_i, [_i, _i, _i]),
+    "gs_lm_head_select": (_i, [_i]),
     "gs_lm_head_logits": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _vp, _sz, _vp, _vp]),
     "gs_spec_accept_workspace": (_sz, [_i, _i, _i]),
     "gs_spec_accept": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _f, _i, _i, _i,
@@ -136,6 +137,10 @@ def gs_lm_head_workspace(T, d, V, dt) -> int:
 
 def gs_lm_head_configure(m_tiles: int = 0, stages: int = 0, k_rows: int = 0):
     _check("gs_lm_head_configure", lib().gs_lm_head_configure(int(m_tiles), int(stages), int(k_rows)))
+
+
+def gs_lm_head_select(variant: int = 0):
+    _check("gs_lm_head_select", lib().gs_lm_head_select(int(variant)))
 
 
 def gs_lm_head_logits(H, W, logits, ws, d_status=None):

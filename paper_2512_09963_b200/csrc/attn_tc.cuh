@@ -221,18 +221,19 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
     }
     __syncwarp();
   } else if (warp == 1) {
-    // ------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      const uint32_t idesc_s = idesc_bf16(128, kAtTile, false, false);     // S = Q K^T, both K-major
-      const uint32_t idesc_o = idesc_bf16(128, kAtHd, false, true);        // O = P V, V is MN-major
-      const uint64_t dk0 = smem_desc_sw128(kv_base, 16u, 1024u);
-      const uint64_t dv0 = smem_desc_sw128(kv_base + 2 * kAtHalfBytes, kAtHalfBytes, 1024u); // 64-column blocks one half apart
-      // Two cursors walk the K/V ring: S = Q K^T runs one tile ahead of O += P V, so the tensor core
-      // computes the next tile's scores while the softmax warps work on the current tile.
-      uint32_t st_s = 0, ph_s = 0, st_v = 0;
-      int n_item = 0, n_tile_total = 0;
-      bool ok = true;
-      auto issue_S = [&](uint32_t stage, int n) {
+    // ------------------------------------------------ MMA issuer: the whole warp walks the loops (loop
+    // state and descriptors stay warp-uniform), one elected lane issues
+    const uint32_t idesc_s = idesc_bf16(128, kAtTile, false, false);     // S = Q K^T, both K-major
+    const uint32_t idesc_o = idesc_bf16(128, kAtHd, false, true);        // O = P V, V is MN-major
+    const uint64_t dk0 = smem_desc_sw128(kv_base, 16u, 1024u);
+    const uint64_t dv0 = smem_desc_sw128(kv_base + 2 * kAtHalfBytes, kAtHalfBytes, 1024u); // 64-column blocks one half apart
+    // Two cursors walk the K/V ring: S = Q K^T runs one tile ahead of O += P V, so the tensor core
+    // computes the next tile's scores while the softmax warps work on the current tile.
+    uint32_t st_s = 0, ph_s = 0, st_v = 0;
+    int n_item = 0, n_tile_total = 0;
+    bool ok = true;
+    auto issue_S = [&](uint32_t stage, int n) {
+      if (elect_one()) {
         const uint64_t dk = dk0 + (uint64_t)(stage * (kAtKvBytes >> 4));
         const uint32_t d = tmem_S + (uint32_t)(n & 1) * 128u;
 #pragma unroll
@@ -241,30 +242,33 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
           umma_bf16_ts(d, tmem_Q + (uint32_t)(kk * 8), b, idesc_s, kk > 0 ? 1u : 0u);
         }
         umma_commit(bar(kSFull + (n & 1)));                                  // S of tile n ready
-      };
-      for (int id = blockIdx.x; id < P.max_items && ok; id += gridDim.x) {
-        const AttnItem it = attn_find_item(P, id);
-        if (!it.valid) break;
-        if (it.n_tiles == 0) continue;
-        // Q of this item sits in tensor memory (written by the softmax warps after they have
-        // drained O of the previous item)
-        if (!mbar_wait(bar(0), (uint32_t)n_item & 1u, abort_flag)) { ok = false; break; }
-        tc_fence_after();
-        if (!mbar_wait(bar(kKvFull + st_s), ph_s, abort_flag)) { ok = false; break; }
-        tc_fence_after();
-        issue_S(st_s, n_tile_total);
-        if (++st_s == kAtStages) { st_s = 0; ph_s ^= 1u; }
-        for (int j = 0; j < it.n_tiles; ++j, ++n_tile_total) {
-          const int n = n_tile_total;
-          if (j + 1 < it.n_tiles) {
-            // The S buffer of tile n+1 was last read for tile n-1, whose P has been consumed below.
-            if (!mbar_wait(bar(kKvFull + st_s), ph_s, abort_flag)) { ok = false; break; }
-            tc_fence_after();
-            issue_S(st_s, n + 1);
-            if (++st_s == kAtStages) { st_s = 0; ph_s ^= 1u; }
-          }
-          if (!mbar_wait(bar(kPFull + (n & 1)), (uint32_t)(n >> 1) & 1u, abort_flag)) { ok = false; break; }   // P ready
+      }
+      __syncwarp();
+    };
+    for (int id = blockIdx.x; id < P.max_items && ok; id += gridDim.x) {
+      const AttnItem it = attn_find_item(P, id);
+      if (!it.valid) break;
+      if (it.n_tiles == 0) continue;
+      // Q of this item sits in tensor memory (written by the softmax warps after they have
+      // drained O of the previous item)
+      if (!mbar_wait_warp(bar(0), (uint32_t)n_item & 1u, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      if (!mbar_wait_warp(bar(kKvFull + st_s), ph_s, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      issue_S(st_s, n_tile_total);
+      if (++st_s == kAtStages) { st_s = 0; ph_s ^= 1u; }
+      for (int j = 0; j < it.n_tiles; ++j, ++n_tile_total) {
+        const int n = n_tile_total;
+        if (j + 1 < it.n_tiles) {
+          // The S buffer of tile n+1 was last read for tile n-1, whose P has been consumed below.
+          if (!mbar_wait_warp(bar(kKvFull + st_s), ph_s, abort_flag)) { ok = false; break; }
           tc_fence_after();
+          issue_S(st_s, n + 1);
+          if (++st_s == kAtStages) { st_s = 0; ph_s ^= 1u; }
+        }
+        if (!mbar_wait_warp(bar(kPFull + (n & 1)), (uint32_t)(n >> 1) & 1u, abort_flag)) { ok = false; break; }   // P ready
+        tc_fence_after();
+        if (elect_one()) {
           const uint64_t dv = dv0 + (uint64_t)(st_v * (kAtKvBytes >> 4));
           const uint32_t pn = tmem_S + (uint32_t)(n & 1) * 128u;       // P sits where the scores were
 #pragma unroll
@@ -274,13 +278,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
           }
           umma_commit(bar(kKvEmpty + st_v));                                 // K/V stage free
           umma_commit(bar(kPvDone));                                         // O holds tiles <= n
-          if (++st_v == kAtStages) st_v = 0;
+          if (j + 1 == it.n_tiles) umma_commit(bar(kOFull));                 // O complete
         }
-        if (ok) umma_commit(bar(kOFull));                                    // O complete
-        ++n_item;
+        __syncwarp();
+        if (++st_v == kAtStages) st_v = 0;
       }
-      if (!ok) { const uint64_t t0 = global_timer_ns(); while (global_timer_ns() - t0 < 200000ull) { } }
+      ++n_item;
     }
+    if (!ok) { const uint64_t t0 = global_timer_ns(); while (global_timer_ns() - t0 < 200000ull) { } }
     __syncwarp();
   } else {
     // ------------------------------------------------ softmax + epilogue: thread = row

@@ -102,6 +102,27 @@ GS_DEVINL void head_tile(const HeadTcParams& P, int i, int& unit0, int& width) {
 
 constexpr int kMaxUnits = 9;                // widest tile, in units
 
+// MMAs of one W stage (KW k rows) for a tile WIDTH units wide: every offset is a compile-time
+// constant added to the per-stage base.
+template <int KW, int NT, int WIDTH>
+GS_DEVINL void head_issue_stage(uint32_t d_acc, uint32_t a_hi, uint32_t a_lo_stage, uint32_t b_hi, uint32_t b_lo_sub,
+                                uint32_t n_tile, uint32_t n_tile_u, uint32_t idesc, uint32_t fresh) {
+  constexpr uint32_t w_box_u = ((uint32_t)KW * 128u) >> 4;
+#pragma unroll
+  for (int kk = 0; kk < KW / 16; ++kk) {
+    const uint32_t accum = (kk == 0) ? (fresh ^ 1u) : 1u;
+#pragma unroll
+    for (int m = 0; m < WIDTH; ++m) {
+      const uint64_t adesc = ((uint64_t)a_hi << 32) | (a_lo_stage + (uint32_t)(m * 2) * w_box_u + (uint32_t)(kk * 128));
+#pragma unroll
+      for (int j = 0; j < NT; ++j) {
+        const uint64_t bdesc = ((uint64_t)b_hi << 32) | (b_lo_sub + (uint32_t)j * n_tile_u + (uint32_t)(kk * 2));
+        umma_bf16(d_acc + (uint32_t)(m * NT + j) * n_tile, adesc, bdesc, idesc, accum);
+      }
+    }
+  }
+}
+
 // KW = k rows of W per ring stage, NT = number of N tiles.  Both are compile-time so that the
 // MMA issue loop unrolls completely: every descriptor is then "a per-stage base plus a constant",
 // which keeps the single issuing thread ahead of the tensor core even when an MMA is short
@@ -186,71 +207,68 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmapW, const __grid_consta
     }
     __syncwarp();
   } else if (warp == 1) {
-    // ---------------- MMA issuer
-    if (lane == 0) {
-      const uint32_t idesc = idesc_bf16(kTileM, (uint32_t)P.n_tile, /*A (W^T) MN-major*/ true, /*B (H) K-major*/ false);
-      // Descriptors differ only in their low word (the start address >> 4).
-      //   A (W^T, MN-major): two 64-column boxes KW*128 bytes apart (leading offset), 8-k groups
-      //                      1024 bytes apart (stride offset); 16 k further = +2048 bytes.
-      //   B (H, K-major):    rows of 128 bytes, 8-row groups 1024 bytes apart; 16 k further = +32 bytes.
-      const uint64_t a_desc0 = smem_desc_sw128(base, w_box_bytes, 1024u);
-      const uint64_t b_desc0 = smem_desc_sw128(h_base, 16u, 1024u);
-      const uint32_t a_hi = (uint32_t)(a_desc0 >> 32), a_lo0 = (uint32_t)a_desc0;
-      const uint32_t b_hi = (uint32_t)(b_desc0 >> 32), b_lo0 = (uint32_t)b_desc0;
-      const uint32_t w_stage_u = P.w_stage_bytes >> 4, h_stage_u = P.h_stage_bytes >> 4;
-      const uint32_t n_tile_u = ((uint32_t)P.n_tile * 128u) >> 4;       // one N tile of H, in 16-byte units
-      const uint32_t n_tile = (uint32_t)P.n_tile;
-      uint32_t ws = 0, wph = 0, hs = 0, hph = 0;
-      int it = 0;
-      bool ok = true;
-      constexpr int k16_per_stage = KW / 16;
-      for (int tile = blockIdx.x; tile < P.num_tiles && ok; tile += gridDim.x, ++it) {
-        int unit0, width;
-        head_tile(P, tile, unit0, width);
-        const int acc = it % P.n_acc;
-        const uint32_t acc_ph = (uint32_t)(it / P.n_acc) & 1u;
-        if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag)) { ok = false; break; }
-        tc_fence_after();
-        const uint32_t d_acc = tmem_base + (uint32_t)acc * P.acc_cols;
-        for (int kb = 0; kb < P.k_blocks && ok; ++kb) {
-          if (!mbar_wait(hfull_bar(hs), hph, abort_flag)) { ok = false; break; }
-          const uint32_t b_lo_stage = b_lo0 + hs * h_stage_u;
+    // ---------------- MMA issuer: the whole warp walks the loops, one elected lane issues
+    const uint32_t idesc = idesc_bf16(kTileM, (uint32_t)P.n_tile, /*A (W^T) MN-major*/ true, /*B (H) K-major*/ false);
+    // Descriptors differ only in their low word (the start address >> 4).
+    //   A (W^T, MN-major): two 64-column boxes KW*128 bytes apart (leading offset), 8-k groups
+    //                      1024 bytes apart (stride offset); 16 k further = +2048 bytes.
+    //   B (H, K-major):    rows of 128 bytes, 8-row groups 1024 bytes apart; 16 k further = +32 bytes.
+    const uint64_t a_desc0 = smem_desc_sw128(base, w_box_bytes, 1024u);
+    const uint64_t b_desc0 = smem_desc_sw128(h_base, 16u, 1024u);
+    const uint32_t a_hi = (uint32_t)(a_desc0 >> 32), a_lo0 = (uint32_t)a_desc0;
+    const uint32_t b_hi = (uint32_t)(b_desc0 >> 32), b_lo0 = (uint32_t)b_desc0;
+    const uint32_t w_stage_u = P.w_stage_bytes >> 4, h_stage_u = P.h_stage_bytes >> 4;
+    const uint32_t n_tile_u = ((uint32_t)P.n_tile * 128u) >> 4;       // one N tile of H, in 16-byte units
+    const uint32_t n_tile = (uint32_t)P.n_tile;
+    uint32_t ws = 0, wph = 0, hs = 0, hph = 0;
+    int it = 0;
+    bool ok = true;
+    constexpr int k16_per_stage = KW / 16;
+    for (int tile = blockIdx.x; tile < P.num_tiles && ok; tile += gridDim.x, ++it) {
+      int unit0, width;
+      head_tile(P, tile, unit0, width);
+      const int acc = it % P.n_acc;
+      const uint32_t acc_ph = (uint32_t)(it / P.n_acc) & 1u;
+      if (!mbar_wait_warp(tempty_bar(acc), acc_ph ^ 1u, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t d_acc = tmem_base + (uint32_t)acc * P.acc_cols;
+      for (int kb = 0; kb < P.k_blocks && ok; ++kb) {
+        if (!mbar_wait_warp(hfull_bar(hs), hph, abort_flag)) { ok = false; break; }
+        const uint32_t b_lo_stage = b_lo0 + hs * h_stage_u;
 #pragma unroll
-          for (int sub = 0; sub < subs; ++sub) {
-            if (!mbar_wait(wfull_bar(ws), wph, abort_flag)) { ok = false; break; }
-            tc_fence_after();
+        for (int sub = 0; sub < subs; ++sub) {
+          if (!mbar_wait_warp(wfull_bar(ws), wph, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          if (elect_one()) {
             const uint32_t a_lo_stage = a_lo0 + ws * w_stage_u;
+            const uint32_t b_lo_sub = b_lo_stage + (uint32_t)(sub * k16_per_stage * 2);
             const uint32_t fresh = (kb == 0 && sub == 0) ? 1u : 0u;    // first MMAs of the tile overwrite
-#pragma unroll
-            for (int kk = 0; kk < k16_per_stage; ++kk) {
-              const uint32_t accum = (kk == 0) ? (fresh ^ 1u) : 1u;
-#pragma unroll
-              for (int m = 0; m < kMaxUnits; ++m) {
-                if (m < width) {
-                  const uint64_t adesc = ((uint64_t)a_hi << 32) |
-                                         (a_lo_stage + (uint32_t)(m * 2 * (int)(w_box_bytes >> 4) + kk * 128));
-#pragma unroll
-                  for (int j = 0; j < NT; ++j) {
-                    const uint64_t bdesc = ((uint64_t)b_hi << 32) |
-                                           (b_lo_stage + (uint32_t)j * n_tile_u + (uint32_t)((sub * k16_per_stage + kk) * 2));
-                    umma_bf16(d_acc + (uint32_t)(m * NT + j) * n_tile, adesc, bdesc, idesc, accum);
-                  }
-                }
-              }
+            switch (width) {
+              case 1: head_issue_stage<KW, NT, 1>(d_acc, a_hi, a_lo_stage, b_hi, b_lo_sub, n_tile, n_tile_u, idesc, fresh); break;
+              case 2: head_issue_stage<KW, NT, 2>(d_acc, a_hi, a_lo_stage, b_hi, b_lo_sub, n_tile, n_tile_u, idesc, fresh); break;
+              case 3: head_issue_stage<KW, NT, 3>(d_acc, a_hi, a_lo_stage, b_hi, b_lo_sub, n_tile, n_tile_u, idesc, fresh); break;
+              case 4: head_issue_stage<KW, NT, 4>(d_acc, a_hi, a_lo_stage, b_hi, b_lo_sub, n_tile, n_tile_u, idesc, fresh); break;
+              case 5: head_issue_stage<KW, NT, 5>(d_acc, a_hi, a_lo_stage, b_hi, b_lo_sub, n_tile, n_tile_u, idesc, fresh); break;
+              case 6: head_issue_stage<KW, NT, 6>(d_acc, a_hi, a_lo_stage, b_hi, b_lo_sub, n_tile, n_tile_u, idesc, fresh); break;
+              case 7: head_issue_stage<KW, NT, 7>(d_acc, a_hi, a_lo_stage, b_hi, b_lo_sub, n_tile, n_tile_u, idesc, fresh); break;
+              case 8: head_issue_stage<KW, NT, 8>(d_acc, a_hi, a_lo_stage, b_hi, b_lo_sub, n_tile, n_tile_u, idesc, fresh); break;
+              default: head_issue_stage<KW, NT, 9>(d_acc, a_hi, a_lo_stage, b_hi, b_lo_sub, n_tile, n_tile_u, idesc, fresh); break;
             }
             umma_commit(wempty_bar(ws));      // frees the W stage once these MMAs have read it
-            if (++ws == (uint32_t)WS) { ws = 0; wph ^= 1u; }
+            if (sub == subs - 1) umma_commit(hempty_bar(hs));
           }
-          if (ok) umma_commit(hempty_bar(hs));
-          if (++hs == (uint32_t)kHStages) { hs = 0; hph ^= 1u; }
+          __syncwarp();
+          if (++ws == (uint32_t)WS) { ws = 0; wph ^= 1u; }
         }
-        if (ok) umma_commit(tfull_bar(acc));
+        if (++hs == (uint32_t)kHStages) { hs = 0; hph ^= 1u; }
       }
-      if (!ok) {
-        // MMAs may still be running: give them (bounded) time before TMEM is freed.
-        const uint64_t t0 = global_timer_ns();
-        while (global_timer_ns() - t0 < 200000ull) { }
-      }
+      if (ok && elect_one()) umma_commit(tfull_bar(acc));
+      __syncwarp();
+    }
+    if (!ok) {
+      // MMAs may still be running: give them (bounded) time before TMEM is freed.
+      const uint64_t t0 = global_timer_ns();
+      while (global_timer_ns() - t0 < 200000ull) { }
     }
     __syncwarp();
   } else {
@@ -302,6 +320,7 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmapW, const __grid_consta
 static int g_head_mt = 0;       // 0 = choose automatically
 static int g_head_stages = 0;
 static int g_head_kw = 0;
+static int g_head_variant = 0;  // 0 = choose automatically, 1 = one CTA per tile, 2 = CTA pairs
 
 inline gs_status launch_lm_head_tc(const void* H, const void* W, float* logits, int T, int d, int V,
                                    int32_t* d_status, cudaStream_t st) {
@@ -380,6 +399,14 @@ inline gs_status launch_lm_head_tc(const void* H, const void* W, float* logits, 
 
 }  // namespace gs
 
+#include "lm_head_pair.cuh"
+
+extern "C" gs_status gs_lm_head_select(int variant) {
+  if (variant < 0 || variant > 2) return GS_ERR_INVALID_ARG;
+  gs::g_head_variant = variant;
+  return GS_OK;
+}
+
 extern "C" gs_status gs_lm_head_configure(int m_tiles, int stages, int k_rows) {
   if (m_tiles < 0 || m_tiles > 9 || stages < 0) return GS_ERR_INVALID_ARG;
   if (k_rows != 0 && k_rows != 16 && k_rows != 32 && k_rows != 64) return GS_ERR_INVALID_ARG;
@@ -409,5 +436,9 @@ extern "C" gs_status gs_lm_head_logits(const void* H, const void* W, float* logi
   const bool tma_ok = d > 0 && (d % 8 == 0) && (V % 8 == 0) && (reinterpret_cast<uintptr_t>(H) % 16 == 0) &&
                       (reinterpret_cast<uintptr_t>(W) % 16 == 0);
   if (!tma_ok) return GS_ERR_UNSUPPORTED;
+  // Above 256 rows a single CTA re-reads H from L2 once per 128 vocabulary columns and that
+  // traffic is the limit: CTA pairs halve it.
+  const bool pair = g_head_variant == 2 || (g_head_variant == 0 && T > 256);
+  if (pair) return launch_lm_head_pair(H, W, logits, T, d, V, d_status, g_head_mt, g_head_stages, st);
   return launch_lm_head_tc(H, W, logits, T, d, V, d_status, st);
 }
