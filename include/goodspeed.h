@@ -105,8 +105,8 @@ size_t gs_lm_head_workspace(int T, int d, int V, gs_dtype dt);
  * stages = upper bound on the depth of the shared-memory ring of W, k_rows = rows of W per ring
  * stage (16, 32 or 64).  Results do not depend on them.  Errors: INVALID_ARG. */
 gs_status gs_lm_head_configure(int m_tiles, int stages, int k_rows);
-/* Kernel choice of the bf16 path (process-wide, not thread-safe): 0 = automatic (CTA pairs above
- * 256 rows), 1 = one CTA per tile, 2 = CTA pairs: two SMs share one M = 256 MMA and each loads
+/* Kernel choice of the bf16 path (process-wide, not thread-safe): 0 = automatic (CTA pairs
+ * where the device can schedule them), 1 = one CTA per tile, 2 = CTA pairs: two SMs share one M = 256 MMA and each loads
  * half of the rows of H, which halves the L2 traffic of H (tile width at most 4 blocks of 256
  * columns; k_rows is ignored).  Results do not depend on the choice.  Errors: INVALID_ARG. */
 gs_status gs_lm_head_select(int variant);

@@ -194,28 +194,30 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
           set_status(P.d_status, GS_ERR_SHAPE);
       }
     }
-    // ------------------------------------------------ TMA producer
-    if (lane == 0) {
+    __syncwarp();
+    // ------------------------------------------------ TMA producer (whole warp in the loops, one elected lane issues)
+    {
       uint32_t st = 0, ph = 0;
-      int n_item = 0;
       bool ok = true;
       for (int id = blockIdx.x; id < P.max_items && ok; id += gridDim.x) {
         const AttnItem it = attn_find_item(P, id);
         if (!it.valid) break;
         if (it.n_tiles == 0) continue;
         for (int j = 0; j < it.n_tiles; ++j) {
-          if (!mbar_wait(bar(kKvEmpty + st), ph ^ 1u, abort_flag)) { ok = false; break; }
-          mbar_arrive_expect_tx(bar(kKvFull + st), kAtKvBytes);
-          const uint32_t dst = kv_base + st * kAtKvBytes;
-          const int key = it.kv0 + (it.tile0 + j) * kAtTile;
-          const int col = it.g * kAtHd;
-          tma_load_2d(dst, &tmapK, col, key, bar(kKvFull + st));
-          tma_load_2d(dst + kAtHalfBytes, &tmapK, col + 64, key, bar(kKvFull + st));
-          tma_load_2d(dst + 2 * kAtHalfBytes, &tmapV, col, key, bar(kKvFull + st));
-          tma_load_2d(dst + 3 * kAtHalfBytes, &tmapV, col + 64, key, bar(kKvFull + st));
+          if (!mbar_wait_warp(bar(kKvEmpty + st), ph ^ 1u, abort_flag)) { ok = false; break; }
+          if (elect_one()) {
+            mbar_arrive_expect_tx(bar(kKvFull + st), kAtKvBytes);
+            const uint32_t dst = kv_base + st * kAtKvBytes;
+            const int key = it.kv0 + (it.tile0 + j) * kAtTile;
+            const int col = it.g * kAtHd;
+            tma_load_2d(dst, &tmapK, col, key, bar(kKvFull + st));
+            tma_load_2d(dst + kAtHalfBytes, &tmapK, col + 64, key, bar(kKvFull + st));
+            tma_load_2d(dst + 2 * kAtHalfBytes, &tmapV, col, key, bar(kKvFull + st));
+            tma_load_2d(dst + 3 * kAtHalfBytes, &tmapV, col + 64, key, bar(kKvFull + st));
+          }
+          __syncwarp();
           if (++st == kAtStages) { st = 0; ph ^= 1u; }
         }
-        ++n_item;
       }
       if (!ok) { const uint64_t t0 = global_timer_ns(); while (global_timer_ns() - t0 < 200000ull) { } }
     }

@@ -172,38 +172,43 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmapW, const __grid_consta
   constexpr uint32_t w_box_bytes = (uint32_t)KW * 128u; // one box: KW k rows x 64 v
 
   if (warp == 0) {
-    // ---------------- TMA producer (loads are issued in the order the MMA warp consumes them)
-    if (lane == 0) {
-      uint32_t ws = 0, wph = 0, hs = 0, hph = 0;
-      bool ok = true;
-      for (int tile = blockIdx.x; tile < P.num_tiles && ok; tile += gridDim.x) {
-        int unit0, width;
-        head_tile(P, tile, unit0, width);
-        const int v0 = unit0 * (int)kTileM;
-        const int boxes = 2 * width;
-        for (int kb = 0; kb < P.k_blocks && ok; ++kb) {
-          const int k0 = kb * (int)kBlockK;
-          if (!mbar_wait(hempty_bar(hs), hph ^ 1u, abort_flag)) { ok = false; break; }
+    // ---------------- TMA producer (loads are issued in the order the MMA warp consumes them);
+    // the whole warp walks the loops, one elected lane issues
+    uint32_t ws = 0, wph = 0, hs = 0, hph = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < P.num_tiles && ok; tile += gridDim.x) {
+      int unit0, width;
+      head_tile(P, tile, unit0, width);
+      const int v0 = unit0 * (int)kTileM;
+      const int boxes = 2 * width;
+      for (int kb = 0; kb < P.k_blocks && ok; ++kb) {
+        const int k0 = kb * (int)kBlockK;
+        if (!mbar_wait_warp(hempty_bar(hs), hph ^ 1u, abort_flag)) { ok = false; break; }
+        if (elect_one()) {
           mbar_arrive_expect_tx(hfull_bar(hs), P.h_stage_bytes);
           for (int j = 0; j < NT; ++j)
             tma_load_2d(h_base + hs * P.h_stage_bytes + (uint32_t)(j * P.n_tile) * 128u, &tmapH, k0,
                         P.row0 + j * P.n_tile, hfull_bar(hs));
-          if (++hs == (uint32_t)kHStages) { hs = 0; hph ^= 1u; }
-          for (int sub = 0; sub < subs; ++sub) {
-            if (!mbar_wait(wempty_bar(ws), wph ^ 1u, abort_flag)) { ok = false; break; }
+        }
+        __syncwarp();
+        if (++hs == (uint32_t)kHStages) { hs = 0; hph ^= 1u; }
+        for (int sub = 0; sub < subs; ++sub) {
+          if (!mbar_wait_warp(wempty_bar(ws), wph ^ 1u, abort_flag)) { ok = false; break; }
+          if (elect_one()) {
             mbar_arrive_expect_tx(wfull_bar(ws), (uint32_t)boxes * w_box_bytes);
             const uint32_t dst = base + ws * P.w_stage_bytes;
             for (int b = 0; b < boxes; ++b)
               tma_load_2d(dst + (uint32_t)b * w_box_bytes, &tmapW, v0 + b * 64, k0 + sub * KW, wfull_bar(ws));
-            if (++ws == (uint32_t)WS) { ws = 0; wph ^= 1u; }
           }
+          __syncwarp();
+          if (++ws == (uint32_t)WS) { ws = 0; wph ^= 1u; }
         }
       }
-      if (!ok) {
-        // Let loads that are still in flight land before the CTA goes away (bounded).
-        const uint64_t t0 = global_timer_ns();
-        while (global_timer_ns() - t0 < 200000ull) { }
-      }
+    }
+    if (!ok) {
+      // Let loads that are still in flight land before the CTA goes away (bounded).
+      const uint64_t t0 = global_timer_ns();
+      while (global_timer_ns() - t0 < 200000ull) { }
     }
     __syncwarp();
   } else if (warp == 1) {
@@ -436,9 +441,12 @@ extern "C" gs_status gs_lm_head_logits(const void* H, const void* W, float* logi
   const bool tma_ok = d > 0 && (d % 8 == 0) && (V % 8 == 0) && (reinterpret_cast<uintptr_t>(H) % 16 == 0) &&
                       (reinterpret_cast<uintptr_t>(W) % 16 == 0);
   if (!tma_ok) return GS_ERR_UNSUPPORTED;
-  // Above 256 rows a single CTA re-reads H from L2 once per 128 vocabulary columns and that
-  // traffic is the limit: CTA pairs halve it.
-  const bool pair = g_head_variant == 2 || (g_head_variant == 0 && T > 256);
-  if (pair) return launch_lm_head_pair(H, W, logits, T, d, V, d_status, g_head_mt, g_head_stages, st);
+  // CTA pairs by default: a single CTA re-reads H from L2 once per 128 vocabulary columns, a pair
+  // half as often, and that traffic is what limits the kernel once there are many rows.  One CTA
+  // per tile remains for devices that cannot co-schedule pairs, and as a cross-check.
+  if (g_head_variant != 1) {
+    const gs_status r = launch_lm_head_pair(H, W, logits, T, d, V, d_status, g_head_mt, g_head_stages, st);
+    if (r != GS_ERR_UNSUPPORTED || g_head_variant == 2) return r;
+  }
   return launch_lm_head_tc(H, W, logits, T, d, V, d_status, st);
 }

@@ -107,17 +107,18 @@ lm_head_pair_kernel(const __grid_constant__ CUtensorMap tmapW, const __grid_cons
   const int half = P.n_tile / 2;                           // rows of H per MMA that this CTA holds
 
   if (warp == 0) {
-    // ---------------- TMA producer: this CTA's columns of W and rows of H
-    if (lane == 0) {
-      uint32_t st = 0, ph = 0;
-      bool ok = true;
-      for (int tile = cluster_id; tile < P.num_tiles && ok; tile += n_clusters) {
-        int unit0, width;
-        head_pair_tile(P, tile, unit0, width);
-        const uint32_t tx = 2u * ((uint32_t)width * kPairWUnitBytes + P.h_bytes);    // both CTAs' bytes
-        for (int kb = 0; kb < P.k_blocks; ++kb) {
-          const int k0 = kb * (int)kPairBlockK;
-          if (!mbar_wait(empty_bar(st), ph ^ 1u, abort_flag)) { ok = false; break; }
+    // ---------------- TMA producer: this CTA's columns of W and rows of H (whole warp in the loops,
+    // one elected lane issues)
+    uint32_t st = 0, ph = 0;
+    bool ok = true;
+    for (int tile = cluster_id; tile < P.num_tiles && ok; tile += n_clusters) {
+      int unit0, width;
+      head_pair_tile(P, tile, unit0, width);
+      const uint32_t tx = 2u * ((uint32_t)width * kPairWUnitBytes + P.h_bytes);    // both CTAs' bytes
+      for (int kb = 0; kb < P.k_blocks; ++kb) {
+        const int k0 = kb * (int)kPairBlockK;
+        if (!mbar_wait_warp(empty_bar(st), ph ^ 1u, abort_flag)) { ok = false; break; }
+        if (elect_one()) {
           const uint32_t full0 = map_to_cta(full_bar(st), 0);
           if (rank == 0) mbar_arrive_expect_tx(full_bar(st), tx);
           const uint32_t dst = base + st * P.stage_bytes;
@@ -129,14 +130,15 @@ lm_head_pair_kernel(const __grid_constant__ CUtensorMap tmapW, const __grid_cons
           for (int j = 0; j < NT; ++j)
             tma_load_2d_pair(dst + h_off + (uint32_t)(j * half) * 128u, &tmapH, k0,
                              P.row0 + j * P.n_tile + (int)rank * half, full0);
-          if (++st == (uint32_t)S) { st = 0; ph ^= 1u; }
         }
+        __syncwarp();
+        if (++st == (uint32_t)S) { st = 0; ph ^= 1u; }
       }
-      if (!ok) {
-        // Let loads that are still in flight land before the CTA goes away (bounded).
-        const uint64_t t0 = global_timer_ns();
-        while (global_timer_ns() - t0 < 200000ull) { }
-      }
+    }
+    if (!ok) {
+      // Let loads that are still in flight land before the CTA goes away (bounded).
+      const uint64_t t0 = global_timer_ns();
+      while (global_timer_ns() - t0 < 200000ull) { }
     }
     __syncwarp();
   } else if (warp == 1) {
@@ -273,7 +275,9 @@ inline HeadPairPlan head_pair_plan(int rows, int row0, int d, int V, int cluster
   P.nt = (rows + 255) / 256;
   P.n_tile = (((rows + P.nt - 1) / P.nt) + 15) / 16 * 16;
   const int total_n = P.nt * P.n_tile;
-  int max_mt = min(512 / total_n, kPairMaxUnits);
+  // Widest tile whose accumulators fit tensor memory twice (the epilogue of one tile then overlaps
+  // the MMAs of the next); a single buffer only when one unit needs more than half of it.
+  int max_mt = min(max(256 / total_n, 1), kPairMaxUnits);
   if (max_units > 0) max_mt = min(max_mt, max_units);
   if (max_mt < 1 || clusters_avail < 1) return pl;
   P.h_bytes = (uint32_t)(P.nt * (P.n_tile / 2)) * 128u;

@@ -304,15 +304,23 @@ def test_attention_bad_offsets_are_flagged():
 
 
 # ------------------------------------------------------------------ LM head
-@pytest.mark.parametrize("T,d,V", [(44, 512, 9000), (96, 1024, 4104), (288, 256, 8192), (1, 64, 8), (130, 136, 1000)])
-def test_lm_head_small(T, d, V):
+@pytest.mark.parametrize("variant", [2, 1], ids=["cta-pairs", "one-cta"])
+@pytest.mark.parametrize("T,d,V", [(44, 512, 9000), (96, 1024, 4104), (288, 256, 8192), (1, 64, 8), (130, 136, 1000),
+                                   (600, 192, 2056), (257, 320, 520)])
+def test_lm_head_small(T, d, V, variant):
+    """Both tensor-core kernels (CTA pairs with M = 256, and one CTA per tile) against the oracle:
+    ragged vocabulary and row tails, one and two MMAs along the rows, more than 512 rows."""
     cfg = wl.shrink(wl.CONFIGS["cfg2"], d=d, V=V, name=f"head_{T}_{d}_{V}")
     W = wl.make_layer(cfg)["W"]
     H = wl.make_hidden(cfg, T)
     logits = torch.full((T, V), float("nan"), dtype=torch.float32, device=DEV)
     ws = torch.empty(max(256, B.gs_lm_head_workspace(T, d, V, B.GS_BF16)), dtype=torch.uint8, device=DEV)
-    B.gs_lm_head_logits(H.to(DEV), W.to(DEV), logits, ws)
-    torch.cuda.synchronize()
+    B.gs_lm_head_select(variant)
+    try:
+        B.gs_lm_head_logits(H.to(DEV), W.to(DEV), logits, ws)
+        torch.cuda.synchronize()
+    finally:
+        B.gs_lm_head_select(0)
     ref = orc.ref_lm_head(H, W)
     pu.assert_close_rel(logits, ref, "logits")
     # bf16 products are exact in fp32 and only the accumulation rounds: far inside the 2e-2 bar
