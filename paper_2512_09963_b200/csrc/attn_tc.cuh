@@ -30,7 +30,8 @@ constexpr int kAtHd = 128;
 constexpr int kAtRows = 128;
 constexpr int kAtStages = 3;
 constexpr uint32_t kAtKvBytes = 2 * kAtTile * kAtHd * 2;       // K + V of one tile: 64 KB
-constexpr uint32_t kAtSmem = kAtStages * kAtKvBytes + 256;     // 192.25 KB: one CTA per SM
+constexpr int kAtMaxCached = 1023;       // servers whose offsets are cached in shared memory
+constexpr uint32_t kAtSmem = kAtStages * kAtKvBytes + 256 + 2 * (kAtMaxCached + 1) * 4;     // 200.25 KB: one CTA per SM
 // Tensor memory (512 columns): S two buffers 0..127 / 128..255 (P, as bf16 pairs, overwrites the first
 // 64 columns of its S buffer once the thread has read its scores), O 256..383, Q (bf16 pairs) 384..447.
 // Q and P are A operands read from tensor memory, so shared memory carries only K and V.
@@ -73,16 +74,16 @@ GS_DEVINL int attn_nsplit(int Lkv, int tiles_per_chunk) {
 }
 
 // Item `id` in the enumeration  server -> position block -> split -> KV head.
-GS_DEVINL AttnItem attn_find_item(const AttnTcParams& P, int id) {
+GS_DEVINL AttnItem attn_find_item(const AttnTcParams& P, const int32_t* cu_q, const int32_t* cu_kv, int id) {
   AttnItem it;
   it.valid = 0;
   int base = 0, gbase = 0;
   for (int i = 0; i < P.N; ++i) {
-    const int q0 = P.cu_q[i], n_new = P.cu_q[i + 1] - q0;
-    const int k0 = P.cu_kv[i], Lkv = P.cu_kv[i + 1] - k0;
+    const int q0 = cu_q[i], n_new = cu_q[i + 1] - q0;
+    const int k0 = cu_kv[i], Lkv = cu_kv[i + 1] - k0;
     if (n_new <= 0 || Lkv < n_new || Lkv > P.max_kv_len || k0 < 0 || k0 + Lkv > P.total_kv || q0 < 0 ||
         q0 + n_new > P.Tq)
-      continue;   // flagged by the checking kernel
+      continue;   // flagged by CTA 0
     const int tgs = (n_new + P.TB - 1) / P.TB;
     const int nsplit = attn_nsplit(Lkv, P.tiles_per_chunk);
     const int cnt = tgs * nsplit * P.Hkv;
@@ -153,6 +154,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 4);
   volatile int* s_last = reinterpret_cast<volatile int*>(tail + 8);
+  // The offsets are read by every role for every item: keep them in shared memory when they fit.
+  int32_t* s_cu = reinterpret_cast<int32_t*>(smem_raw + kAtStages * kAtKvBytes + 256);
+  const bool cached = P.N <= kAtMaxCached;
+  const int32_t* cu_q = cached ? s_cu : P.cu_q;
+  const int32_t* cu_kv = cached ? s_cu + (P.N + 1) : P.cu_kv;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if ((base & 1023u) != 0) {                     // the operand layouts need a 1024-byte aligned base
@@ -174,6 +180,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
   if (warp == 1) {
     tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kAtTmemCols);
     tmem_relinquish();
+  } else if (cached) {
+    const int t = (warp == 0) ? (int)threadIdx.x : (int)threadIdx.x - 32;      // 160 loading threads
+    for (int i = t; i <= P.N; i += kAtThreads - 32) { s_cu[i] = P.cu_q[i]; s_cu[P.N + 1 + i] = P.cu_kv[i]; }
   }
   tc_fence_before();
   __syncthreads();
@@ -200,7 +209,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
       uint32_t st = 0, ph = 0;
       bool ok = true;
       for (int id = blockIdx.x; id < P.max_items && ok; id += gridDim.x) {
-        const AttnItem it = attn_find_item(P, id);
+        const AttnItem it = attn_find_item(P, cu_q, cu_kv, id);
         if (!it.valid) break;
         if (it.n_tiles == 0) continue;
         for (int j = 0; j < it.n_tiles; ++j) {
@@ -248,7 +257,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
       __syncwarp();
     };
     for (int id = blockIdx.x; id < P.max_items && ok; id += gridDim.x) {
-      const AttnItem it = attn_find_item(P, id);
+      const AttnItem it = attn_find_item(P, cu_q, cu_kv, id);
       if (!it.valid) break;
       if (it.n_tiles == 0) continue;
       // Q of this item sits in tensor memory (written by the softmax warps after they have
@@ -297,7 +306,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
     int n_item = 0, n_tile_total = 0, n_ticket = 0;
     bool ok = true;
     for (int id = blockIdx.x; id < P.max_items && ok; id += gridDim.x) {
-      const AttnItem it = attn_find_item(P, id);
+      const AttnItem it = attn_find_item(P, cu_q, cu_kv, id);
       if (!it.valid) break;
       if (it.n_tiles == 0) continue;
       const int R = it.n_t * P.G;
@@ -514,7 +523,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
               }
             }
           };
-          if (it.n_used <= 4) {
+          if (it.n_used <= 2) {                    // 32 rows per round trip to L2
+            merge_rows(std::integral_constant<int, 2>{}, std::integral_constant<int, 8>{});
+          } else if (it.n_used <= 4) {
             merge_rows(std::integral_constant<int, 4>{}, std::integral_constant<int, 4>{});
           } else if (it.n_used <= 8) {
             merge_rows(std::integral_constant<int, 8>{}, std::integral_constant<int, 2>{});
