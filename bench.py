@@ -203,6 +203,7 @@ def run_ours(args, cfg, rank, world, local_rank):
     if world > 1:
         dist.barrier()
     B.lib()
+    B.gs_set_dependent_launch(not args.no_dependent_launch)
     dev = torch.device("cuda", local_rank)
     cfg_r = dataclasses.replace(cfg, seed_tag=f"/rank{rank}") if world > 1 else cfg
     inp, host = make_host_inputs(cfg_r, dev)
@@ -473,6 +474,8 @@ def main():
     ap.add_argument("--rounds", type=int, default=1000, help="rounds of the closed loop (--config cfg5)")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--no-dependent-launch", action="store_true",
+                    help="launch the kernels without the programmatic-dependent-launch attribute")
     ap.add_argument("--profile-small", action="store_true",
                     help="profiling case: vocabulary cut to 32768 (W = 336 MB, still larger than L2), eager "
                          "launches, no CPU baseline and no end-to-end leg; for ncu --set full captures")

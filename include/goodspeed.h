@@ -56,6 +56,14 @@ const char* gs_status_str(gs_status s);
 /* Library/ABI version (major*100 + minor). */
 int gs_version(void);
 
+/* Process-wide switch (not thread-safe; default on): whether the library's kernels are launched
+ * with the programmatic-dependent-launch attribute.  With it, a kernel's set-up (barrier and
+ * tensor-memory allocation, descriptor fetch, cluster rendezvous) overlaps the tail of the kernel
+ * before it on the stream; every kernel still waits for its predecessor to finish, with its
+ * writes visible, before it touches global memory, so results do not depend on the switch.
+ * The paper has no counterpart: this is launch plumbing. */
+gs_status gs_set_dependent_launch(int on);
+
 /* --------------------------------------------------------------------------------------------
  * gs_verify_attn -- Sec. II-A2: the target model scores all drafted positions of all servers
  * in one parallel pass.  The paper gives no attention formula; this is scaled-dot-product
@@ -146,6 +154,14 @@ gs_status gs_lm_head_logits(const void* H, const void* W, float* logits, int T, 
  * offsets, GS_ERR_INVALID_ARG for a draft token outside [0, V) (it is then rejected).
  */
 size_t gs_spec_accept_workspace(int N, int Tq, int V);
+/* Kernel choice of the second pass (process-wide, not thread-safe): 0 = automatic: one thread-block
+ * cluster per server, slices of the selected row held in shared memory and slice masses exchanged
+ * through distributed shared memory, where V % 4 == 0, the rows are 16-byte aligned and one row
+ * slice fits a CTA's shared memory; 1 = always the ticket kernel (chunk masses through the
+ * workspace, the last CTA of a server draws).  Accept decisions, ratios and estimators do not depend
+ * on the choice; the drawn token can differ only when u_sample * total lies within rounding of a
+ * CDF step.  Errors: INVALID_ARG. */
+gs_status gs_spec_accept_select(int variant);
 gs_status gs_spec_accept(const float* logits, const float* q_probs, const int32_t* draft_tok,
                          const int32_t* cu_q, const float* u_accept, const float* u_sample,
                          float temperature, int N, int Tq, int V,
@@ -199,6 +215,13 @@ gs_status gs_spec_accept_static(const float* logits, const float* q_probs, const
 gs_status gs_schedule(const double* X, const double* alpha_hat, int N, int C,
                       const int32_t* s_min, const int32_t* s_max, int32_t* S_out,
                       int32_t* d_status, void* stream);
+/* Kernel choice (process-wide, not thread-safe): 0 = automatic: for N <= 32 (and N*C*8 bytes of
+ * shared memory available) every server's gain list is written out once and each server finds by
+ * bisection how many of its entries rank among the `budget` largest of all lists in the order
+ * (gain descending, server ascending, step ascending), which is the set the greedy hands out;
+ * 1 = always the token-by-token greedy.  The allocation does not depend on the choice.
+ * Errors: INVALID_ARG. */
+gs_status gs_schedule_select(int variant);
 
 /* --------------------------------------------------------------------------------------------
  * gs_verify_round_host -- Algorithm 1, the verification-server steps of one round (batching,

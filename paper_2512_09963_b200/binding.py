@@ -32,6 +32,9 @@ SIGNATURES = {
     "gs_lm_head_workspace": (_sz, [_i, _i, _i, _i]),
     "gs_lm_head_configure": (_i, [_i, _i, _i]),
     "gs_lm_head_select": (_i, [_i]),
+    "gs_spec_accept_select": (_i, [_i]),
+    "gs_schedule_select": (_i, [_i]),
+    "gs_set_dependent_launch": (_i, [_i]),
     "gs_lm_head_logits": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _vp, _sz, _vp, _vp]),
     "gs_spec_accept_workspace": (_sz, [_i, _i, _i]),
     "gs_spec_accept": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _f, _i, _i, _i,
@@ -141,6 +144,18 @@ def gs_lm_head_configure(m_tiles: int = 0, stages: int = 0, k_rows: int = 0):
 
 def gs_lm_head_select(variant: int = 0):
     _check("gs_lm_head_select", lib().gs_lm_head_select(int(variant)))
+
+
+def gs_spec_accept_select(variant: int = 0):
+    _check("gs_spec_accept_select", lib().gs_spec_accept_select(int(variant)))
+
+
+def gs_schedule_select(variant: int = 0):
+    _check("gs_schedule_select", lib().gs_schedule_select(int(variant)))
+
+
+def gs_set_dependent_launch(on: bool = True):
+    _check("gs_set_dependent_launch", lib().gs_set_dependent_launch(1 if on else 0))
 
 
 def gs_lm_head_logits(H, W, logits, ws, d_status=None):

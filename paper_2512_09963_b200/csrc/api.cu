@@ -4,7 +4,14 @@
 namespace gs {
 static std::atomic<unsigned long long> g_launches{0};
 void count_launches(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+static std::atomic<int> g_dependent_launch{1};
+bool dependent_launch_enabled() { return g_dependent_launch.load(std::memory_order_relaxed) != 0; }
 }  // namespace gs
+
+extern "C" gs_status gs_set_dependent_launch(int on) {
+  gs::g_dependent_launch.store(on != 0 ? 1 : 0, std::memory_order_relaxed);
+  return GS_OK;
+}
 
 extern "C" unsigned long long gs_launch_count(void) { return gs::g_launches.load(std::memory_order_relaxed); }
 

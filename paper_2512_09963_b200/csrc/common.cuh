@@ -29,6 +29,39 @@ inline gs_status launch_status() {
   return cudaGetLastError() == cudaSuccess ? GS_OK : GS_ERR_CUDA;
 }
 
+// Programmatic dependent launch.  A kernel launched with the attribute may start while its
+// predecessor on the stream is still running; it must execute pdl_wait() before its first access
+// to global memory (the wait returns once the predecessor grid has finished and its writes are
+// visible).  pdl_launch_dependents() tells the scheduler that the successor may be started.
+// Both are no-ops in a kernel launched without the attribute.
+GS_DEVINL void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+GS_DEVINL void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Whether launches carry the programmatic-dependent-launch attribute (process-wide switch).
+bool dependent_launch_enabled();
+
+// Kernel launch with optional attributes: programmatic dependent launch and a cluster width.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_ex(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                             bool dependent, int cluster_x, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  unsigned n = 0;
+  if (dependent && dependent_launch_enabled()) {
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
+  if (cluster_x > 1) {
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = (unsigned)cluster_x; attr[n].val.clusterDim.y = 1; attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  cfg.attrs = attr; cfg.numAttrs = n;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 inline int sm_count() {
   static int cached = 0;
   if (cached == 0) {

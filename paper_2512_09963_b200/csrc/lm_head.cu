@@ -167,6 +167,8 @@ lm_head_tc_kernel(const __grid_constant__ CUtensorMap tmapW, const __grid_consta
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  pdl_wait();                    // the prologue above overlaps the previous kernel's tail
+  pdl_launch_dependents();       // after the wait: what the successor reads before its own wait is complete by now
   const uint32_t tmem_base = *tmem_slot;
   constexpr int subs = (int)kBlockK / KW;               // W stages per H stage
   constexpr uint32_t w_box_bytes = (uint32_t)KW * 128u; // one box: KW k rows x 64 v
@@ -395,8 +397,11 @@ inline gs_status launch_lm_head_tc(const void* H, const void* W, float* logits, 
     const size_t smem = 1024u + (size_t)stages * P.w_stage_bytes + (size_t)kHStages * P.h_stage_bytes +
                         8u * (2u * (uint32_t)stages + 2u * kHStages + 4u) + 64u;
     const int grid = min(P.num_tiles, sms);
-    kernels[kw == 16 ? 0 : (kw == 32 ? 1 : 2)][P.nt - 1]<<<grid, kTcThreads, smem, st>>>(tmapW, tmapH, P);
-    if (cudaGetLastError() != cudaSuccess) return GS_ERR_CUDA;
+    if (launch_ex(kernels[kw == 16 ? 0 : (kw == 32 ? 1 : 2)][P.nt - 1], dim3(grid), dim3(kTcThreads), smem, st, true, 1,
+                  tmapW, tmapH, P) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return GS_ERR_CUDA;
+    }
     count_launches(1);
   }
   return GS_OK;

@@ -102,6 +102,8 @@ lm_head_pair_kernel(const __grid_constant__ CUtensorMap tmapW, const __grid_cons
   __syncthreads();
   cluster_sync_all();            // the partner's barriers are initialised before anything signals them
   tc_fence_after();
+  pdl_wait();                    // the prologue above overlaps the previous kernel's tail
+  pdl_launch_dependents();       // after the wait: what the successor reads before its own wait is complete by now
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t h_off = P.stage_bytes - P.h_bytes;        // H share sits at the end of a stage
   const int half = P.n_tile / 2;                           // rows of H per MMA that this CTA holds
@@ -337,10 +339,12 @@ inline gs_status launch_lm_head_pair(const void* H, const void* W, float* logits
     cfg.blockDim = dim3(kPairThreads);
     cfg.dynamicSmemBytes = pl.smem;
     cfg.stream = st;
-    cudaLaunchAttribute at[1];
+    cudaLaunchAttribute at[2];
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-    cfg.attrs = at; cfg.numAttrs = 1;
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = dependent_launch_enabled() ? 2 : 1;
     if (cudaLaunchKernelEx(&cfg, kernels[pl.P.nt - 1], tmapW, tmapH, pl.P) != cudaSuccess) {
       (void)cudaGetLastError();
       return GS_ERR_CUDA;

@@ -1,13 +1,23 @@
 // gs_schedule: GoodSpeed-sched (Eq. goodspeed_sched, Sec. III-C) solved by marginal allocation.
 //
-// One CTA.  Thread i owns server i and keeps its current marginal gain
-// Delta_i = alpha_hat_i^(S_i+1) / X_i in a register (fp64, formed by repeated multiplication).
-// Each of the C budget steps is a block-wide arg-max over (gain, lowest index); the winner
-// multiplies its gain by alpha_hat_i and increments S_i.  For N <= 32 the arg-max is three
-// warp-wide integer reductions on the bit pattern of the (non-negative) gain.
+// The greedy gives the budget, one token at a time, to the largest marginal gain
+// Delta_i(s) = alpha_hat_i^(s+1) / X_i (fp64, formed by repeated multiplication), lowest index on
+// ties.  Because every server's gains are non-increasing, the tokens the greedy hands out are exactly
+// the `budget` first entries of all (server, step) pairs ordered by (gain descending, server
+// ascending, step ascending).  Two kernels produce that allocation:
+//   * schedule_rank_kernel (N <= 32): warp i owns server i.  One lane writes the server's gain list
+//     to shared memory (the same chain of fp64 multiplications as the greedy); then the warp finds,
+//     by bisection over its own list, how many of its entries rank among the first `budget`: the rank
+//     of an entry is its own step plus, per other server j (one lane each), the number of j's entries
+//     that precede it (a bisection in j's list).  About log^2 steps instead of `budget` rounds.
+//   * schedule_kernel: the greedy itself, one block-wide arg-max per token; any N <= 1024, and the
+//     path taken when an alpha_hat lies outside [0, 1] (gains no longer non-increasing).
 #include "common.cuh"
 
 namespace gs {
+
+// 0 = automatic (the rank kernel where it applies), 1 = always the greedy kernel.
+static int g_schedule_variant = 0;
 
 // Non-negative doubles order like their bit patterns.  Ineligible servers use key 0 with flag.
 GS_DEVINL unsigned long long gain_key(double g) {
@@ -24,6 +34,8 @@ schedule_kernel(const double* __restrict__ X, const double* __restrict__ alpha_h
   __shared__ int s_winner;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int nwarp = (blockDim.x + 31) >> 5;
+  pdl_wait();
+  pdl_launch_dependents();
   const bool live = tid < N;
   double a = 0.0, gain = 0.0;
   int S = 0, cap = 0;
@@ -85,7 +97,109 @@ schedule_kernel(const double* __restrict__ X, const double* __restrict__ alpha_h
   if (live) S_out[tid] = S;
 }
 
+
+// Gains are compared through their bit patterns: non-negative doubles order like unsigned integers.
+// cnt = number of entries of list[0..len) that precede key k: entries > k, or >= k when `ties_first`
+// (the list is non-increasing, so they form a prefix).
+GS_DEVINL int precede_count(const unsigned long long* list, int len, unsigned long long k, bool ties_first) {
+  int lo = 0, hi = len;                       // first index whose entry does NOT precede k
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    const unsigned long long e = list[mid];
+    const bool before = ties_first ? (e >= k) : (e > k);
+    if (before) lo = mid + 1; else hi = mid;
+  }
+  return lo;
+}
+
+__global__ void __launch_bounds__(1024)
+schedule_rank_kernel(const double* __restrict__ X, const double* __restrict__ alpha_hat, int N, int C,
+                     const int32_t* __restrict__ s_min, const int32_t* __restrict__ s_max,
+                     int32_t* __restrict__ S_out, int32_t* d_status) {
+  extern __shared__ __align__(8) unsigned char sched_smem[];
+  unsigned long long* table = reinterpret_cast<unsigned long long*>(sched_smem);      // [N][C]
+  __shared__ int s_S0[32], s_len[32], s_bad;
+  __shared__ double s_a[32], s_g0[32];
+  const int tid = threadIdx.x, lane = tid & 31, i = tid >> 5;       // warp i = server i
+  pdl_wait();
+  pdl_launch_dependents();
+  if (tid == 0) s_bad = 0;
+  __syncthreads();
+  if (tid < N) {
+    const double a = alpha_hat[tid];
+    int S = s_min ? s_min[tid] : 0;
+    int cap = s_max ? s_max[tid] : C;
+    if (S < 0) S = 0;
+    double gain = a / X[tid];
+    for (int k = 0; k < S; ++k) gain = __dmul_rn(gain, a);
+    if (!(gain >= 0.0)) gain = 0.0;           // negative or NaN inputs never win
+    if (!(a >= 0.0 && a <= 1.0)) s_bad = 1;   // the ordering argument needs non-increasing gains
+    s_a[tid] = a; s_g0[tid] = gain; s_S0[tid] = S;
+    s_len[tid] = max(0, min(cap - S, C));
+  }
+  __syncthreads();
+  int used = 0;
+  for (int j = 0; j < N; ++j) used += s_S0[j];
+  int budget = C - used;
+  if (budget < 0) {
+    if (tid == 0) set_status(d_status, GS_ERR_SHAPE);
+    budget = 0;
+  }
+  if (s_bad) {
+    // plain greedy by warp 0 (lane = server)
+    if (i == 0) {
+      const bool live = lane < N;
+      double a = live ? s_a[lane] : 0.0, gain = live ? s_g0[lane] : 0.0;
+      int S = live ? s_S0[lane] : 0;
+      const int cap = live ? S + s_len[lane] : 0;
+      for (int step = 0; step < budget; ++step) {
+        const bool elig = live && S < cap;
+        const unsigned long long key = elig ? (unsigned long long)__double_as_longlong(gain) + 1ull : 0ull;
+        const unsigned hi = (unsigned)(key >> 32), lo = (unsigned)key;
+        const unsigned mhi = __reduce_max_sync(0xffffffffu, hi);
+        const unsigned mlo = __reduce_max_sync(0xffffffffu, hi == mhi ? lo : 0u);
+        if ((((unsigned long long)mhi << 32) | mlo) == 0ull) break;
+        const int winner = __ffs(__ballot_sync(0xffffffffu, hi == mhi && lo == mlo)) - 1;
+        if (lane == winner) { S += 1; gain = __dmul_rn(gain, a); }
+      }
+      if (live) S_out[lane] = S;
+    }
+    return;
+  }
+  const int len_i = (i < N) ? min(s_len[i], budget) : 0;
+  if (i < N && lane == 0) {
+    const double a = s_a[i];
+    double g = s_g0[i];
+    unsigned long long* mine = table + (size_t)i * C;
+    for (int t = 0; t < len_i; ++t) {
+      mine[t] = (unsigned long long)__double_as_longlong(g);
+      g = __dmul_rn(g, a);
+    }
+  }
+  __syncthreads();
+  if (i >= N) return;
+  // Largest c in [0, len_i] with c == 0 or rank(i, c-1) < budget; ranks grow with the step.
+  const unsigned long long* mine = table + (size_t)i * C;
+  const int len_j = (lane < N && lane != i) ? min(s_len[lane], budget) : 0;
+  const unsigned long long* theirs = table + (size_t)min(lane, N - 1) * C;
+  int lo = 0, hi = len_i;                     // invariant: entries < lo are in, entries >= hi are out
+  while (lo < hi) {
+    const int t = (lo + hi) >> 1;
+    const unsigned long long k = mine[t];
+    const int cnt = len_j > 0 ? precede_count(theirs, len_j, k, lane < i) : 0;
+    const int rank = t + __reduce_add_sync(0xffffffffu, cnt);
+    if (rank < budget) lo = t + 1; else hi = t;
+  }
+  if (lane == 0) S_out[i] = s_S0[i] + lo;
+}
+
 }  // namespace gs
+
+extern "C" gs_status gs_schedule_select(int variant) {
+  if (variant < 0 || variant > 1) return GS_ERR_INVALID_ARG;
+  gs::g_schedule_variant = variant;
+  return GS_OK;
+}
 
 extern "C" gs_status gs_schedule(const double* X, const double* alpha_hat, int N, int C,
                                  const int32_t* s_min, const int32_t* s_max, int32_t* S_out,
@@ -94,9 +208,29 @@ extern "C" gs_status gs_schedule(const double* X, const double* alpha_hat, int N
   if (N == 0) return GS_OK;
   if (!X || !alpha_hat || !S_out) return GS_ERR_INVALID_ARG;
   if (N > 1024) return GS_ERR_UNSUPPORTED;
+  const size_t table = (size_t)N * (size_t)(C > 0 ? C : 1) * 8;
+  if (N <= 32 && table <= 160 * 1024 && gs::g_schedule_variant != 1) {
+    static bool attr_set = false;
+    if (!attr_set) {
+      if (cudaFuncSetAttribute(gs::schedule_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024) !=
+          cudaSuccess)
+        return GS_ERR_CUDA;
+      attr_set = true;
+    }
+    if (gs::launch_ex(gs::schedule_rank_kernel, dim3(1), dim3(32 * N), table, static_cast<cudaStream_t>(stream), true, 1,
+                      X, alpha_hat, N, C, s_min, s_max, S_out, d_status) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return GS_ERR_CUDA;
+    }
+    gs::count_launches(1);
+    return GS_OK;
+  }
   const int threads = (N + 31) / 32 * 32;
-  gs::schedule_kernel<<<1, threads, 0, static_cast<cudaStream_t>(stream)>>>(
-      X, alpha_hat, N, C, s_min, s_max, S_out, d_status);
+  if (gs::launch_ex(gs::schedule_kernel, dim3(1), dim3(threads), 0, static_cast<cudaStream_t>(stream), true, 1,
+                    X, alpha_hat, N, C, s_min, s_max, S_out, d_status) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return GS_ERR_CUDA;
+  }
   gs::count_launches(1);
-  return gs::launch_status();
+  return GS_OK;
 }

@@ -16,6 +16,7 @@
 // Only one row per server is read a second time.  All cross-thread sums are fp64 in a fixed
 // order, so two runs give identical bits.
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace gs {
 
@@ -96,6 +97,10 @@ sa_row_stats(const float* __restrict__ logits, int V, int n_chunk, float k2, Chu
   __shared__ double s_z[kSaThreads / 32];
   __shared__ float s_bm;
   const int tid = threadIdx.x, c = blockIdx.x, r = blockIdx.y;
+  // The successor is released only after this kernel's own wait: whatever it reads before ITS wait
+  // was then complete before this kernel touched memory.
+  pdl_wait();
+  pdl_launch_dependents();
   if (c == 0 && r == 0)
     for (int i = tid; i < N; i += kSaThreads) tickets[i] = 0;     // for the next kernel
   const float* row = logits + (size_t)r * V;
@@ -132,6 +137,9 @@ sa_row_stats(const float* __restrict__ logits, int V, int n_chunk, float k2, Chu
     stats[(size_t)r * n_chunk + c] = st;
   }
 }
+
+// 0 = automatic (a cluster per server where the shape allows it), 1 = the ticket kernel.
+static int g_sa_finish_variant = 0;
 
 struct SaFinishArgs {
   const float* logits; const float* q_probs; const int32_t* draft_tok; const int32_t* cu_q;
@@ -228,51 +236,55 @@ GS_DEVINL void scan_chunk(const float* __restrict__ lrow, const float* __restric
   __syncthreads();
 }
 
-template <bool VEC>
-__global__ void __launch_bounds__(kSaThreads) sa_finish(SaFinishArgs A) {
-  extern __shared__ unsigned char smem_raw[];
-  __shared__ int s_acc, s_is_last, s_chunk, s_tok, s_last;
-  __shared__ double s_before, s_thr, s_total, s_lo, s_hi;
-  __shared__ double s_warp[kSaThreads / 32];
-  const int c = blockIdx.x, i = blockIdx.y, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-  const bool writer = (c == 0);           // one CTA per server owns the outputs
-  const int r0 = A.cu_q[i], r1 = A.cu_q[i + 1];
-  const int gamma = r1 - r0 - 1;
-  if (r0 < 0 || gamma < 0 || r1 > A.Tq) {
-    if (writer && tid == 0) {
-      set_status(A.d_status, GS_ERR_SHAPE);
-      A.accepted[i] = 0; A.n_out[i] = 0;
-    }
-    return;
-  }
-  const int g0 = r0 - i;
-  // per-row merged statistics, rows j = 0..gamma
-  float* sM = reinterpret_cast<float*>(smem_raw);                // [gamma+1]
-  int* sArg = reinterpret_cast<int*>(sM + (gamma + 1));          // [gamma+1]
-  int* sRej = sArg + (gamma + 1);                                // [gamma+1] 1 = would be rejected
+// Pointers into the dynamic shared memory of a finish kernel: merged row statistics (rows
+// j = 0..gamma) and the scalars of the draft positions (j = 0..gamma-1).
+struct SaDecideSmem {
+  float* sM; int* sArg; int* sRej; double* sZ; double* sRatio; float* sL; float* sQ; float* sU; int* sTok;
+};
+inline size_t sa_decide_bytes(size_t rows) { return align_up(3 * rows * 4, 8) + 2 * rows * 8 + 4 * rows * 4; }
+GS_DEVINL SaDecideSmem sa_decide_carve(unsigned char* raw, int gamma) {
+  SaDecideSmem S;
+  S.sM = reinterpret_cast<float*>(raw);
+  S.sArg = reinterpret_cast<int*>(S.sM + (gamma + 1));
+  S.sRej = S.sArg + (gamma + 1);
   size_t off = (size_t)(3 * (gamma + 1)) * 4;
   off = (off + 7) / 8 * 8;
-  double* sZ = reinterpret_cast<double*>(smem_raw + off);        // [gamma+1]
-  double* sRatio = sZ + (gamma + 1);                             // [gamma+1] clipped ratios
+  S.sZ = reinterpret_cast<double*>(raw + off);
+  S.sRatio = S.sZ + (gamma + 1);
+  S.sL = reinterpret_cast<float*>(S.sRatio + (gamma + 1));
+  S.sQ = S.sL + (gamma + 1);
+  S.sU = S.sQ + (gamma + 1);
+  S.sTok = reinterpret_cast<int*>(S.sU + (gamma + 1));
+  return S;
+}
 
-  // ---- decide.  First every draft position's scalars are fetched in parallel (token -> logit and
-  // draft probability are dependent loads), then a warp per row merges that row's chunk statistics.
-  float* sL = reinterpret_cast<float*>(sRatio + (gamma + 1));    // [gamma] logit of the draft token
-  float* sQ = sL + (gamma + 1);                                  // [gamma] q of the draft token
-  float* sU = sQ + (gamma + 1);                                  // [gamma] uniform
-  int* sTok = reinterpret_cast<int*>(sU + (gamma + 1));          // [gamma] token, -1 if out of range
-  for (int j = tid; j < gamma; j += kSaThreads) {
+// First half of the "decide" step: the scalars of every draft position of server i (token, its
+// logit and draft probability -- dependent loads -- and the uniform) go to shared memory.  Reads
+// nothing the statistics pass writes.  The caller synchronises the CTA before sa_decide.
+GS_DEVINL void sa_fetch_scalars(const SaFinishArgs& A, int i, int r0, int gamma, bool writer, const SaDecideSmem& S) {
+  const int g0 = r0 - i;
+  for (int j = threadIdx.x; j < gamma; j += blockDim.x) {
     const int s = A.draft_tok[g0 + j];
     const bool in = (s >= 0 && s < A.V);
-    sTok[j] = in ? s : -1;
-    sL[j] = in ? A.logits[(size_t)(r0 + j) * A.V + s] : 0.f;
-    sQ[j] = in ? A.q_probs[(size_t)(g0 + j) * A.V + s] : 0.f;
-    sU[j] = A.u_accept[g0 + j];
+    S.sTok[j] = in ? s : -1;
+    S.sL[j] = in ? A.logits[(size_t)(r0 + j) * A.V + s] : 0.f;
+    S.sQ[j] = in ? A.q_probs[(size_t)(g0 + j) * A.V + s] : 0.f;
+    S.sU[j] = A.u_accept[g0 + j];
     if (!in && writer) set_status(A.d_status, GS_ERR_INVALID_ARG);
   }
-  __syncthreads();
+}
+
+// Second half, run by a whole CTA after a barrier: a warp per row merges that row's chunk
+// statistics (weights 2^((m_c - M) k2) from the special-function unit, sums in fp64), evaluates
+// p(s_j), the ratio and the accept test; one thread scans for the first rejection.  `writer` CTAs
+// also store ratio / p_tok / margin / accepted / n_out, and one of their threads does the estimator
+// update off the other threads' path.  Returns a_i (uniform over the CTA).
+GS_DEVINL int sa_decide(const SaFinishArgs& A, int i, int r0, int gamma, bool writer, const SaDecideSmem& S,
+                        int* s_acc) {
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nthr = blockDim.x, nwarp = nthr >> 5;
+  const int g0 = r0 - i;
   const double inv_tau = A.tau > 0.f ? 1.0 / (double)A.tau : 0.0;
-  for (int j = wid; j <= gamma; j += kSaThreads / 32) {
+  for (int j = wid; j <= gamma; j += nwarp) {
     const ChunkStat* st = A.stats + (size_t)(r0 + j) * A.n_chunk;
     float M = -INFINITY; int arg = INT_MAX;
     double z = 0.0;
@@ -286,34 +298,34 @@ __global__ void __launch_bounds__(kSaThreads) sa_finish(SaFinishArgs A) {
       argmax_merge(M, arg, c1s.m, c1s.arg);
       warp_argmax(M, arg);
       if (A.tau > 0.f) {
-        if (c0s.m > -INFINITY) z += c0s.z * exp(((double)c0s.m - (double)M) * inv_tau);
-        if (c1s.m > -INFINITY) z += c1s.z * exp(((double)c1s.m - (double)M) * inv_tau);
+        if (c0s.m > -INFINITY) z += c0s.z * (double)fast_exp2((c0s.m - M) * A.k2);
+        if (c1s.m > -INFINITY) z += c1s.z * (double)fast_exp2((c1s.m - M) * A.k2);
       }
     } else {
       for (int cc = lane; cc < A.n_chunk; cc += 32) argmax_merge(M, arg, st[cc].m, st[cc].arg);
       warp_argmax(M, arg);
       if (A.tau > 0.f)
         for (int cc = lane; cc < A.n_chunk; cc += 32)
-          if (st[cc].m > -INFINITY) z += st[cc].z * exp(((double)st[cc].m - (double)M) * inv_tau);
+          if (st[cc].m > -INFINITY) z += st[cc].z * (double)fast_exp2((st[cc].m - M) * A.k2);
     }
     const double Z = warp_sum_f64(z);
     if (lane == 0) {
-      sM[j] = M; sArg[j] = arg; sZ[j] = Z;
+      S.sM[j] = M; S.sArg[j] = arg; S.sZ[j] = Z;
       if (j < gamma) {
-        const int s = sTok[j];
+        const int s = S.sTok[j];
         double p = 0.0, q = 0.0, rho = 0.0;
         if (s >= 0) {
-          const float l = sL[j];
+          const float l = S.sL[j];
           if (A.tau > 0.f) p = (Z > 0.0) ? exp(((double)l - (double)M) * inv_tau) / Z : 0.0;
           else p = (s == arg) ? 1.0 : 0.0;
-          q = (double)sQ[j];
+          q = (double)S.sQ[j];
           if (q > 0.0) rho = p / q;
           else rho = (p > 0.0) ? (double)INFINITY : 0.0;
         }
-        const double u = (double)sU[j];
-        sRej[j] = (u > rho) ? 1 : 0;
+        const double u = (double)S.sU[j];
+        S.sRej[j] = (u > rho) ? 1 : 0;
         const double clipped = rho < 1.0 ? rho : 1.0;
-        sRatio[j] = clipped;
+        S.sRatio[j] = clipped;
         if (writer) {
           A.ratio[g0 + j] = (float)clipped;
           A.p_tok[g0 + j] = (float)p;
@@ -326,27 +338,60 @@ __global__ void __launch_bounds__(kSaThreads) sa_finish(SaFinishArgs A) {
   if (tid == 0) {
     int a = gamma;
     for (int j = 0; j < gamma; ++j) {
-      if (sRej[j]) { a = j; break; }
+      if (S.sRej[j]) { a = j; break; }
     }
-    s_acc = a;
-    if (writer) {
-      A.accepted[i] = a;
-      A.n_out[i] = a + 1;
-      if (A.alpha_hat != nullptr && A.X != nullptr) {
-        if (gamma > 0) {
-          double sum = 0.0;
-          for (int j = 0; j < gamma; ++j) sum += sRatio[j];
-          const double obs = sum / (double)gamma;
-          double ah = (1.0 - A.eta) * A.alpha_hat[i] + A.eta * obs;
-          ah = ah < A.alpha_min ? A.alpha_min : ah;
-          ah = ah > A.alpha_max ? A.alpha_max : ah;
-          A.alpha_hat[i] = ah;
-        }
-        A.X[i] = (1.0 - A.beta) * A.X[i] + A.beta * (double)(a + 1);
-      }
-    }
+    *s_acc = a;
   }
   __syncthreads();
+  const int a = *s_acc;
+  // Estimator update (Eq. updatealpha, Eq. updateX): one thread of another warp, so that its
+  // loads of the old state do not hold up the CTA.
+  if (writer && tid == (nthr > 32 ? 32 : 0)) {
+    A.accepted[i] = a;
+    A.n_out[i] = a + 1;
+    if (A.alpha_hat != nullptr && A.X != nullptr) {
+      const double x_old = A.X[i];
+      if (gamma > 0) {
+        const double ah_old = A.alpha_hat[i];
+        double sum = 0.0;
+        for (int j = 0; j < gamma; ++j) sum += S.sRatio[j];
+        const double obs = sum / (double)gamma;
+        double ah = (1.0 - A.eta) * ah_old + A.eta * obs;
+        ah = ah < A.alpha_min ? A.alpha_min : ah;
+        ah = ah > A.alpha_max ? A.alpha_max : ah;
+        A.alpha_hat[i] = ah;
+      }
+      A.X[i] = (1.0 - A.beta) * x_old + A.beta * (double)(a + 1);
+    }
+  }
+  return a;
+}
+
+template <bool VEC>
+__global__ void __launch_bounds__(kSaThreads) sa_finish(SaFinishArgs A) {
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ int s_acc, s_is_last, s_chunk, s_tok, s_last;
+  __shared__ double s_before, s_thr, s_total, s_lo, s_hi;
+  __shared__ double s_warp[kSaThreads / 32];
+  pdl_wait();
+  pdl_launch_dependents();
+  const int c = blockIdx.x, i = blockIdx.y, tid = threadIdx.x;
+  const bool writer = (c == 0);           // one CTA per server owns the outputs
+  const int r0 = A.cu_q[i], r1 = A.cu_q[i + 1];
+  const int gamma = r1 - r0 - 1;
+  if (r0 < 0 || gamma < 0 || r1 > A.Tq) {
+    if (writer && tid == 0) {
+      set_status(A.d_status, GS_ERR_SHAPE);
+      A.accepted[i] = 0; A.n_out[i] = 0;
+    }
+    return;
+  }
+  const int g0 = r0 - i;
+  const SaDecideSmem S = sa_decide_carve(smem_raw, gamma);
+  sa_fetch_scalars(A, i, r0, gamma, writer, S);
+  __syncthreads();
+  sa_decide(A, i, r0, gamma, writer, S, &s_acc);
+  float* const sM = S.sM; int* const sArg = S.sArg; double* const sZ = S.sZ;
   const int a = s_acc;
   const int row = r0 + a;                                  // the row the last token is drawn from
   const bool resid = a < gamma;                            // correction (max(0,p-q)) or bonus (p)
@@ -451,7 +496,242 @@ __global__ void __launch_bounds__(kSaThreads) sa_finish(SaFinishArgs A) {
   }
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// sa_finish_cluster: the finish step with one thread-block cluster per server.
+//
+// CTA k of the cluster owns the k-th slice of the vocabulary.  The draft tokens' scalars are fetched
+// while the statistics pass is still running (programmatic dependent launch); after the (redundant,
+// cheap) decide step every CTA brings its slice of the selected draft row into shared memory with
+// bulk copies, reads the matching logits from global memory, and overwrites the slice with the
+// masses max(p - q, 0) (or p for a bonus row).  The CTAs exchange their slice totals through
+// distributed shared memory around one cluster barrier; the CTA whose slice holds u * total then
+// finds the token in the masses it already has in shared memory: no ticket, no second trip to
+// global memory.  Thread t sums one contiguous run of the slice (an odd number of elements, so the
+// strided shared-memory reads do not collide).  One slice per CTA lets two clusters share an SM.
+constexpr int kFcThreads = 512;
+constexpr int kFcCluster = 8;
+constexpr int kFcWarps = kFcThreads / 32;
+constexpr uint32_t kFcPiece = 16384;               // bytes per bulk copy
+
+inline int fc_slice(int V) { return ((V + kFcCluster - 1) / kFcCluster + 3) / 4 * 4; }
+
+__global__ void __launch_bounds__(kFcThreads, 2) sa_finish_cluster(SaFinishArgs A, int slice) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  __shared__ __align__(8) uint64_t s_bar;
+  __shared__ int s_acc, s_abort, s_found, s_lastpos;
+  __shared__ double s_warp[kFcWarps];
+  __shared__ double s_cta_mass[2][kFcCluster];     // written by the peers (and by this CTA for itself)
+  cluster_arrive_release();                        // phase 0: "my shared memory exists"; waited for before the first remote store
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const int rank = (int)cluster_cta_rank(), i = blockIdx.y;
+  const uint32_t bar = smem_u32(&s_bar);
+  if (tid == 0) {
+    mbar_init(bar, 1);
+    s_abort = 0; s_found = INT_MAX; s_lastpos = -1;
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  // Before the wait: only data that was complete before the statistics pass started (that kernel
+  // releases this one after its own wait): offsets, draft tokens, their logits and draft
+  // probabilities, uniforms.  The statistics themselves are read after the wait.
+  const bool writer = (rank == 0);
+  const int r0 = A.cu_q[i], r1 = A.cu_q[i + 1];
+  const int gamma = r1 - r0 - 1;
+  bool live = !(r0 < 0 || gamma < 0 || r1 > A.Tq);           // uniform over the cluster
+  float* sx = reinterpret_cast<float*>(smem_raw);            // the slice: first the draft row, then the masses in place
+  const SaDecideSmem S = sa_decide_carve(smem_raw + (size_t)slice * 4, live ? gamma : 0);
+  if (live) sa_fetch_scalars(A, i, r0, gamma, writer, S);
+  const double u = (double)A.u_sample[i];
+  pdl_wait();
+  pdl_launch_dependents();
+  __syncthreads();
+  if (!live && writer && tid == 0) {
+    set_status(A.d_status, GS_ERR_SHAPE);
+    A.accepted[i] = 0; A.n_out[i] = 0;
+  }
+  int a = 0, row = 0, selArg = 0;
+  bool resid = false;
+  float selM = 0.f;
+  double invZ = 0.0;
+  if (live) {
+    const int g0 = r0 - i;
+    a = sa_decide(A, i, r0, gamma, writer, S, &s_acc);
+    row = r0 + a;                                            // the row the last token is drawn from
+    resid = a < gamma;                                       // correction (max(0,p-q)) or bonus (p)
+    selM = S.sM[a]; selArg = S.sArg[a];
+    invZ = (S.sZ[a] > 0.0) ? 1.0 / S.sZ[a] : 0.0;
+    if (writer)
+      for (int j = tid; j <= gamma; j += kFcThreads)
+        if (j != a) A.out_tok[r0 + j] = (j < a) ? A.draft_tok[g0 + j] : -1;
+    if (A.k2 <= 0.f) {   // greedy target: the one-hot (and its residual) sits on the argmax
+      if (writer && tid == 0) {
+        A.out_tok[row] = selArg;
+        if (A.margin != nullptr) A.margin[A.Gamma + i] = 1.0f;
+      }
+      live = false;
+    }
+  }
+  if (!live) {           // the whole cluster takes this path together; close the open barrier phase
+    cluster_wait_acquire();
+    return;
+  }
+  const int g0 = r0 - i;
+  const int start = rank * slice;
+  const int len = max(0, min(slice, A.V - start));           // a multiple of 4 (V is)
+  const float4* l4 = reinterpret_cast<const float4*>(A.logits + (size_t)row * A.V + start);
+  // ---- this CTA's slice of the draft row -> shared memory (bulk copies, one barrier)
+  if (resid && len > 0 && wid == 0) {
+    const char* qsrc = reinterpret_cast<const char*>(A.q_probs + (size_t)(g0 + a) * A.V + start);
+    const uint32_t bytes = (uint32_t)len * 4u;
+    if (lane == 0) mbar_arrive_expect_tx(bar, bytes);
+    __syncwarp();
+    for (uint32_t off = lane * kFcPiece; off < bytes; off += 32 * kFcPiece)
+      bulk_load_1d(smem_u32(sx) + off, qsrc + off, min(kFcPiece, bytes - off), bar);
+  }
+  // ---- masses in place: x = max(p - q, 0) after a rejection, p for the bonus row.  Logits come
+  // straight from global memory (the statistics pass has just read them), four 16-byte loads per
+  // thread in flight.  Element masses are fp32 (the exponential is an fp32 approximation in either
+  // kernel); every sum over them is fp64.
+  const float invZf = (float)invZ, negMk = -selM * A.k2;
+  bool q_here = !resid;
+  auto fill_masses = [&](bool res) {
+    const int n4 = len >> 2;
+    for (int f0 = tid; f0 < n4; f0 += 4 * kFcThreads) {
+      float4 l[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int f = f0 + k * kFcThreads;
+        l[k] = (f < n4) ? __ldg(l4 + f) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        l[k].x = fast_exp2(fmaf(l[k].x, A.k2, negMk)) * invZf;
+        l[k].y = fast_exp2(fmaf(l[k].y, A.k2, negMk)) * invZf;
+        l[k].z = fast_exp2(fmaf(l[k].z, A.k2, negMk)) * invZf;
+        l[k].w = fast_exp2(fmaf(l[k].w, A.k2, negMk)) * invZf;
+      }
+      if (!q_here) {       // first use of the draft row: its copies have landed
+        if (!mbar_wait(bar, 0u, &s_abort)) set_status(A.d_status, GS_ERR_TIMEOUT);
+        q_here = true;
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int f = f0 + k * kFcThreads;
+        if (f < n4) {
+          float4* dst = reinterpret_cast<float4*>(sx) + f;
+          if (res) {
+            const float4 q = *dst;
+            l[k].x = fmaxf(l[k].x - q.x, 0.f); l[k].y = fmaxf(l[k].y - q.y, 0.f);
+            l[k].z = fmaxf(l[k].z - q.z, 0.f); l[k].w = fmaxf(l[k].w - q.w, 0.f);
+          }
+          *dst = l[k];
+        }
+      }
+    }
+    if (!q_here) {         // threads without elements still have to see the copies complete
+      if (!mbar_wait(bar, 0u, &s_abort)) set_status(A.d_status, GS_ERR_TIMEOUT);
+      q_here = true;
+    }
+    __syncthreads();
+  };
+  if (len == 0) q_here = true;                               // nothing was requested for an empty slice
+  const int E = ((len + kFcThreads - 1) / kFcThreads) | 1;   // elements per thread, odd
+  const int e0 = min(len, tid * E), e1 = min(len, e0 + E);
+
+  int tok = -1;
+  float marg = 0.f;
+  for (int pass = 0; pass < 2; ++pass) {
+    fill_masses(resid);
+    // ---- mass of the thread's run, then the CTA-wide prefix in thread order
+    double tot = 0.0;
+    int last_pos = -1;
+    for (int e = e0; e < e1; ++e) {
+      const float x = sx[e];
+      if (x > 0.f) last_pos = e;
+      tot += (double)x;
+    }
+    double incl = tot;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const double t = shfl_up_f64(incl, d);
+      if (lane >= d) incl += t;
+    }
+    const double prev = shfl_up_f64(incl, 1);
+    if (lane == 31) s_warp[wid] = incl;
+    __syncthreads();
+    double woff = 0.0;
+    for (int k = 0; k < wid; ++k) woff += s_warp[k];
+    const double excl = (lane == 0) ? woff : woff + prev;     // CTA prefix before this thread
+    const double G = woff + incl;                             // and including it
+    if (pass == 0) cluster_wait_acquire();                    // every peer's shared memory is there
+    if (tid == kFcThreads - 1) {
+#pragma unroll
+      for (int k = 0; k < kFcCluster; ++k)
+        st_cluster_f64(map_to_cta(smem_u32(&s_cta_mass[pass][rank]), (uint32_t)k), G);
+    }
+    cluster_arrive_release();
+    cluster_wait_acquire();
+    double total = 0.0;
+#pragma unroll
+    for (int k = 0; k < kFcCluster; ++k) total += s_cta_mass[pass][k];
+    if (!(total > 0.0)) {
+      if (resid) { resid = false; continue; }       // max(0, p - q) has no mass: draw from p itself
+      if (writer && tid == 0) { tok = selArg; }     // no mass at all (cannot happen for finite logits)
+      break;
+    }
+    const double thr = u * total;
+    int owner = -1, last_rank = -1;
+    double before = 0.0, run = 0.0;
+#pragma unroll
+    for (int k = 0; k < kFcCluster; ++k) {
+      const double mk = s_cta_mass[pass][k];
+      if (mk > 0.0) last_rank = k;
+      if (owner < 0 && run + mk > thr) { owner = k; before = run; }
+      run += mk;
+    }
+    if (owner >= 0) {
+      if (rank == owner) {
+        // first thread whose inclusive prefix exceeds the threshold, then first such element
+        if (before + G > thr) atomicMin(&s_found, tid);
+        __syncthreads();
+        if (tid == s_found) {
+          double r2 = 0.0, lo = before + excl, hi = lo;
+          int pick = -1, pos = -1;
+          for (int e = e0; e < e1; ++e) {
+            const double x = (double)sx[e];
+            if (x > 0.0) {
+              pos = e;
+              const double c = before + (excl + (r2 + x));
+              if (c > thr) { pick = e; lo = before + (excl + r2); hi = c; break; }
+              r2 += x;
+            }
+          }
+          if (pick < 0) pick = pos;                 // rounding between the two prefix forms: last element with mass
+          else { const double x = thr - lo, y = hi - thr; marg = (float)((x < y ? x : y) / total); }
+          tok = (pick >= 0) ? start + pick : selArg;
+        }
+      }
+    } else if (rank == last_rank) {                 // rounding left no slice: the last token that has mass
+      if (last_pos >= 0) atomicMax(&s_lastpos, last_pos);
+      __syncthreads();
+      if (tid == 0) tok = (s_lastpos >= 0) ? start + s_lastpos : selArg;
+    }
+    break;
+  }
+  if (tok >= 0) {
+    A.out_tok[row] = tok;
+    if (A.margin != nullptr) A.margin[A.Gamma + i] = marg;
+  }
+}
+
 }  // namespace gs
+
+extern "C" gs_status gs_spec_accept_select(int variant) {
+  if (variant < 0 || variant > 1) return GS_ERR_INVALID_ARG;
+  gs::g_sa_finish_variant = variant;
+  return GS_OK;
+}
 
 extern "C" size_t gs_spec_accept_workspace(int N, int Tq, int V) {
   if (N <= 0 || Tq <= 0 || V <= 0) return 256;
@@ -486,8 +766,9 @@ extern "C" gs_status gs_spec_accept(const float* logits, const float* q_probs, c
                    (q_probs == nullptr || reinterpret_cast<uintptr_t>(q_probs) % 16 == 0);
 
   dim3 g1(n_chunk, Tq);
-  if (vec) sa_row_stats<true><<<g1, kSaThreads, 0, st>>>(logits, V, n_chunk, k2, w.stats, w.tickets, N);
-  else sa_row_stats<false><<<g1, kSaThreads, 0, st>>>(logits, V, n_chunk, k2, w.stats, w.tickets, N);
+  if (launch_ex(vec ? sa_row_stats<true> : sa_row_stats<false>, g1, dim3(kSaThreads), 0, st, true, 1,
+                logits, V, n_chunk, k2, w.stats, w.tickets, N) != cudaSuccess)
+    return GS_ERR_CUDA;
 
   SaFinishArgs A;
   A.logits = logits; A.q_probs = q_probs; A.draft_tok = draft_tok; A.cu_q = cu_q; A.u_accept = u_accept;
@@ -499,7 +780,26 @@ extern "C" gs_status gs_spec_accept(const float* logits, const float* q_probs, c
   A.stats = w.stats; A.tickets = w.tickets; A.mass = w.mass; A.d_status = d_status;
   // rows of one server are bounded by Tq - (N-1); size the dynamic shared memory for that
   const size_t max_rows = (size_t)(Tq - N + 1);
-  const size_t smem = align_up(3 * max_rows * 4, 8) + 2 * max_rows * 8 + 4 * max_rows * 4;
+  const size_t smem = sa_decide_bytes(max_rows);
+  // One cluster per server when the two row slices fit a CTA's shared memory next to the decide arrays.
+  const int slice = fc_slice(V);
+  const size_t smem_fc = (size_t)slice * 4 + smem;
+  if (vec && g_sa_finish_variant != 1 && smem_fc <= 200 * 1024) {
+    static bool attr_set = false;
+    if (!attr_set) {
+      if (cudaFuncSetAttribute(sa_finish_cluster, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
+        return GS_ERR_CUDA;
+      attr_set = true;
+    }
+    A.smem_bytes = (int)smem_fc;
+    if (launch_ex(sa_finish_cluster, dim3(kFcCluster, N), dim3(kFcThreads), smem_fc, st, true, kFcCluster, A, slice) !=
+        cudaSuccess) {
+      (void)cudaGetLastError();
+      return GS_ERR_CUDA;
+    }
+    count_launches(2);
+    return launch_status();
+  }
   if (smem > 160 * 1024) return GS_ERR_UNSUPPORTED;
   A.smem_bytes = (int)smem;
   if (smem > 40 * 1024) {
@@ -508,8 +808,8 @@ extern "C" gs_status gs_spec_accept(const float* logits, const float* q_probs, c
       return GS_ERR_CUDA;
   }
   dim3 g2(k2 > 0.f ? n_chunk : 1, N);
-  if (vec) sa_finish<true><<<g2, kSaThreads, smem, st>>>(A);
-  else sa_finish<false><<<g2, kSaThreads, smem, st>>>(A);
+  if (launch_ex(vec ? sa_finish<true> : sa_finish<false>, g2, dim3(kSaThreads), smem, st, true, 1, A) != cudaSuccess)
+    return GS_ERR_CUDA;
   count_launches(2);
   return launch_status();
 }

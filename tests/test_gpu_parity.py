@@ -103,8 +103,18 @@ ACCEPT_CASES = [
 ]
 
 
-@pytest.mark.parametrize("name,base,V,tau", ACCEPT_CASES)
-def test_spec_accept_small(name, base, V, tau):
+@pytest.fixture(params=[0, 1], ids=["cluster-finish", "ticket-finish"])
+def finish_variant(request):
+    """Both second-pass kernels of gs_spec_accept: a cluster per server (where the shape allows
+    it) and the ticket kernel."""
+    B.gs_spec_accept_select(request.param)
+    yield request.param
+    B.gs_spec_accept_select(0)
+
+
+@pytest.mark.parametrize("name,base,V,tau", ACCEPT_CASES + [("two-slices", "cfg2", 8, 1.0),
+                                                            ("ragged-slices", "cfg3", 30004, 0.7)])
+def test_spec_accept_small(name, base, V, tau, finish_variant):
     cfg = wl.shrink(wl.CONFIGS[base], V=V, d=64, prefix_scale=0.01, name=f"{base}_acc_{V}")
     inp = wl.make_step(cfg, tau=tau, synthetic_logits=True, allocator=orc.ref_schedule_greedy)
     rnd = run_accept_only(inp)
@@ -119,7 +129,22 @@ def test_spec_accept_small(name, base, V, tau):
         assert np.array_equal(v, first[k]), k
 
 
-def test_spec_accept_zero_length_drafts_and_single_server():
+def test_spec_accept_without_dependent_launch():
+    """The programmatic-dependent-launch attribute is launch plumbing: results are identical without it."""
+    cfg = wl.shrink(wl.CONFIGS["cfg2"], V=20000, d=64, prefix_scale=0.01, name="cfg2_acc_20000")
+    inp = wl.make_step(cfg, tau=0.7, synthetic_logits=True)
+    with_pdl = pu.gpu_accept_dict(run_accept_only(inp))
+    B.gs_set_dependent_launch(False)
+    try:
+        rnd = run_accept_only(inp)
+        check_accept(inp, rnd)
+        for k, v in pu.gpu_accept_dict(rnd).items():
+            assert np.array_equal(v, with_pdl[k]), k
+    finally:
+        B.gs_set_dependent_launch(True)
+
+
+def test_spec_accept_zero_length_drafts_and_single_server(finish_variant):
     cfg = wl.shrink(wl.CONFIGS["cfg2"], V=10000, d=64, prefix_scale=0.01, name="acc_gamma0")
     inp = wl.make_step(cfg, gamma=[0, 3, 0, 0, 5, 1, 0, 2], synthetic_logits=True)
     rnd = run_accept_only(inp)
@@ -176,17 +201,36 @@ def test_spec_accept_estimators_and_device_status():
 
 
 # ------------------------------------------------------------------ scheduler
-@pytest.mark.parametrize("N,C", [(1, 5), (4, 10), (16, 128), (32, 256), (33, 64), (100, 300), (1024, 512), (8, 0)])
-def test_schedule_bit_exact(N, C):
+@pytest.fixture(params=[0, 1], ids=["rank-kernel", "greedy-kernel"])
+def schedule_variant(request):
+    """Both scheduler kernels: ranks by bisection (N <= 32) and the token-by-token greedy."""
+    B.gs_schedule_select(request.param)
+    yield request.param
+    B.gs_schedule_select(0)
+
+
+@pytest.mark.parametrize("N,C", [(1, 5), (4, 10), (8, 64), (16, 128), (32, 256), (32, 600), (33, 64), (100, 300),
+                                 (1024, 512), (8, 0)])
+def test_schedule_bit_exact(N, C, schedule_variant):
     r = np.random.default_rng(N * 1000 + C)
-    for trial in range(4):
+    for trial in range(8):
         X = r.uniform(0.5, 8.0, N)
         al = r.uniform(0.001, 0.999, N)
         if trial == 1:                      # many exact ties
             X[:] = 2.0
             al[:] = 0.75
+        if trial == 4:                      # gains that underflow to zero, and zero / unit rates
+            al = r.choice([0.0, 1e-3, 0.5, 1.0], N)
+            X = r.choice([1.0, 1e-300, 3.0], N)
+        if trial == 5:                      # ties between servers at every step, in groups
+            al = r.choice([0.5, 0.25], N)
+            X = r.choice([1.0, 2.0, 4.0], N)
+        if trial == 6:                      # a rate outside [0, 1]: gains grow, the greedy is still defined
+            al[r.integers(0, N)] = 1.25
+        if trial == 7:                      # a starved server: its huge gain is served first
+            X[r.integers(0, N)] = 1e-12
         lo = hi = None
-        if trial >= 2:
+        if trial in (2, 3, 5):
             lo = r.integers(0, 2, N).astype(np.int32)
             hi = (lo + r.integers(0, 20, N)).astype(np.int32)
             if lo.sum() > C:
