@@ -89,6 +89,12 @@ gs_status gs_set_dependent_launch(int on);
  */
 size_t gs_verify_attn_workspace(int N, int Tq, int total_kv, int max_kv_len, int Hq, int Hkv, int hd,
                                 gs_dtype dt);
+/* Tuning knob of the tensor-core kernel (process-wide, not thread-safe): the number of 128-key tiles
+ * one split of a server's KV range covers at most; 0 = automatic (enough splits to give every SM
+ * work, but no split shorter than 12 tiles and at most 8 per server).  A large value means no
+ * splitting.  Results agree to rounding.  The workspace size depends
+ * on it: set it before gs_verify_attn_workspace.  Errors: INVALID_ARG. */
+gs_status gs_verify_attn_configure(int tiles_per_split);
 gs_status gs_verify_attn(const void* Q, const void* K, const void* V, void* O,
                          const int32_t* cu_q, const int32_t* cu_kv,
                          int N, int Tq, int total_kv, int max_kv_len, int Hq, int Hkv, int hd,

@@ -33,6 +33,7 @@ SIGNATURES = {
     "gs_lm_head_configure": (_i, [_i, _i, _i]),
     "gs_lm_head_select": (_i, [_i]),
     "gs_spec_accept_select": (_i, [_i]),
+    "gs_verify_attn_configure": (_i, [_i]),
     "gs_schedule_select": (_i, [_i]),
     "gs_set_dependent_launch": (_i, [_i]),
     "gs_lm_head_logits": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _vp, _sz, _vp, _vp]),
@@ -120,6 +121,10 @@ def gs_status_str(code: int) -> str:
 
 def gs_verify_attn_workspace(N, Tq, total_kv, max_kv_len, Hq, Hkv, hd, dt) -> int:
     return lib().gs_verify_attn_workspace(N, Tq, total_kv, max_kv_len, Hq, Hkv, hd, dt)
+
+
+def gs_verify_attn_configure(tiles_per_split: int = 0):
+    _check("gs_verify_attn_configure", lib().gs_verify_attn_configure(int(tiles_per_split)))
 
 
 def gs_verify_attn(Q, K, V, O, cu_q, cu_kv, max_kv_len, scale, ws, d_status=None):

@@ -24,14 +24,17 @@
 
 namespace gs {
 
-constexpr int kAtThreads = 192;          // warp 0 TMA, warp 1 MMA, warps 2-5 softmax/epilogue
+constexpr int kAtThreads = 320;          // warp 0 TMA, warp 1 MMA, warps 2-5 softmax, warps 6-9 epilogue
 constexpr int kAtTile = 128;             // keys per tile
 constexpr int kAtHd = 128;
 constexpr int kAtRows = 128;
 constexpr int kAtStages = 3;
 constexpr uint32_t kAtKvBytes = 2 * kAtTile * kAtHd * 2;       // K + V of one tile: 64 KB
+constexpr int kAtMinSplitTiles = 12;     // smallest split the automatic plan makes (tiles of 128 keys)
 constexpr int kAtMaxCached = 1023;       // servers whose offsets are cached in shared memory
-constexpr uint32_t kAtSmem = kAtStages * kAtKvBytes + 256 + 2 * (kAtMaxCached + 1) * 4;     // 200.25 KB: one CTA per SM
+constexpr int kAtItemCache = 32;         // items of a CTA whose descriptors are worked out once, in parallel
+constexpr uint32_t kAtItemCacheBytes = 2304; // >= kAtItemCache * sizeof(AttnItem)
+constexpr uint32_t kAtSmem = kAtStages * kAtKvBytes + 256 + 1024 + 4 * (kAtMaxCached + 1) * 4 + kAtItemCacheBytes;     // 211.5 KB: one CTA per SM
 // Tensor memory (512 columns): S two buffers 0..127 / 128..255 (P, as bf16 pairs, overwrites the first
 // 64 columns of its S buffer once the thread has read its scores), O 256..383, Q (bf16 pairs) 384..447.
 // Q and P are A operands read from tensor memory, so shared memory carries only K and V.
@@ -51,6 +54,7 @@ struct AttnTcParams {
   int32_t* d_status;
   int N, Tq, total_kv, max_kv_len, Hq, Hkv, G, TB;   // TB = 128 / G query positions per item
   int tiles_per_chunk;      // KV tiles per split (upper bound; splits of a server are balanced)
+  int min_split_tiles;      // a server is split only into parts of at least this many tiles
   int max_items;
   float scale_log2;         // scale * log2(e)
 };
@@ -66,56 +70,90 @@ struct AttnItem {
   int valid;
 };
 
-// Splits of a server: its ceil(Lkv/64) tiles are spread over nsplit = ceil(tiles/tiles_per_chunk)
-// splits whose sizes differ by at most one tile.
-GS_DEVINL int attn_nsplit(int Lkv, int tiles_per_chunk) {
+// Splits of a server: its ceil(Lkv/128) tiles are spread over nsplit = ceil(tiles/tiles_per_chunk)
+// splits whose sizes differ by at most one tile -- but never so many that a split falls below
+// min_split_tiles: a split costs a partial result, a ticket and a merge (several microseconds of
+// dependent round trips), which a handful of tiles at about 1.3 us each does not buy back.
+GS_DEVINL int attn_nsplit(int Lkv, int tiles_per_chunk, int min_split_tiles) {
   const int tiles = (Lkv + kAtTile - 1) / kAtTile;
-  return max(1, (tiles + tiles_per_chunk - 1) / tiles_per_chunk);
+  return max(1, min((tiles + tiles_per_chunk - 1) / tiles_per_chunk, tiles / min_split_tiles));
 }
 
-// Item `id` in the enumeration  server -> position block -> split -> KV head.
-GS_DEVINL AttnItem attn_find_item(const AttnTcParams& P, const int32_t* cu_q, const int32_t* cu_kv, int id) {
+// Items of one server (0 when its offsets are inconsistent: such servers are skipped everywhere
+// and flagged by CTA 0) and its (position block, KV head) groups.
+GS_DEVINL bool attn_server_ok(const AttnTcParams& P, int q0, int n_new, int k0, int Lkv) {
+  return !(n_new <= 0 || Lkv < n_new || Lkv > P.max_kv_len || k0 < 0 || k0 + Lkv > P.total_kv || q0 < 0 ||
+           q0 + n_new > P.Tq);
+}
+GS_DEVINL void attn_server_counts(const AttnTcParams& P, int q0, int n_new, int k0, int Lkv, int& items, int& groups) {
+  items = 0; groups = 0;
+  if (!attn_server_ok(P, q0, n_new, k0, Lkv)) return;
+  const int tgs = (n_new + P.TB - 1) / P.TB;
+  groups = tgs * P.Hkv;
+  items = groups * attn_nsplit(Lkv, P.tiles_per_chunk, P.min_split_tiles);
+}
+
+// Item `id` of server i, whose first item is `base` and first group `gbase`, in the enumeration
+// position block -> split -> KV head.
+GS_DEVINL AttnItem attn_item_of_server(const AttnTcParams& P, int i, int q0, int n_new, int k0, int Lkv, int base,
+                                       int gbase, int id) {
+  AttnItem it;
+  const int nsplit = attn_nsplit(Lkv, P.tiles_per_chunk, P.min_split_tiles);
+  int rem = id - base;
+  it.g = rem % P.Hkv; rem /= P.Hkv;
+  it.split = rem % nsplit; it.tg = rem / nsplit;
+  it.server = i;
+  it.item_base = base; it.nsplit = nsplit;
+  it.group = gbase + it.tg * P.Hkv + it.g;
+  it.q_row0 = q0 + it.tg * P.TB;
+  it.n_t = min(P.TB, n_new - it.tg * P.TB);
+  it.kv0 = k0; it.Lkv = Lkv; it.L = Lkv - n_new;
+  const int tiles = (Lkv + kAtTile - 1) / kAtTile;
+  const int tb = tiles / nsplit, tr = tiles % nsplit;
+  it.tile0 = it.split * tb + min(it.split, tr);
+  it.n_tiles = tb + (it.split < tr ? 1 : 0);
+  // keys the block can see end at L + (last position) ; later tiles hold nothing visible
+  const int last_key = it.L + it.tg * P.TB + it.n_t - 1;
+  const int last_tile = last_key / kAtTile;
+  if (it.tile0 + it.n_tiles - 1 > last_tile) it.n_tiles = max(0, last_tile - it.tile0 + 1);
+  it.n_used = 0;
+  for (int sp = 0; sp < nsplit; ++sp)
+    if (sp * tb + min(sp, tr) <= last_tile) it.n_used = sp + 1;
+  it.valid = 1;
+  return it;
+}
+
+// Item `id` in the enumeration  server -> position block -> split -> KV head.  With the per-server
+// prefix counts in shared memory (s_base[0..N], s_gbase[0..N-1]) the server is found by bisection;
+// without them (more servers than the cache holds) by a walk over the offsets.
+GS_DEVINL AttnItem attn_find_item(const AttnTcParams& P, const int32_t* cu_q, const int32_t* cu_kv,
+                                  const int32_t* s_base, const int32_t* s_gbase, int id) {
   AttnItem it;
   it.valid = 0;
+  if (s_base != nullptr) {
+    if (id >= s_base[P.N]) return it;
+    int lo = 0, hi = P.N;                      // the largest i with s_base[i] <= id
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (s_base[mid] <= id) lo = mid; else hi = mid;
+    }
+    const int q0 = cu_q[lo], k0 = cu_kv[lo];
+    return attn_item_of_server(P, lo, q0, cu_q[lo + 1] - q0, k0, cu_kv[lo + 1] - k0, s_base[lo], s_gbase[lo], id);
+  }
   int base = 0, gbase = 0;
   for (int i = 0; i < P.N; ++i) {
     const int q0 = cu_q[i], n_new = cu_q[i + 1] - q0;
     const int k0 = cu_kv[i], Lkv = cu_kv[i + 1] - k0;
-    if (n_new <= 0 || Lkv < n_new || Lkv > P.max_kv_len || k0 < 0 || k0 + Lkv > P.total_kv || q0 < 0 ||
-        q0 + n_new > P.Tq)
-      continue;   // flagged by CTA 0
-    const int tgs = (n_new + P.TB - 1) / P.TB;
-    const int nsplit = attn_nsplit(Lkv, P.tiles_per_chunk);
-    const int cnt = tgs * nsplit * P.Hkv;
-    if (id < base + cnt) {
-      int rem = id - base;
-      it.g = rem % P.Hkv; rem /= P.Hkv;
-      it.split = rem % nsplit; it.tg = rem / nsplit;
-      it.server = i;
-      it.item_base = base; it.nsplit = nsplit;
-      it.group = gbase + it.tg * P.Hkv + it.g;
-      it.q_row0 = q0 + it.tg * P.TB;
-      it.n_t = min(P.TB, n_new - it.tg * P.TB);
-      it.kv0 = k0; it.Lkv = Lkv; it.L = Lkv - n_new;
-      const int tiles = (Lkv + kAtTile - 1) / kAtTile;
-      const int tb = tiles / nsplit, tr = tiles % nsplit;
-      it.tile0 = it.split * tb + min(it.split, tr);
-      it.n_tiles = tb + (it.split < tr ? 1 : 0);
-      // keys the block can see end at L + (last position) ; later tiles hold nothing visible
-      const int last_key = it.L + it.tg * P.TB + it.n_t - 1;
-      const int last_tile = last_key / kAtTile;
-      if (it.tile0 + it.n_tiles - 1 > last_tile) it.n_tiles = max(0, last_tile - it.tile0 + 1);
-      it.n_used = 0;
-      for (int sp = 0; sp < nsplit; ++sp)
-        if (sp * tb + min(sp, tr) <= last_tile) it.n_used = sp + 1;
-      it.valid = 1;
-      return it;
-    }
+    int cnt, grp;
+    attn_server_counts(P, q0, n_new, k0, Lkv, cnt, grp);
+    if (id < base + cnt) return attn_item_of_server(P, i, q0, n_new, k0, Lkv, base, gbase, id);
     base += cnt;
-    gbase += tgs * P.Hkv;
+    gbase += grp;
   }
   return it;
 }
+
+static_assert(sizeof(AttnItem) * kAtItemCache <= kAtItemCacheBytes, "item cache too small");
 
 // 2^x on the FMA pipe (x <= 127): floor by the 1.5*2^23 trick, a cubic for 2^f on [0,1] (relative
 // error 9e-5, far below bf16 resolution) and an integer add to the exponent.  One softmax thread
@@ -145,20 +183,28 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
   const uint32_t kv_base = base;
   const uint32_t bars = kv_base + kAtStages * kAtKvBytes;
   // barriers: 0 q_full, 1 item_done, 2-3 s_full[2], 4-5 p_full[2], 6 o_full, 7 pv_done,
-  //           8.. kv_full[S], kv_empty[S], then epi_a, epi_b (the 128 softmax threads meet twice
-  //           per item that took a ticket)
+  //           8.. kv_full[S], kv_empty[S], then epi_a, epi_b (the 128 epilogue threads meet twice
+  //           per item that took a ticket), stats_full (row maxima and sums of an item handed from
+  //           the softmax warps to the epilogue warps), o_drained (O of an item read out of tensor
+  //           memory: the next item's first product may overwrite it)
   auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
   constexpr int kSFull = 2, kPFull = 4, kOFull = 6, kPvDone = 7, kKvFull = 8, kKvEmpty = 8 + kAtStages;
-  constexpr int kEpiA = 8 + 2 * kAtStages, kEpiB = kEpiA + 1;
-  uint8_t* tail = smem_raw + (bars - base) + 8 * (10 + 2 * kAtStages);
+  constexpr int kEpiA = 8 + 2 * kAtStages, kEpiB = kEpiA + 1, kStatsFull = kEpiA + 2, kODrained = kEpiA + 3;
+  uint8_t* tail = smem_raw + (bars - base) + 8 * (12 + 2 * kAtStages);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 4);
   volatile int* s_last = reinterpret_cast<volatile int*>(tail + 8);
   // The offsets are read by every role for every item: keep them in shared memory when they fit.
-  int32_t* s_cu = reinterpret_cast<int32_t*>(smem_raw + kAtStages * kAtKvBytes + 256);
+  float* s_ml = reinterpret_cast<float*>(smem_raw + kAtStages * kAtKvBytes + 256);     // [128][2] row maximum, row sum
+  int32_t* s_cu = reinterpret_cast<int32_t*>(smem_raw + kAtStages * kAtKvBytes + 256 + 1024);
   const bool cached = P.N <= kAtMaxCached;
   const int32_t* cu_q = cached ? s_cu : P.cu_q;
   const int32_t* cu_kv = cached ? s_cu + (P.N + 1) : P.cu_kv;
+  // first item and first group of every server (exclusive prefix sums; entry N = number of items)
+  int32_t* s_base_w = s_cu + 2 * (kAtMaxCached + 1);
+  int32_t* s_gbase_w = s_base_w + (kAtMaxCached + 1);
+  const int32_t* s_base = cached ? s_base_w : nullptr;
+  const int32_t* s_gbase = cached ? s_gbase_w : nullptr;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if ((base & 1023u) != 0) {                     // the operand layouts need a 1024-byte aligned base
@@ -172,6 +218,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
     mbar_init(bar(kOFull), 1); mbar_init(bar(kPvDone), 1);
     for (int s = 0; s < kAtStages; ++s) { mbar_init(bar(kKvFull + s), 1); mbar_init(bar(kKvEmpty + s), 1); }
     mbar_init(bar(kEpiA), 128); mbar_init(bar(kEpiB), 128);
+    mbar_init(bar(kStatsFull), 4); mbar_init(bar(kODrained), 4);
     *abort_flag = 0;
     fence_barrier_init();
     fence_proxy_async();
@@ -181,12 +228,50 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
     tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kAtTmemCols);
     tmem_relinquish();
   } else if (cached) {
-    const int t = (warp == 0) ? (int)threadIdx.x : (int)threadIdx.x - 32;      // 160 loading threads
-    for (int i = t; i <= P.N; i += kAtThreads - 32) { s_cu[i] = P.cu_q[i]; s_cu[P.N + 1 + i] = P.cu_kv[i]; }
+    const int t = (warp == 0) ? (int)threadIdx.x : (int)threadIdx.x - 32;      // every thread but the allocating warp's
+    for (int i = t; i <= P.N; i += kAtThreads - 32) {
+      const int q0 = P.cu_q[i], k0 = P.cu_kv[i];
+      s_cu[i] = q0; s_cu[P.N + 1 + i] = k0;
+      int cnt = 0, grp = 0;
+      if (i < P.N) attn_server_counts(P, q0, P.cu_q[i + 1] - q0, k0, P.cu_kv[i + 1] - k0, cnt, grp);
+      s_base_w[i] = cnt; s_gbase_w[i] = grp;
+    }
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  if (cached && warp == 2) {
+    // counts -> exclusive prefix sums, 32 servers per step
+    int carry = 0, gcarry = 0;
+    for (int c = 0; c <= P.N; c += 32) {
+      const int i = c + lane;
+      const int v = (i < P.N) ? s_base_w[i] : 0, gv = (i < P.N) ? s_gbase_w[i] : 0;
+      int inc = v, ginc = gv;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const int a = __shfl_up_sync(0xffffffffu, inc, d), b = __shfl_up_sync(0xffffffffu, ginc, d);
+        if (lane >= d) { inc += a; ginc += b; }
+      }
+      if (i <= P.N) { s_base_w[i] = carry + inc - v; s_gbase_w[i] = gcarry + ginc - gv; }
+      carry += __shfl_sync(0xffffffffu, inc, 31);
+      gcarry += __shfl_sync(0xffffffffu, ginc, 31);
+    }
+  }
+  __syncthreads();
+  // The descriptors of this CTA's first items, one thread each: a descriptor costs a dozen integer
+  // divisions, which every role would otherwise repeat, one after the other, at every item.
+  AttnItem* s_items = reinterpret_cast<AttnItem*>(s_gbase_w + (kAtMaxCached + 1));
+  if (warp == 3) {
+    const long long id = (long long)blockIdx.x + (long long)lane * gridDim.x;
+    AttnItem it;
+    it.valid = 0;
+    if (id < P.max_items) it = attn_find_item(P, cu_q, cu_kv, s_base, s_gbase, (int)id);
+    s_items[lane] = it;
+  }
+  __syncthreads();
+  auto item_at = [&](int k, int id) -> AttnItem {
+    return k < kAtItemCache ? s_items[k] : attn_find_item(P, cu_q, cu_kv, s_base, s_gbase, id);
+  };
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t tmem_S = tmem_base + kAtColS, tmem_O = tmem_base + kAtColO;     // S buffer b at tmem_S + 128 b
   const uint32_t tmem_Q = tmem_base + kAtColQ;
@@ -208,8 +293,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
     {
       uint32_t st = 0, ph = 0;
       bool ok = true;
-      for (int id = blockIdx.x; id < P.max_items && ok; id += gridDim.x) {
-        const AttnItem it = attn_find_item(P, cu_q, cu_kv, id);
+      for (int id = blockIdx.x, k_item = 0; id < P.max_items && ok; id += gridDim.x, ++k_item) {
+        const AttnItem it = item_at(k_item, id);
         if (!it.valid) break;
         if (it.n_tiles == 0) continue;
         for (int j = 0; j < it.n_tiles; ++j) {
@@ -256,8 +341,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
       }
       __syncwarp();
     };
-    for (int id = blockIdx.x; id < P.max_items && ok; id += gridDim.x) {
-      const AttnItem it = attn_find_item(P, cu_q, cu_kv, id);
+    for (int id = blockIdx.x, k_item = 0; id < P.max_items && ok; id += gridDim.x, ++k_item) {
+      const AttnItem it = item_at(k_item, id);
       if (!it.valid) break;
       if (it.n_tiles == 0) continue;
       // Q of this item sits in tensor memory (written by the softmax warps after they have
@@ -278,6 +363,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
           if (++st_s == kAtStages) { st_s = 0; ph_s ^= 1u; }
         }
         if (!mbar_wait_warp(bar(kPFull + (n & 1)), (uint32_t)(n >> 1) & 1u, abort_flag)) { ok = false; break; }   // P ready
+        if (j == 0 && n_item > 0) {      // the first product overwrites O: the previous item's O must have been read out
+          if (!mbar_wait_warp(bar(kODrained), (uint32_t)(n_item - 1) & 1u, abort_flag)) { ok = false; break; }
+        }
         tc_fence_after();
         if (elect_one()) {
           const uint64_t dv = dv0 + (uint64_t)(st_v * (kAtKvBytes >> 4));
@@ -298,15 +386,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
     }
     if (!ok) { const uint64_t t0 = global_timer_ns(); while (global_timer_ns() - t0 < 200000ull) { } }
     __syncwarp();
-  } else {
-    // ------------------------------------------------ softmax + epilogue: thread = row
+  } else if (warp < 6) {
+    // ------------------------------------------------ softmax: thread = row
     const int q = warp & 3;
     const int r = q * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-    int n_item = 0, n_tile_total = 0, n_ticket = 0;
+    int n_item = 0, n_tile_total = 0;
     bool ok = true;
-    for (int id = blockIdx.x; id < P.max_items && ok; id += gridDim.x) {
-      const AttnItem it = attn_find_item(P, cu_q, cu_kv, id);
+    for (int id = blockIdx.x, k_item = 0; id < P.max_items && ok; id += gridDim.x, ++k_item) {
+      const AttnItem it = item_at(k_item, id);
       if (!it.valid) break;
       if (it.n_tiles == 0) continue;
       const int R = it.n_t * P.G;
@@ -314,7 +402,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
       const int t = it.tg * P.TB + r / P.G;              // position index inside the server
       const int last_visible = it.L + t;                 // keys 0..L+t
       // This thread's query row goes to tensor memory as packed bf16 pairs (the A operand of
-      // S = Q K^T).  The previous item's MMAs are finished: its O was drained above.
+      // S = Q K^T).  The previous item's S products, the only readers of Q, finished before its
+      // last tile of scores was handed to this thread.
       {
         const uint4* qrow = reinterpret_cast<const uint4*>(
             P.Q + ((size_t)(it.q_row0 + r / P.G) * P.Hq + it.g * P.G + (r % P.G)) * kAtHd);
@@ -428,7 +517,31 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
         if (lane == 0) mbar_arrive(bar(kPFull + (n & 1)));
       }
       if (!ok) break;
-      // epilogue
+      // Hand the row statistics to the epilogue warps and go on with the next item.  An item of one
+      // or two tiles can end before the epilogue has picked up the previous item's statistics: wait
+      // until it has (it reads them before it reports O as read out).
+      if (n_item > 0 && !mbar_wait(bar(kODrained), (uint32_t)(n_item - 1) & 1u, abort_flag)) { ok = false; break; }
+      s_ml[2 * r] = m_run; s_ml[2 * r + 1] = l_run;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(kStatsFull));
+      ++n_item;
+    }
+  } else {
+    // ------------------------------------------------ epilogue: thread = row; runs one item behind
+    // the softmax warps, so partial stores, tickets and merges overlap the next item's tiles
+    const int q = warp & 3;
+    const int r = q * 32 + lane;
+    const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+    int n_item = 0, n_ticket = 0;
+    bool ok = true;
+    for (int id = blockIdx.x, k_item = 0; id < P.max_items && ok; id += gridDim.x, ++k_item) {
+      const AttnItem it = item_at(k_item, id);
+      if (!it.valid) break;
+      if (it.n_tiles == 0) continue;
+      const int R = it.n_t * P.G;
+      const bool row_ok = r < R;
+      if (!mbar_wait(bar(kStatsFull), (uint32_t)n_item & 1u, abort_flag)) { ok = false; break; }
+      const float m_run = s_ml[2 * r], l_run = s_ml[2 * r + 1];
       if (!mbar_wait(bar(kOFull), (uint32_t)n_item & 1u, abort_flag)) { ok = false; break; }
       tc_fence_after();
       __nv_bfloat16* orow = P.O + ((size_t)(it.q_row0 + r / P.G) * P.Hq + it.g * P.G + (r % P.G)) * kAtHd;
@@ -462,6 +575,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
         }
       }
       tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(kODrained));          // the statistics were read before this point too
       if (!single) {
         if (row_ok) { out[kAtHd] = m_run; out[kAtHd + 1] = l_run; }
         // One ticket per group: the CTA that takes the last one finds the other splits' rows
@@ -569,8 +684,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
 }
 
 // ------------------------------------------------------------------ host side
+// KV tiles per split forced by gs_verify_attn_configure (0 = automatic).
+inline int& attn_tiles_per_split_override() {
+  static int v = 0;
+  return v;
+}
+
 struct AttnTcPlan {
-  int TB, tiles_per_chunk, max_items, max_groups, grid;
+  int TB, tiles_per_chunk, min_split_tiles, max_items, max_groups, grid;
   size_t ticket_bytes, ws_bytes;
 };
 
@@ -589,9 +710,17 @@ inline AttnTcPlan attn_tc_plan(int N, int Tq, int total_kv, int max_kv_len, int 
   const int tiles_avg = max(1, (total_kv / max(1, N) + kAtTile - 1) / kAtTile);
   const int nsplit_target = max(1, slots / heads_total);
   pl.tiles_per_chunk = max(1, (tiles_avg + nsplit_target - 1) / nsplit_target);
+  pl.min_split_tiles = kAtMinSplitTiles;
+  // at most eight splits per group: the merge handles up to eight partial results per round trip
+  pl.tiles_per_chunk = max(pl.tiles_per_chunk, ((max_kv_len + kAtTile - 1) / kAtTile + 7) / 8);
+  if (attn_tiles_per_split_override() > 0) {
+    pl.tiles_per_chunk = attn_tiles_per_split_override();
+    pl.min_split_tiles = 1;
+  }
   const int max_tiles = (max_kv_len + kAtTile - 1) / kAtTile;
   const long long blocks = (long long)N + Tq / pl.TB;      // sum over servers of ceil(n_new / TB)
-  const long long items = (long long)Hkv * blocks * ((max_tiles + pl.tiles_per_chunk - 1) / pl.tiles_per_chunk);
+  const int max_nsplit = max(1, min((max_tiles + pl.tiles_per_chunk - 1) / pl.tiles_per_chunk, max_tiles / pl.min_split_tiles));
+  const long long items = (long long)Hkv * blocks * max_nsplit;
   pl.max_items = (int)min(items, (long long)INT_MAX / 2);
   pl.grid = min(pl.max_items, slots);
   pl.max_groups = (int)min((long long)Hkv * blocks, (long long)INT_MAX / 2);
@@ -617,7 +746,8 @@ inline gs_status launch_attn_tc(const void* Q, const void* K, const void* V, voi
   P.O = static_cast<__nv_bfloat16*>(O);
   P.Q = static_cast<const __nv_bfloat16*>(Q);
   P.N = N; P.Tq = Tq; P.total_kv = total_kv; P.max_kv_len = max_kv_len; P.Hq = Hq; P.Hkv = Hkv;
-  P.G = Hq / Hkv; P.TB = pl.TB; P.tiles_per_chunk = pl.tiles_per_chunk; P.max_items = pl.max_items;
+  P.G = Hq / Hkv; P.TB = pl.TB; P.tiles_per_chunk = pl.tiles_per_chunk; P.min_split_tiles = pl.min_split_tiles;
+  P.max_items = pl.max_items;
   P.scale_log2 = scale * kAtLog2e;
   auto enc = tensor_map_encoder();
   if (enc == nullptr) return GS_ERR_CUDA;

@@ -4,6 +4,12 @@
 #include "attn_generic.cuh"
 #include "attn_tc.cuh"
 
+extern "C" gs_status gs_verify_attn_configure(int tiles_per_split) {
+  if (tiles_per_split < 0) return GS_ERR_INVALID_ARG;
+  gs::attn_tiles_per_split_override() = tiles_per_split;
+  return GS_OK;
+}
+
 extern "C" size_t gs_verify_attn_workspace(int N, int Tq, int total_kv, int max_kv_len, int Hq, int Hkv,
                                            int hd, gs_dtype dt) {
   using namespace gs;
