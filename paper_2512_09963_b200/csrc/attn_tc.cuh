@@ -207,6 +207,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
   const int32_t* s_gbase = cached ? s_gbase_w : nullptr;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // The next kernel on the stream may set itself up on idle SMs right away (it still waits for this
+  // grid to finish before it touches global memory).  This kernel follows a memset and has no
+  // programmatic predecessor of its own.
+  pdl_launch_dependents();
   if ((base & 1023u) != 0) {                     // the operand layouts need a 1024-byte aligned base
     if (threadIdx.x == 0) set_status(P.d_status, GS_ERR_CUDA);
     return;

@@ -289,8 +289,18 @@ ATTN_CASES = [
 ]
 
 
+@pytest.fixture(params=[0, 1, 3], ids=["auto-splits", "one-tile-splits", "three-tile-splits"])
+def attn_splits(request):
+    """The automatic plan only splits long caches; one- and three-tile splits force partial
+    results, tickets and merges (more than eight splits per group included) and CTAs that walk
+    through many short items."""
+    B.gs_verify_attn_configure(request.param)
+    yield request.param
+    B.gs_verify_attn_configure(0)
+
+
 @pytest.mark.parametrize("name,cfg", ATTN_CASES)
-def test_attention_small(name, cfg):
+def test_attention_small(name, cfg, attn_splits):
     inp = attn_case(cfg)
     O, st = run_attn(inp)
     assert st == 0
@@ -298,6 +308,20 @@ def test_attention_small(name, cfg):
     pu.assert_close_rel(O, ref, f"attention {name}")
     O2, _ = run_attn(inp)
     assert torch.equal(O, O2)                     # deterministic
+
+
+def test_attention_many_short_servers():
+    """More items per CTA than the kernel caches descriptors for (700 servers x 8 KV heads over 148
+    CTAs), most of them a single tile, a few long ones in between."""
+    base = wl.shrink(wl.CONFIGS["cfg2"], prefix_scale=0.0, N=700, name="attn_many")
+    r = np.random.default_rng(7)
+    gamma = r.integers(0, 4, 700)
+    prefix = r.integers(0, 40, 700)
+    prefix[[5, 333, 699]] = [1500, 700, 2600]
+    inp = wl.make_attention_inputs(base, gamma, prefix)
+    O, st = run_attn(inp)
+    assert st == 0
+    pu.assert_close_rel(O, orc.ref_attention(inp["Q"], inp["K"], inp["V"], inp["cu_q"], inp["cu_kv"]), "many servers")
 
 
 def test_attention_edge_shapes():
