@@ -243,9 +243,14 @@ gs_status gs_schedule_select(int variant);
  *            attention output O and the logits of the round
  *   outputs  h_accepted[N], h_out_tok[T_q], h_n_out[N], h_S_next[N], h_status[1] (device status)
  * The call enqueues host->device copies, gs_verify_attn, gs_lm_head_logits, gs_spec_accept (with
- * the estimator update), gs_schedule and the device->host copies on `stream` and returns; the host
- * outputs are valid after the caller synchronises the stream.  Host buffers must stay untouched
- * until then.  Errors: as the four calls; CUDA if a copy could not be enqueued.
+ * the estimator update), gs_schedule and the device->host copies and returns; the host outputs are
+ * valid after the caller synchronises `stream`.  Host buffers must stay untouched until then.
+ * The draft distributions, tokens and uniforms (read only by the acceptance pass) are copied on a
+ * stream of the library's own (one per device, created on the first call together with two events;
+ * make that first call outside any stream capture) while attention and the LM head run on `stream`;
+ * `stream` waits for them before gs_spec_accept, and they wait for `stream` to reach this call, so
+ * back-to-back rounds on one stream are ordered.  Rounds issued on DIFFERENT streams with the same
+ * d_ws race, as they would anyway.  Errors: as the four calls; CUDA if a copy could not be enqueued.
  */
 typedef struct gs_round_desc {
   int N, Tq, total_kv, max_kv_len, Hq, Hkv, hd, d, V, C;

@@ -1,7 +1,10 @@
 // gs_verify_round_host: one whole verification round for a caller whose per-round data lives in
 // host memory (what the draft servers sent this round), with the model state resident on the GPU.
-// It stages the inputs with cudaMemcpyAsync, enqueues the four steps of the round on the same
-// stream and copies the small results back; nothing here computes.
+// It stages the inputs with cudaMemcpyAsync, enqueues the four steps of the round and copies the
+// small results back; nothing here computes.  The draft distributions are by far the largest
+// input (Gamma x V floats) and only the acceptance pass reads them, so they travel on a copy stream
+// of the library's own while attention and the LM head run; an event hands them to the caller's
+// stream before gs_spec_accept.
 #include "common.cuh"
 
 namespace gs {
@@ -48,6 +51,30 @@ static RoundLayout round_layout(const gs_round_desc& r) {
   return L;
 }
 
+// One copy stream and two events per device, created on first use and kept for the process.
+struct RoundSide {
+  cudaStream_t copy = nullptr;
+  cudaEvent_t begin = nullptr, staged = nullptr;
+  bool ok = false;
+};
+static RoundSide* round_side() {
+  constexpr int kMaxDevices = 64;
+  static RoundSide side[kMaxDevices];
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  RoundSide& s = side[dev];
+  if (!s.ok) {
+    if (cudaStreamCreateWithFlags(&s.copy, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&s.begin, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&s.staged, cudaEventDisableTiming) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return nullptr;
+    }
+    s.ok = true;
+  }
+  return &s;
+}
+
 static bool desc_ok(const gs_round_desc* r) {
   return r != nullptr && r->N > 0 && r->Tq >= r->N && r->total_kv > 0 && r->max_kv_len > 0 && r->Hq > 0 &&
          r->Hkv > 0 && r->hd > 0 && r->d > 0 && r->V > 0 && r->C >= 0 && (r->dt == GS_F32 || r->dt == GS_BF16);
@@ -83,17 +110,27 @@ extern "C" gs_status gs_verify_round_host(const gs_round_desc* r,
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   char* w = static_cast<char*>(d_ws);
   const size_t Tq = (size_t)r->Tq, N = (size_t)r->N, V = (size_t)r->V, es = esize(r->dt);
-  auto h2d = [&](size_t off, const void* src, size_t bytes) {
-    return bytes == 0 || cudaMemcpyAsync(w + off, src, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  auto h2d_on = [&](cudaStream_t q, size_t off, const void* src, size_t bytes) {
+    return bytes == 0 || cudaMemcpyAsync(w + off, src, bytes, cudaMemcpyHostToDevice, q) == cudaSuccess;
   };
+  auto h2d = [&](size_t off, const void* src, size_t bytes) { return h2d_on(st, off, src, bytes); };
   auto d2h = [&](void* dst, size_t off, size_t bytes) {
     return cudaMemcpyAsync(dst, w + off, bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
   };
+  // First what attention and the LM head need, on the caller's stream (copies are served in the
+  // order they are issued, so the large one must not be queued ahead of these) ...
   bool ok = h2d(L.Q, h_Q, Tq * r->Hq * r->hd * es) && h2d(L.H, h_H, Tq * r->d * es) &&
-            h2d(L.q_probs, h_q_probs, Gamma * V * 4) && h2d(L.draft_tok, h_draft_tok, Gamma * 4) &&
-            h2d(L.u_accept, h_u_accept, Gamma * 4) && h2d(L.u_sample, h_u_sample, N * 4) &&
             h2d(L.cu_q, h_cu_q, (N + 1) * 4) && h2d(L.cu_kv, h_cu_kv, (N + 1) * 4);
   if (!ok || cudaMemsetAsync(w + L.status, 0, 4, st) != cudaSuccess) return GS_ERR_CUDA;
+  // ... then what only the acceptance pass reads, over the copy stream.  It starts once the caller's
+  // stream has reached this call (the previous round may still be reading the staging area).
+  RoundSide* side = round_side();
+  if (side == nullptr) return GS_ERR_CUDA;
+  if (cudaEventRecord(side->begin, st) != cudaSuccess || cudaStreamWaitEvent(side->copy, side->begin, 0) != cudaSuccess)
+    return GS_ERR_CUDA;
+  ok = h2d_on(side->copy, L.draft_tok, h_draft_tok, Gamma * 4) && h2d_on(side->copy, L.u_accept, h_u_accept, Gamma * 4) &&
+       h2d_on(side->copy, L.u_sample, h_u_sample, N * 4) && h2d_on(side->copy, L.q_probs, h_q_probs, Gamma * V * 4);
+  if (!ok || cudaEventRecord(side->staged, side->copy) != cudaSuccess) return GS_ERR_CUDA;
   int32_t* d_status = reinterpret_cast<int32_t*>(w + L.status);
   const int32_t* cu_q = reinterpret_cast<const int32_t*>(w + L.cu_q);
   const int32_t* cu_kv = reinterpret_cast<const int32_t*>(w + L.cu_kv);
@@ -103,6 +140,7 @@ extern "C" gs_status gs_verify_round_host(const gs_round_desc* r,
   s = gs_lm_head_logits(w + L.H, d_W, reinterpret_cast<float*>(w + L.logits), r->Tq, r->d, r->V, r->dt,
                         w + L.ws_head, L.ws_head_bytes, d_status, st);
   if (s != GS_OK) return s;
+  if (cudaStreamWaitEvent(st, side->staged, 0) != cudaSuccess) return GS_ERR_CUDA;
   s = gs_spec_accept(reinterpret_cast<const float*>(w + L.logits), reinterpret_cast<const float*>(w + L.q_probs),
                      reinterpret_cast<const int32_t*>(w + L.draft_tok), cu_q,
                      reinterpret_cast<const float*>(w + L.u_accept), reinterpret_cast<const float*>(w + L.u_sample),

@@ -371,6 +371,42 @@ def test_attention_bad_offsets_are_flagged():
     assert st == 2
 
 
+# ------------------------------------------------------------------ the round from host buffers
+def test_verify_round_host_matches_device_path():
+    """gs_verify_round_host (inputs in pinned host memory, draft distributions copied on the
+    library's copy stream while attention and the LM head run) gives what the four calls give on
+    device-resident inputs; two rounds back to back with different drafts reuse the staging area."""
+    cfg = wl.shrink(wl.CONFIGS["cfg2"], d=256, V=16384, prefix_scale=0.1, name="host_round")
+    for round_idx in (0, 1):
+        inp = wl.make_step(cfg, round_idx=round_idx, gamma=[3, 1, 8, 2, 5, 4, 7, 6])     # same shapes, new drafts
+        d = to_dev(inp)
+        N, Tq = cfg.N, int(inp["cu_q"][-1])
+        rnd = VerifyRound.for_inputs(d, C=4 * N)
+        rnd.run(d)
+        torch.cuda.synchronize()
+        assert int(rnd.d_status.item()) == 0
+        desc = B.RoundDesc(N=N, Tq=Tq, total_kv=d["K"].shape[0], max_kv_len=rnd.max_kv_len, Hq=cfg.Hq, Hkv=cfg.Hkv,
+                           hd=cfg.hd, d=cfg.d, V=cfg.V, C=4 * N, dt=B.GS_BF16, scale=cfg.hd ** -0.5,
+                           temperature=float(inp["tau"]), eta=0.1, beta=0.5, alpha_min=1e-3, alpha_max=0.999)
+        if round_idx == 0:
+            ws = torch.empty(B.gs_verify_round_workspace(desc), dtype=torch.uint8, device=DEV)
+        pin = {k: inp[k].contiguous().pin_memory() for k in
+               ("Q", "H", "q_probs", "draft_tok", "u_accept", "u_sample", "cu_q", "cu_kv")}
+        outs = {k: torch.full((n,), -9, dtype=torch.int32).pin_memory() for k, n in
+                (("accepted", N), ("out_tok", Tq), ("n_out", N), ("S_next", N), ("status", 1))}
+        a_hat = torch.full((N,), 0.5, dtype=torch.float64, device=DEV)
+        X = torch.ones(N, dtype=torch.float64, device=DEV)
+        B.gs_verify_round_host(desc, pin["Q"], pin["H"], pin["q_probs"], pin["draft_tok"], pin["u_accept"],
+                               pin["u_sample"], pin["cu_q"], pin["cu_kv"], d["K"], d["V"], d["W"], a_hat, X,
+                               None, None, ws, outs["accepted"], outs["out_tok"], outs["n_out"], outs["S_next"],
+                               outs["status"])
+        torch.cuda.synchronize()
+        assert int(outs["status"][0]) == 0
+        for k in ("accepted", "out_tok", "n_out", "S_next"):
+            assert torch.equal(outs[k], getattr(rnd, k).cpu()), (round_idx, k)
+        assert torch.equal(a_hat, rnd.alpha_hat) and torch.equal(X, rnd.X)
+
+
 # ------------------------------------------------------------------ LM head
 @pytest.mark.parametrize("variant", [2, 1], ids=["cta-pairs", "one-cta"])
 @pytest.mark.parametrize("T,d,V", [(44, 512, 9000), (96, 1024, 4104), (288, 256, 8192), (1, 64, 8), (130, 136, 1000),
