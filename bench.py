@@ -502,7 +502,15 @@ def main():
             from paper_2512_09963_b200 import build as gs_build
             from paper_2512_09963_b200.closed_loop import run_closed_loop
             gs_build.build()
-            rep = run_closed_loop(cfg, args.rounds, device=f"cuda:{local_rank}")
+            rep = run_closed_loop(cfg, args.rounds, device=f"cuda:{local_rank}", curve_every=max(1, args.rounds // 20))
+            # the paper's two baselines on the same simulated servers (Sec. V): Fixed-S and Random-S
+            rep["baseline_policies"] = {}
+            for pol in ("fixed", "random"):
+                r2 = run_closed_loop(cfg, args.rounds, device=f"cuda:{local_rank}", policy=pol,
+                                     curve_every=max(1, args.rounds // 20))
+                rep["baseline_policies"][pol] = {k: r2[k] for k in ("utility_sum_log", "jain", "goodput_tokens_per_s",
+                                                                     "verified_tokens_per_s", "gpu_ms_per_round",
+                                                                     "utility_curve")}
             rep.update(metric=METRIC, unit=UNIT, value=rep["verified_tokens_per_s"], n_gpus=1, dtype=cfg.dtype,
                        data="synthetic", config={"workload": "cfg5", "servers": cfg.N, "budget_C": cfg.C,
                                                  "drift": "true alpha ~ Beta(4,2) redrawn every 100 rounds",

@@ -18,10 +18,24 @@ from . import binding as B
 from . import workloads as wl
 
 
+POLICIES = ("goodspeed", "fixed", "random")
+
+
 class ClosedLoop:
-    def __init__(self, cfg: wl.VerifyConfig, device="cuda", epoch=100, eta=0.1, beta=0.5, s_min=0):
+    """policy: who decides S(t+1).  "goodspeed" = the scheduler's allocation (Eq. goodspeed_sched);
+    "fixed" = Fixed-S, C/N tokens for every server; "random" = Random-S, the budget thrown at the
+    servers uniformly at random (the two baselines of Sec. V).  The estimators are updated in every
+    case.  step_decay > 0 shrinks both smoothing steps as (t+1)^-step_decay (Assumption 3 asks for
+    steps with divergent sum and convergent sum of squares, e.g. 0.5 < step_decay <= 1)."""
+
+    def __init__(self, cfg: wl.VerifyConfig, device="cuda", epoch=100, eta=0.1, beta=0.5, s_min=0,
+                 policy="goodspeed", step_decay=0.0):
+        if policy not in POLICIES:
+            raise ValueError(f"policy must be one of {POLICIES}")
         self.cfg, self.dev, self.epoch = cfg, torch.device(device), epoch
+        self.eta0, self.beta0, self.step_decay = eta, beta, float(step_decay)
         self.eta, self.beta = eta, beta
+        self.policy = policy
         N, C = cfg.N, cfg.C
         self.N, self.C = N, C
         self.max_new = C + 1                                   # a single server can get the whole budget
@@ -92,6 +106,22 @@ class ClosedLoop:
         inp["u_sample"] = torch.from_numpy(wl.open_uniform(wl._rng(cfg, "u_sample", t), self.N)).to(self.dev)
         return inp
 
+    def set_round(self, t):
+        """Step sizes of round t."""
+        if self.step_decay > 0.0:
+            f = float(t + 1) ** -self.step_decay
+            self.eta, self.beta = self.eta0 * f, self.beta0 * f
+
+    def next_allocation(self, t):
+        """S(t+1) under the loop's policy (host integers); gs_schedule has already run."""
+        N, C = self.N, self.C
+        if self.policy == "goodspeed":
+            return self.S_next.cpu().numpy().astype(np.int64)
+        if self.policy == "fixed":
+            return np.full(N, C // N, dtype=np.int64)
+        rng = wl._rng(self.cfg, "random_s", t)
+        return np.bincount(rng.integers(0, N, size=C), minlength=N).astype(np.int64)
+
     # ---------------------------------------------------------------- one round on the GPU
     def gpu_round(self, inp):
         cfg = self.cfg
@@ -114,10 +144,13 @@ def jain(x):
     return float(x.sum() ** 2 / (len(x) * (x * x).sum()))
 
 
-def run_closed_loop(cfg: wl.VerifyConfig, rounds: int, device="cuda", on_round=None):
+def run_closed_loop(cfg: wl.VerifyConfig, rounds: int, device="cuda", on_round=None, policy="goodspeed",
+                    step_decay=0.0, curve_every=0):
     """Runs `rounds` rounds; returns the report dict.  on_round(t, loop, inp, O, logits) is called after
-    each round is enqueued and synchronised (tests use it to compare with the oracle in lock-step)."""
-    loop = ClosedLoop(cfg, device)
+    each round is enqueued and synchronised (tests use it to compare with the oracle in lock-step).
+    curve_every > 0 adds the utility of the running mean goodput, U(x_bar(t)), every that many rounds."""
+    loop = ClosedLoop(cfg, device, policy=policy, step_decay=step_decay)
+    curve = []
     N = cfg.N
     tot = np.zeros(N)
     x_hist, X_hist = [], []
@@ -126,6 +159,7 @@ def run_closed_loop(cfg: wl.VerifyConfig, rounds: int, device="cuda", on_round=N
     drafted = 0
     for t in range(rounds):
         inp = loop.make_inputs(t, loop.S)
+        loop.set_round(t)
         e0.record()
         O, logits = loop.gpu_round(inp)
         e1.record()
@@ -139,12 +173,15 @@ def run_closed_loop(cfg: wl.VerifyConfig, rounds: int, device="cuda", on_round=N
         drafted += int(loop.S.sum())
         x_hist.append(x)
         X_hist.append(loop.X.cpu().numpy().copy())
-        loop.S = loop.S_next.cpu().numpy().astype(np.int64)
+        loop.S = loop.next_allocation(t)
+        if curve_every > 0 and (t + 1) % curve_every == 0:
+            curve.append([t + 1, float(np.log(tot / (t + 1)).sum())])
     xbar = tot / rounds
     xh, Xh = np.asarray(x_hist), np.asarray(X_hist)
     ma = lambda a: np.convolve(a, np.ones(10) / 10, mode="valid") if len(a) >= 10 else a
     est_err = float(np.mean(np.abs(ma(xh.sum(1)) - ma(Xh.sum(1))))) if rounds >= 10 else None
-    return {"rounds": rounds, "goodput_per_server": [float(v) for v in xbar], "jain": jain(xbar),
+    return {"policy": policy, "step_decay": step_decay, "utility_curve": curve,
+            "rounds": rounds, "goodput_per_server": [float(v) for v in xbar], "jain": jain(xbar),
             "utility_sum_log": float(np.log(xbar).sum()), "gpu_ms_per_round": gpu_ms / rounds,
             "verified_tokens_per_s": drafted / (gpu_ms * 1e-3), "goodput_tokens_per_s": float(tot.sum()) / (gpu_ms * 1e-3),
             "estimated_vs_realised_goodput_ma10_abs_err": est_err,

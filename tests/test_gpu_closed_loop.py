@@ -78,3 +78,29 @@ def test_closed_loop_full_shapes_few_rounds():
     rep, state = lockstep(wl.CONFIGS["cfg5"], 3)
     assert rep["rounds"] == 3 and len(rep["goodput_per_server"]) == 16
     assert state["flips"] <= 1
+
+
+def test_policies_goodspeed_beats_fixed_and_random_in_utility():
+    """Sec. V compares GoodSpeed with Fixed-S and Random-S on the utility of the mean goodput,
+    sum_i log x_bar_i.  Same simulated servers, same rounds, the library's round on the GPU; only the
+    rule for S(t+1) differs.  Stationary, spread-out acceptance rates (one epoch)."""
+    cfg = dataclasses.replace(wl.CONFIGS["cfg5"], name="cfg5_policies", d=128, V=4096, Hq=8, Hkv=1, hd=128,
+                              prefix_lo=96, prefix_hi=96, N=8, C=40)
+    rounds = 100
+    util = {}
+    for pol in ("goodspeed", "fixed", "random"):
+        rep = run_closed_loop(cfg, rounds, policy=pol, curve_every=20)
+        util[pol] = rep["utility_sum_log"]
+        assert rep["policy"] == pol and len(rep["utility_curve"]) == 5
+        assert all(x >= 1.0 for x in rep["goodput_per_server"])          # every server gets its bonus/correction token
+    assert util["goodspeed"] >= util["fixed"] - 1e-9, util
+    assert util["goodspeed"] > util["random"], util
+
+
+def test_decaying_steps_run_and_converge():
+    """Assumption 3 (steps with divergent sum, convergent sum of squares): the loop runs with
+    (t+1)^-0.6 steps and the goodput estimate X stays within the range of per-round goodputs."""
+    cfg = dataclasses.replace(wl.CONFIGS["cfg5"], name="cfg5_decay", d=128, V=4096, Hq=8, Hkv=1, hd=128,
+                              prefix_lo=96, prefix_hi=96, N=8, C=40)
+    rep = run_closed_loop(cfg, 60, step_decay=0.6)
+    assert rep["step_decay"] == 0.6 and 0.5 < rep["jain"] <= 1.0
