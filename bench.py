@@ -164,7 +164,7 @@ def run_reference(args, cfg, rank, world):
     _, host = make_host_inputs(cfg, dev)
     if dev == "cuda":
         torch.cuda.empty_cache()
-    C = 8 * cfg.N
+    C = cfg.C if cfg.C else 8 * cfg.N
     t0 = time.time()
     oracle_round(subset_servers(host, 1), 1, 8)            # calibration: one server
     t1 = time.time() - t0
@@ -209,7 +209,7 @@ def run_ours(args, cfg, rank, world, local_rank):
     inp, host = make_host_inputs(cfg_r, dev)
     N, Tq = cfg.N, int(inp["cu_q"][-1])
     Gamma = int(inp["gamma"].sum())
-    C = 8 * N
+    C = cfg.C if cfg.C else 8 * N
     rnd = VerifyRound.for_inputs(inp, C=C, eta=ETA, beta=BETA)
     s_min = torch.ones(N * world, dtype=torch.int32, device=dev)
     s_max = torch.full((N * world,), 8, dtype=torch.int32, device=dev)
@@ -470,7 +470,7 @@ def main():
                     help="timed steps (default 2000; 20 for --impl reference, whose steps are CPU-seconds long)")
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--config", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5", "cfg6"])
     ap.add_argument("--rounds", type=int, default=1000, help="rounds of the closed loop (--config cfg5)")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--skip-cpu-baseline", action="store_true")

@@ -79,7 +79,7 @@ gs_status gs_set_dependent_launch(int on);
  *   dt: GS_F32 (fp32 in/out) or GS_BF16 (bf16 in/out); scores, softmax and accumulation fp32.
  *   max_kv_len: an upper bound on any server's cu_kv[i+1]-cu_kv[i] (sizes the split-KV scratch).
  *   scale: multiplies q.k (pass 1/sqrt(hd)).
- * GS_BF16 with hd = 128 and a group size Hq/Hkv that divides 128 runs on the tensor cores
+ * GS_BF16 with hd = 128 and a group size Hq/Hkv of at most 128 runs on the tensor cores
  * (tcgen05, split over the KV length, partial results merged from the workspace); every other
  * shape runs a plain kernel.
  * Errors: INVALID_ARG (null/negative), SHAPE (Hq % Hkv != 0), UNSUPPORTED (hd > 256, T_q > 65535),

@@ -702,7 +702,7 @@ struct AttnTcPlan {
 inline bool attn_tc_supported(int Hq, int Hkv, int hd, gs_dtype dt) {
   if (dt != GS_BF16 || hd != kAtHd || Hkv <= 0 || Hq % Hkv != 0) return false;
   const int G = Hq / Hkv;
-  return G >= 1 && G <= 128 && (128 % G) == 0 && (Hkv * hd) % 8 == 0;
+  return G >= 1 && G <= 128 && (Hkv * hd) % 8 == 0;     // floor(128 / G) positions per tile; leftover rows are masked
 }
 
 inline AttnTcPlan attn_tc_plan(int N, int Tq, int total_kv, int max_kv_len, int Hq, int Hkv) {

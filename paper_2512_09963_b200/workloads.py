@@ -80,6 +80,13 @@ CONFIGS = {
     "cfg5": VerifyConfig("cfg5", N=16, d=5120, Hq=64, Hkv=8, hd=128, V=151936, dtype="bf16", tau=0.7,
                          gamma_mode="given", C=128,
                          prefix_mode="fixed", prefix_lo=2048, prefix_hi=2048),
+    # The paper's own deployment scale (Sec. V: 8 clients, token budget C = 20, up to 150 generated
+    # tokens per prompt) on a 14B-class layer: 40 query heads over 8 KV heads (a group of 5, which
+    # does not divide the 128 rows of a score tile), short ragged prefixes, small drafts.
+    "cfg6": VerifyConfig("cfg6", N=8, d=5120, Hq=40, Hkv=8, hd=128, V=151936, dtype="bf16", tau=1.0,
+                         gamma_mode="alloc", gamma_lo=1, gamma_hi=8, C=20,
+                         prefix_mode="uniform", prefix_lo=200, prefix_hi=1200,
+                         sigma_lo=0.2, sigma_hi=1.5),
 }
 
 

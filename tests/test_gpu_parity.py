@@ -310,6 +310,20 @@ def test_attention_small(name, cfg, attn_splits):
     assert torch.equal(O, O2)                     # deterministic
 
 
+@pytest.mark.parametrize("Hq,Hkv", [(40, 8), (6, 2), (4, 4), (7, 1), (128, 1)],
+                         ids=["group-5", "group-3", "no-grouping", "group-7", "group-128"])
+def test_attention_group_sizes(Hq, Hkv):
+    """Query-to-KV head ratios that do not divide the 128 rows of a score tile (floor(128/G) positions
+    per tile, the leftover rows masked), no grouping at all, and one position per tile."""
+    import dataclasses
+    cfg = dataclasses.replace(wl.shrink(wl.CONFIGS["cfg2"], prefix_scale=0.12, N=3, name=f"attn_g{Hq}_{Hkv}"),
+                              Hq=Hq, Hkv=Hkv)
+    inp = wl.make_attention_inputs(cfg, np.array([8, 0, 30]), np.array([245, 130, 300]))
+    O, st = run_attn(inp)
+    assert st == 0
+    pu.assert_close_rel(O, orc.ref_attention(inp["Q"], inp["K"], inp["V"], inp["cu_q"], inp["cu_kv"]), f"G={Hq // Hkv}")
+
+
 def test_attention_many_short_servers():
     """More items per CTA than the kernel caches descriptors for (700 servers x 8 KV heads over 148
     CTAs), most of them a single tile, a few long ones in between."""
@@ -489,3 +503,7 @@ def test_cfg3_full_size():
 
 def test_cfg4_full_size():
     _full_round("cfg4", C=128)
+
+
+def test_cfg6_paper_scale_full_size():
+    _full_round("cfg6", C=20)
