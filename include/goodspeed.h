@@ -102,6 +102,31 @@ gs_status gs_verify_attn(const void* Q, const void* K, const void* V, void* O,
                          void* ws, size_t ws_bytes, int32_t* d_status, void* stream);
 
 /* --------------------------------------------------------------------------------------------
+ * gs_verify_attn_paged -- the same attention (Sec. II-A2) over caches that grow: Sec. III-A has
+ * every round append the verified tokens to each server's prefix, so the caches are kept as pages
+ * of a pool and a server's cache grows by whole pages without being moved.
+ *
+ *   K_pool, V_pool [n_pages * 128, Hkv, hd]   pages of 128 rows (bf16)
+ *   block_table    [N, max_pages] int32       page of server i's t-th run of 128 keys (entries beyond
+ *                                             the server's length are not read)
+ *   cu_kv          [N+1] int32                running sum of the cache LENGTHS (new positions included);
+ *                                             key k of server i is row (block_table[i][k/128]*128 + k%128)
+ *   everything else as gs_verify_attn; max_kv_len <= max_pages * 128 bounds every length.
+ *   Rows of a page beyond the cache length are masked by index but still pass through the tensor
+ *   cores with weight zero: they must hold finite numbers (initialise the pool once; stale rows of
+ *   earlier use are fine, NaN or Inf bit patterns are not).
+ * Tensor-core path only (GS_BF16, hd = 128): other shapes return UNSUPPORTED.
+ * Errors: INVALID_ARG, SHAPE, UNSUPPORTED, WORKSPACE.  Device status: GS_ERR_SHAPE as gs_verify_attn,
+ * GS_ERR_INVALID_ARG for a block-table entry outside [0, n_pages).
+ */
+size_t gs_verify_attn_paged_workspace(int N, int Tq, int max_kv_len, int Hq, int Hkv, int hd, gs_dtype dt);
+gs_status gs_verify_attn_paged(const void* Q, const void* K_pool, const void* V_pool, void* O,
+                               const int32_t* cu_q, const int32_t* cu_kv, const int32_t* block_table,
+                               int N, int Tq, int n_pages, int max_pages, int max_kv_len,
+                               int Hq, int Hkv, int hd, float scale, gs_dtype dt,
+                               void* ws, size_t ws_bytes, int32_t* d_status, void* stream);
+
+/* --------------------------------------------------------------------------------------------
  * gs_lm_head_logits -- Sec. II-A1: logits = W h for every verify position.
  *
  *   H      [T, d]   hidden states, row-major (d contiguous)

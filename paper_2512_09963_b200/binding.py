@@ -29,6 +29,9 @@ SIGNATURES = {
     "gs_verify_attn_workspace": (_sz, [_i, _i, _i, _i, _i, _i, _i, _i]),
     "gs_verify_attn": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _i, _f, _i,
                             _vp, _sz, _vp, _vp]),
+    "gs_verify_attn_paged_workspace": (_sz, [_i, _i, _i, _i, _i, _i, _i]),
+    "gs_verify_attn_paged": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _i, _i, _f, _i,
+                                  _vp, _sz, _vp, _vp]),
     "gs_lm_head_workspace": (_sz, [_i, _i, _i, _i]),
     "gs_lm_head_configure": (_i, [_i, _i, _i]),
     "gs_lm_head_select": (_i, [_i]),
@@ -137,6 +140,25 @@ def gs_verify_attn(Q, K, V, O, cu_q, cu_kv, max_kv_len, scale, ws, d_status=None
                                 _ptr(ws), ws.numel() * ws.element_size(), _ptr(d_status, torch.int32),
                                 _stream())
     _check("gs_verify_attn", code)
+
+
+def gs_verify_attn_paged_workspace(N, Tq, max_kv_len, Hq, Hkv, hd, dt) -> int:
+    return lib().gs_verify_attn_paged_workspace(N, Tq, max_kv_len, Hq, Hkv, hd, dt)
+
+
+def gs_verify_attn_paged(Q, K_pool, V_pool, O, cu_q, cu_kv, block_table, max_kv_len, scale, ws, d_status=None):
+    """K_pool, V_pool: [n_pages * 128, Hkv, hd]; block_table: [N, max_pages] int32; cu_kv: running sum
+    of the cache lengths."""
+    Tq, Hq, hd = Q.shape
+    rows, Hkv, _ = K_pool.shape
+    N, max_pages = block_table.shape
+    code = lib().gs_verify_attn_paged(_ptr(Q), _ptr(K_pool, Q.dtype), _ptr(V_pool, Q.dtype), _ptr(O, Q.dtype),
+                                      _ptr(cu_q, torch.int32), _ptr(cu_kv, torch.int32),
+                                      _ptr(block_table, torch.int32), N, Tq, rows // 128, max_pages,
+                                      int(max_kv_len), Hq, Hkv, hd, float(scale), _dt(Q),
+                                      _ptr(ws), ws.numel() * ws.element_size(), _ptr(d_status, torch.int32),
+                                      _stream())
+    _check("gs_verify_attn_paged", code)
 
 
 def gs_lm_head_workspace(T, d, V, dt) -> int:

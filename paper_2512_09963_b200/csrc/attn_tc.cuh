@@ -47,6 +47,8 @@ constexpr float kAtLog2e = 1.4426950408889634f;
 struct AttnTcParams {
   const int32_t* cu_q;
   const int32_t* cu_kv;
+  const int32_t* block_table;   // paged caches: [N][max_pages] page of every 128-key tile of a server; NULL = contiguous
+  int max_pages, n_pages;
   float* part;              // [items][128][132]
   int* tickets;             // [groups] splits of a (server, position block, KV head) that are done
   __nv_bfloat16* O;
@@ -82,6 +84,7 @@ GS_DEVINL int attn_nsplit(int Lkv, int tiles_per_chunk, int min_split_tiles) {
 // Items of one server (0 when its offsets are inconsistent: such servers are skipped everywhere
 // and flagged by CTA 0) and its (position block, KV head) groups.
 GS_DEVINL bool attn_server_ok(const AttnTcParams& P, int q0, int n_new, int k0, int Lkv) {
+  if (P.block_table != nullptr && Lkv > P.max_pages * kAtTile) return false;
   return !(n_new <= 0 || Lkv < n_new || Lkv > P.max_kv_len || k0 < 0 || k0 + Lkv > P.total_kv || q0 < 0 ||
            q0 + n_new > P.Tq);
 }
@@ -287,9 +290,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
       for (int i = lane - 1; i < P.N; i += 31) {
         const int q0 = P.cu_q[i], n_new = P.cu_q[i + 1] - q0;
         const int k0 = P.cu_kv[i], Lkv = P.cu_kv[i + 1] - k0;
-        if (n_new <= 0 || Lkv < n_new || Lkv > P.max_kv_len || k0 < 0 || k0 + Lkv > P.total_kv || q0 < 0 ||
-            q0 + n_new > P.Tq)
+        if (!attn_server_ok(P, q0, n_new, k0, Lkv)) {
           set_status(P.d_status, GS_ERR_SHAPE);
+        } else if (P.block_table != nullptr) {
+          // every tile of the server must name a page of the pool (a bad entry would only read the
+          // tensor map's fill value, but the result would be meaningless)
+          for (int t = 0; t < (Lkv + kAtTile - 1) / kAtTile; ++t) {
+            const int pg = P.block_table[(size_t)i * P.max_pages + t];
+            if (pg < 0 || pg >= P.n_pages) set_status(P.d_status, GS_ERR_INVALID_ARG);
+          }
+        }
       }
     }
     __syncwarp();
@@ -306,7 +316,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
           if (elect_one()) {
             mbar_arrive_expect_tx(bar(kKvFull + st), kAtKvBytes);
             const uint32_t dst = kv_base + st * kAtKvBytes;
-            const int key = it.kv0 + (it.tile0 + j) * kAtTile;
+            // contiguous caches: the server's rows follow one another; paged caches: tile = page
+            const int key = (P.block_table == nullptr)
+                                ? it.kv0 + (it.tile0 + j) * kAtTile
+                                : P.block_table[(size_t)it.server * P.max_pages + it.tile0 + j] * kAtTile;
             const int col = it.g * kAtHd;
             tma_load_2d(dst, &tmapK, col, key, bar(kKvFull + st));
             tma_load_2d(dst + kAtHalfBytes, &tmapK, col + 64, key, bar(kKvFull + st));
@@ -733,9 +746,13 @@ inline AttnTcPlan attn_tc_plan(int N, int Tq, int total_kv, int max_kv_len, int 
   return pl;
 }
 
+// block_table == NULL: K, V are [total_kv] rows, server i at cu_kv[i].  Otherwise K, V are pools of
+// n_pages pages of 128 rows, block_table[i][t] is the page of server i's t-th tile, and cu_kv only
+// carries the lengths (total_kv is then the bound on cu_kv[N] the plan was made for).
 inline gs_status launch_attn_tc(const void* Q, const void* K, const void* V, void* O, const int32_t* cu_q,
                                 const int32_t* cu_kv, int N, int Tq, int total_kv, int max_kv_len, int Hq, int Hkv,
-                                float scale, void* ws, int32_t* d_status, cudaStream_t st) {
+                                float scale, void* ws, int32_t* d_status, cudaStream_t st,
+                                const int32_t* block_table = nullptr, int max_pages = 0, int n_pages = 0) {
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAtSmem) != cudaSuccess)
@@ -745,6 +762,7 @@ inline gs_status launch_attn_tc(const void* Q, const void* K, const void* V, voi
   const AttnTcPlan pl = attn_tc_plan(N, Tq, total_kv, max_kv_len, Hq, Hkv);
   AttnTcParams P;
   P.cu_q = cu_q; P.cu_kv = cu_kv; P.d_status = d_status;
+  P.block_table = block_table; P.max_pages = max_pages; P.n_pages = n_pages;
   P.tickets = static_cast<int*>(ws);
   P.part = reinterpret_cast<float*>(static_cast<char*>(ws) + pl.ticket_bytes);
   P.O = static_cast<__nv_bfloat16*>(O);
@@ -756,9 +774,10 @@ inline gs_status launch_attn_tc(const void* Q, const void* K, const void* V, voi
   auto enc = tensor_map_encoder();
   if (enc == nullptr) return GS_ERR_CUDA;
   CUtensorMap tmK, tmV;
-  // K, V [total_kv][Hkv*hd]: box = 64 columns x 128 keys
-  if (!make_tmap_bf16_2d(&tmK, K, (uint64_t)total_kv, (uint64_t)Hkv * kAtHd, (uint64_t)Hkv * kAtHd, kAtTile, 64) ||
-      !make_tmap_bf16_2d(&tmV, V, (uint64_t)total_kv, (uint64_t)Hkv * kAtHd, (uint64_t)Hkv * kAtHd, kAtTile, 64))
+  // K, V [rows][Hkv*hd]: box = 64 columns x 128 keys
+  const uint64_t kv_rows = block_table == nullptr ? (uint64_t)total_kv : (uint64_t)n_pages * kAtTile;
+  if (!make_tmap_bf16_2d(&tmK, K, kv_rows, (uint64_t)Hkv * kAtHd, (uint64_t)Hkv * kAtHd, kAtTile, 64) ||
+      !make_tmap_bf16_2d(&tmV, V, kv_rows, (uint64_t)Hkv * kAtHd, (uint64_t)Hkv * kAtHd, kAtTile, 64))
     return GS_ERR_CUDA;
   if (cudaMemsetAsync(P.tickets, 0, pl.ticket_bytes, st) != cudaSuccess) return GS_ERR_CUDA;
   attn_tc_kernel<<<pl.grid, kAtThreads, kAtSmem, st>>>(tmK, tmV, P);

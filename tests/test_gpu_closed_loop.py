@@ -104,3 +104,30 @@ def test_decaying_steps_run_and_converge():
                               prefix_lo=96, prefix_hi=96, N=8, C=40)
     rep = run_closed_loop(cfg, 60, step_decay=0.6)
     assert rep["step_decay"] == 0.6 and 0.5 < rep["jain"] <= 1.0
+
+
+def test_growing_paged_caches():
+    """Sec. III-A: every round's output tokens join the server's prefix.  The caches live in a page
+    pool (pages handed out in shuffled order as they are needed) and attention reads them through
+    the block table; the oracle gets the same keys and values gathered into its contiguous layout."""
+    cfg = dataclasses.replace(wl.CONFIGS["cfg5"], name="cfg5_grow", d=128, V=4096, Hq=8, Hkv=1, hd=128,
+                              prefix_lo=100, prefix_hi=100, N=6, C=30)
+    seen = {"rounds": 0, "grown": 0}
+
+    def on_round(t, loop, inp, O, logits):
+        lens = (inp["cu_kv"][1:] - inp["cu_kv"][:-1]).cpu().numpy() - (inp["gamma"] + 1)
+        assert np.array_equal(lens, loop.len)
+        if t % 4 == 0:
+            K, V = loop.gather_contiguous(inp)
+            ref = orc.ref_attention(inp["Q"].cpu(), K.cpu(), V.cpu(), inp["cu_q"].cpu(), inp["cu_kv"].cpu())
+            pu.assert_close_rel(O, ref, f"round {t} attention over paged caches")
+        seen["rounds"] += 1
+
+    rep = run_closed_loop(cfg, 40, on_round=on_round, grow=True, max_len=700)
+    assert seen["rounds"] == 40
+    total_out = np.asarray(rep["goodput_per_server"]) * 40
+    final = np.asarray(rep["final_cache_len"])
+    # every cache grew by exactly its output tokens until it hit the cap
+    cap = 700 - (cfg.C + 1)
+    assert np.array_equal(final, np.minimum(100 + np.rint(total_out).astype(np.int64), cap))
+    assert final.max() > 128 * 2          # caches crossed page boundaries

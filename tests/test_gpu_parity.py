@@ -324,6 +324,53 @@ def test_attention_group_sizes(Hq, Hkv):
     pu.assert_close_rel(O, orc.ref_attention(inp["Q"], inp["K"], inp["V"], inp["cu_q"], inp["cu_kv"]), f"G={Hq // Hkv}")
 
 
+@pytest.mark.parametrize("splits", [0, 2], ids=["auto-splits", "two-tile-splits"])
+def test_attention_paged_caches(splits):
+    """gs_verify_attn_paged: the caches scattered over a pool of 128-row pages in shuffled order (with
+    unused pages in between) give what the contiguous layout gives, i.e. the oracle's attention."""
+    cfg = wl.shrink(wl.CONFIGS["cfg2"], prefix_scale=0.3, N=5, name="attn_paged")
+    gamma, prefix = np.array([3, 0, 8, 1, 5]), np.array([700, 90, 1300, 128, 255])
+    inp = wl.make_attention_inputs(cfg, gamma, prefix)
+    cu_kv = inp["cu_kv"].numpy()
+    N = len(gamma)
+    lens = cu_kv[1:] - cu_kv[:-1]
+    pages_of = [(int(l) + 127) // 128 for l in lens]
+    max_pages = max(pages_of) + 2
+    n_pages = sum(pages_of) + 7
+    order = np.random.default_rng(3).permutation(n_pages)
+    table = np.full((N, max_pages), -1, np.int32)            # unused entries are never read
+    K_pool = torch.full((n_pages * 128, cfg.Hkv, cfg.hd), 300.0, dtype=torch.bfloat16)    # stale but finite rows
+    V_pool = torch.full_like(K_pool, -70.0)
+    nxt = 0
+    for i in range(N):
+        for t in range(pages_of[i]):
+            pg = int(order[nxt]); nxt += 1
+            table[i, t] = pg
+            lo = cu_kv[i] + t * 128
+            n = min(128, cu_kv[i + 1] - lo)
+            K_pool[pg * 128: pg * 128 + n] = inp["K"][lo: lo + n]
+            V_pool[pg * 128: pg * 128 + n] = inp["V"][lo: lo + n]
+    # rows of a server's last page beyond its length hold stale values: they are masked by index
+    d = to_dev(inp)
+    Tq, Hq, hd = d["Q"].shape
+    max_len = int(lens.max())
+    B.gs_verify_attn_configure(splits)
+    try:
+        ws = torch.empty(max(256, B.gs_verify_attn_paged_workspace(N, Tq, max_len, Hq, cfg.Hkv, hd, B.GS_BF16)),
+                         dtype=torch.uint8, device=DEV)
+        O = torch.full_like(d["Q"], float("nan"))
+        st = torch.zeros(1, dtype=torch.int32, device=DEV)
+        B.gs_verify_attn_paged(d["Q"], K_pool.to(DEV), V_pool.to(DEV), O, d["cu_q"], d["cu_kv"],
+                               torch.from_numpy(table).to(DEV), max_len, hd ** -0.5, ws, st)
+        torch.cuda.synchronize()
+        O2, _ = run_attn(inp)          # the contiguous layout under the same split plan
+    finally:
+        B.gs_verify_attn_configure(0)
+    assert int(st.item()) == 0
+    pu.assert_close_rel(O, orc.ref_attention(inp["Q"], inp["K"], inp["V"], inp["cu_q"], inp["cu_kv"]), "paged")
+    assert torch.equal(O, O2)          # bit-identical to the contiguous layout (same tiles, same order)
+
+
 def test_attention_many_short_servers():
     """More items per CTA than the kernel caches descriptors for (700 servers x 8 KV heads over 148
     CTAs), most of them a single tile, a few long ones in between."""
