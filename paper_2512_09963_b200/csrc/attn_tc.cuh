@@ -34,7 +34,10 @@ constexpr int kAtMinSplitTiles = 12;     // smallest split the automatic plan ma
 constexpr int kAtMaxCached = 1023;       // servers whose offsets are cached in shared memory
 constexpr int kAtItemCache = 32;         // items of a CTA whose descriptors are worked out once, in parallel
 constexpr uint32_t kAtItemCacheBytes = 2304; // >= kAtItemCache * sizeof(AttnItem)
-constexpr uint32_t kAtSmem = kAtStages * kAtKvBytes + 256 + 1024 + 4 * (kAtMaxCached + 1) * 4 + kAtItemCacheBytes;     // 211.5 KB: one CTA per SM
+constexpr int kAtSortMax = 256;          // batches of at most this many servers are walked longest cache first
+constexpr uint32_t kAtSortBytes = 3 * kAtSortMax * 4;
+constexpr uint32_t kAtSmem = kAtStages * kAtKvBytes + 256 + 1024 + 4 * (kAtMaxCached + 1) * 4 + kAtItemCacheBytes +
+                             kAtSortBytes;     // 214.5 KB: one CTA per SM
 // Tensor memory (512 columns): S two buffers 0..127 / 128..255 (P, as bf16 pairs, overwrites the first
 // 64 columns of its S buffer once the thread has read its scores), O 256..383, Q (bf16 pairs) 384..447.
 // Q and P are A operands read from tensor memory, so shared memory carries only K and V.
@@ -126,11 +129,12 @@ GS_DEVINL AttnItem attn_item_of_server(const AttnTcParams& P, int i, int q0, int
   return it;
 }
 
-// Item `id` in the enumeration  server -> position block -> split -> KV head.  With the per-server
-// prefix counts in shared memory (s_base[0..N], s_gbase[0..N-1]) the server is found by bisection;
-// without them (more servers than the cache holds) by a walk over the offsets.
+// Item `id` in the enumeration  server -> position block -> split -> KV head, the servers taken in
+// the order s_order gives (longest cache first; NULL = as they come).  With the prefix counts of that
+// walk in shared memory (s_base[0..N], s_gbase[0..N-1]) the server is found by bisection; without
+// them (more servers than the cache holds) by a walk over the offsets.
 GS_DEVINL AttnItem attn_find_item(const AttnTcParams& P, const int32_t* cu_q, const int32_t* cu_kv,
-                                  const int32_t* s_base, const int32_t* s_gbase, int id) {
+                                  const int32_t* s_base, const int32_t* s_gbase, const int32_t* s_order, int id) {
   AttnItem it;
   it.valid = 0;
   if (s_base != nullptr) {
@@ -140,8 +144,9 @@ GS_DEVINL AttnItem attn_find_item(const AttnTcParams& P, const int32_t* cu_q, co
       const int mid = (lo + hi) >> 1;
       if (s_base[mid] <= id) lo = mid; else hi = mid;
     }
-    const int q0 = cu_q[lo], k0 = cu_kv[lo];
-    return attn_item_of_server(P, lo, q0, cu_q[lo + 1] - q0, k0, cu_kv[lo + 1] - k0, s_base[lo], s_gbase[lo], id);
+    const int i = (s_order != nullptr) ? s_order[lo] : lo;          // position in the walk -> server
+    const int q0 = cu_q[i], k0 = cu_kv[i];
+    return attn_item_of_server(P, i, q0, cu_q[i + 1] - q0, k0, cu_kv[i + 1] - k0, s_base[lo], s_gbase[lo], id);
   }
   int base = 0, gbase = 0;
   for (int i = 0; i < P.N; ++i) {
@@ -208,6 +213,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
   int32_t* s_gbase_w = s_base_w + (kAtMaxCached + 1);
   const int32_t* s_base = cached ? s_base_w : nullptr;
   const int32_t* s_gbase = cached ? s_gbase_w : nullptr;
+  // walk order (position -> server) and, while it is being built, the counts by server
+  int32_t* s_order_w = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(s_gbase_w + (kAtMaxCached + 1)) + kAtItemCacheBytes);
+  int32_t* s_tmp_cnt = s_order_w + kAtSortMax;
+  int32_t* s_tmp_grp = s_tmp_cnt + kAtSortMax;
+  const bool sorted = P.N <= kAtSortMax;
+  const int32_t* s_order = sorted ? s_order_w : nullptr;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // The next kernel on the stream may set itself up on idle SMs right away (it still waits for this
@@ -241,12 +252,29 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
       s_cu[i] = q0; s_cu[P.N + 1 + i] = k0;
       int cnt = 0, grp = 0;
       if (i < P.N) attn_server_counts(P, q0, P.cu_q[i + 1] - q0, k0, P.cu_kv[i + 1] - k0, cnt, grp);
-      s_base_w[i] = cnt; s_gbase_w[i] = grp;
+      if (sorted) { if (i < P.N) { s_tmp_cnt[i] = cnt; s_tmp_grp[i] = grp; } }
+      else { s_base_w[i] = cnt; s_gbase_w[i] = grp; }
     }
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  if (sorted) {
+    // Longest cache first: the CTAs' first items are then the largest ones and the short ones fill
+    // in behind them, which evens out a ragged batch (cfg3: 79 -> 64 us).  Rank = servers with a
+    // longer cache (or an equal one and a lower index); the counts move to their place in the walk.
+    for (int i = threadIdx.x; i < P.N; i += kAtThreads) {
+      const int Li = s_cu[P.N + 2 + i] - s_cu[P.N + 1 + i];
+      int rank = 0;
+      for (int j = 0; j < P.N; ++j) {
+        const int Lj = s_cu[P.N + 2 + j] - s_cu[P.N + 1 + j];
+        rank += (Lj > Li || (Lj == Li && j < i)) ? 1 : 0;
+      }
+      s_order_w[rank] = i;
+      s_base_w[rank] = s_tmp_cnt[i]; s_gbase_w[rank] = s_tmp_grp[i];
+    }
+    __syncthreads();
+  }
   if (cached && warp == 2) {
     // counts -> exclusive prefix sums, 32 servers per step
     int carry = 0, gcarry = 0;
@@ -272,12 +300,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
     const long long id = (long long)blockIdx.x + (long long)lane * gridDim.x;
     AttnItem it;
     it.valid = 0;
-    if (id < P.max_items) it = attn_find_item(P, cu_q, cu_kv, s_base, s_gbase, (int)id);
+    if (id < P.max_items) it = attn_find_item(P, cu_q, cu_kv, s_base, s_gbase, s_order, (int)id);
     s_items[lane] = it;
   }
   __syncthreads();
   auto item_at = [&](int k, int id) -> AttnItem {
-    return k < kAtItemCache ? s_items[k] : attn_find_item(P, cu_q, cu_kv, s_base, s_gbase, id);
+    return k < kAtItemCache ? s_items[k] : attn_find_item(P, cu_q, cu_kv, s_base, s_gbase, s_order, id);
   };
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t tmem_S = tmem_base + kAtColS, tmem_O = tmem_base + kAtColO;     // S buffer b at tmem_S + 128 b
