@@ -463,6 +463,46 @@ def run_ours(args, cfg, rank, world, local_rank):
     print(json.dumps(line), flush=True)
 
 
+def run_head_sweep(args, cfg, local_rank):
+    """LM head alone over a range of row counts at the workload's d and V: where it is bound by HBM
+    (few rows) and where by the tensor pipe (many rows), against the measured peaks of both."""
+    from paper_2512_09963_b200 import binding as B
+    from paper_2512_09963_b200 import build as gs_build
+    gs_build.build()
+    B.lib()
+    dev = torch.device("cuda", local_rank)
+    peak_hbm, kind, peaks = _peaks()
+    tf_burst = float(peaks.get("bf16_tflops", 1590.0))
+    tf_sust = float(peaks.get("bf16_tflops_sustained", 1400.0))
+    W = wl.make_layer(cfg, dev)["W"]
+    d, V = cfg.d, cfg.V
+    rows_out = []
+    for T in (16, 46, 96, 144, 256, 288, 512, 1024, 2048):
+        H = wl.make_hidden(cfg, T, 0, dev)
+        logits = torch.empty((T, V), dtype=torch.float32, device=dev)
+        ws = torch.empty(max(256, B.gs_lm_head_workspace(T, d, V, B.GS_BF16)), dtype=torch.uint8, device=dev)
+        for _ in range(3):
+            B.gs_lm_head_logits(H, W, logits, ws)
+        n = 20
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(n):                       # W (1.5 GB) streams through L2 every launch: inputs are cold
+            B.gs_lm_head_logits(H, W, logits, ws)
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / n
+        by = d * V * 2 + T * V * 4 + T * d * 2
+        fl = 2.0 * T * d * V
+        gbs, tfs = by / us / 1e3, fl / us / 1e6
+        rows_out.append({"rows": T, "us": us, "GBps": gbs, "frac_hbm": gbs / peak_hbm, "TFLOPs": tfs,
+                         "frac_bf16_burst": tfs / tf_burst, "frac_bf16_sustained": tfs / tf_sust,
+                         "bound": "hbm" if by / peak_hbm / 1e3 > fl / tf_burst / 1e6 else "tensor"})
+        del H, logits, ws
+    print(json.dumps({"head_sweep": rows_out, "d": d, "V": V, "peaks": {"hbm_gbs": peak_hbm, "bf16_tflops": tf_burst,
+                                                                      "bf16_tflops_sustained": tf_sust, "source": kind}}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -474,6 +514,8 @@ def main():
     ap.add_argument("--rounds", type=int, default=1000, help="rounds of the closed loop (--config cfg5)")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--head-sweep", action="store_true",
+                    help="time gs_lm_head_logits alone for 16..2048 rows at the workload's d and V")
     ap.add_argument("--no-dependent-launch", action="store_true",
                     help="launch the kernels without the programmatic-dependent-launch attribute")
     ap.add_argument("--profile-small", action="store_true",
@@ -496,6 +538,10 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
     torch.cuda.set_device(local_rank)
+    if args.head_sweep:
+        if rank == 0:
+            run_head_sweep(args, cfg, local_rank)
+        return
     if args.config == "cfg5":
         # closed-loop scheduling: Algorithm 1 for --rounds rounds with gs_schedule in the loop
         if rank == 0:
