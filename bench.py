@@ -38,8 +38,8 @@ ETA, BETA = 0.1, 0.5
 # per launch), keyed by the sha256 of the kernel source it was taken on; a changed kernel reports null.
 # cfg2's full launch is within ncu's single-pass size rule only for the launch list, so the counters
 # were taken on a smaller vocabulary and scale with the units processed (see profiles/).
-# small case (V = 32768): 336.072 MB read + 4.417 MB written per launch, times 151936/32768
-NCU_TRAFFIC = {"5d714646504583d3": {"cfg2": 1578749171}}
+# small case (V = 32768): 336.067 MB read + 3.770 MB written per launch, times 151936/32768
+NCU_TRAFFIC = {"26b8c6888d7758e0": {"cfg2": 1575730630}}
 
 
 def _kernel_hash():
@@ -226,10 +226,41 @@ def run_ours(args, cfg, rank, world, local_rank):
         rnd.alpha_hat.fill_(0.5)
         rnd.X.fill_(1.0)
 
+    # Does this shape have the LM head that writes the softmax statistics in its epilogue (then the
+    # acceptance step does not read the logits a second time)?
+    # Measured on B200: the statistics cost the LM head 4-5 us (they sit in the epilogue of its last,
+    # not overlapped, tile) and save the acceptance step its pass over T_q x V logits; that pays from
+    # about 64 verify positions on (cfg4: -2.7 % per step, cfg2 with 46 positions: +0.4 %).
+    fused = False
+    if not args.no_fused_stats and (Tq >= 64 or args.fused_stats):
+        fused = rnd.head_accept_fused(inp["H"], inp["W"], inp["q_probs"], inp["draft_tok"], inp["cu_q"],
+                                      inp["u_accept"], inp["u_sample"], inp["tau"], update=False)
+        torch.cuda.synchronize()
+    n_chunk_fused = None
+
+    def head_call():
+        nonlocal n_chunk_fused
+        if fused:
+            n_chunk_fused = B.gs_lm_head_logits_stats(inp["H"], inp["W"], rnd.logits, inp["tau"], rnd.stats, rnd.ws_head,
+                                                      rnd.d_status)
+        else:
+            rnd.head(inp["H"], inp["W"])
+
+    def accept_call():
+        if fused:
+            ok = B.gs_spec_accept_prestats(rnd.logits, inp["q_probs"], inp["draft_tok"], inp["cu_q"], inp["u_accept"],
+                                           inp["u_sample"], inp["tau"], rnd.accepted, rnd.out_tok, rnd.n_out, rnd.ratio,
+                                           rnd.p_tok, rnd.stats, n_chunk_fused, rnd.margin, rnd.alpha_hat, rnd.X,
+                                           rnd.eta, rnd.beta, rnd.alpha_min, rnd.alpha_max, ws=rnd.ws_acc,
+                                           d_status=rnd.d_status)
+            assert ok
+        else:
+            rnd.accept(inp["q_probs"], inp["draft_tok"], inp["cu_q"], inp["u_accept"], inp["u_sample"], inp["tau"])
+
     def step():
         rnd.attn(inp["Q"], inp["K"], inp["V"], inp["cu_q"], inp["cu_kv"])
-        rnd.head(inp["H"], inp["W"])
-        rnd.accept(inp["q_probs"], inp["draft_tok"], inp["cu_q"], inp["u_accept"], inp["u_sample"], inp["tau"])
+        head_call()
+        accept_call()
         if world == 1:
             rnd.schedule(s_min, s_max)
         else:
@@ -303,9 +334,8 @@ def run_ours(args, cfg, rank, world, local_rank):
     names = ("verify_attn", "lm_head_logits", "spec_accept", "gs_schedule")
     calls = {
         "verify_attn": lambda: rnd.attn(inp["Q"], inp["K"], inp["V"], inp["cu_q"], inp["cu_kv"]),
-        "lm_head_logits": lambda: rnd.head(inp["H"], inp["W"]),
-        "spec_accept": lambda: rnd.accept(inp["q_probs"], inp["draft_tok"], inp["cu_q"], inp["u_accept"],
-                                          inp["u_sample"], inp["tau"]),
+        "lm_head_logits": head_call,
+        "spec_accept": accept_call,
         "gs_schedule": lambda: rnd.schedule(s_min[:N], s_max[:N]),
     }
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(n_k)]
@@ -364,7 +394,8 @@ def run_ours(args, cfg, rank, world, local_rank):
     total_kv = int(inp["K"].shape[0])
     bytes_head = d * V * es + Tq * V * 4 + Tq * d * es
     bytes_attn = 2 * total_kv * cfg.Hkv * cfg.hd * es + 2 * Tq * cfg.Hq * cfg.hd * es
-    bytes_acc = Tq * V * 4 + N * V * 8
+    # with the statistics from the LM head's epilogue the pass over all logits is gone
+    bytes_acc = N * V * 8 if fused else Tq * V * 4 + N * V * 8
     flops_head = 2.0 * Tq * d * V
     ach = bytes_head / (k_us["lm_head_logits"] * 1e-6) / 1e9
     khash = _kernel_hash()
@@ -454,7 +485,9 @@ def run_ours(args, cfg, rank, world, local_rank):
                    "prefix": int(inp["prefix"][0]), "d": d, "V": V, "heads": f"{cfg.Hq}q/{cfg.Hkv}kv x {cfg.hd}",
                    "temperature": float(inp["tau"]), "parallelism": f"dp{world} over draft servers",
                    "l2": "inputs larger than L2: the 1.56 GB head weight streams through L2 every step and evicts the KV cache and logits",
-                   "launch": "CUDA graph replay of the four calls" if graph is not None else "eager, four calls per step"},
+                   "launch": "CUDA graph replay of the four calls" if graph is not None else "eager, four calls per step",
+                   "softmax_statistics": "LM-head epilogue (gs_lm_head_logits_stats + gs_spec_accept_prestats)" if fused
+                   else "statistics pass of gs_spec_accept"},
         "goodput_tokens_per_s": goodput,
         "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu, "e2e": e2e,
         "gpu_launches": int(launches_per_step) * args.steps, "launches_per_step": int(launches_per_step),
@@ -514,6 +547,10 @@ def main():
     ap.add_argument("--rounds", type=int, default=1000, help="rounds of the closed loop (--config cfg5)")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--fused-stats", action="store_true",
+                    help="softmax statistics from the LM head's epilogue even below 64 verify positions")
+    ap.add_argument("--no-fused-stats", action="store_true",
+                    help="plain gs_lm_head_logits + gs_spec_accept even where the LM head could write the softmax statistics")
     ap.add_argument("--head-sweep", action="store_true",
                     help="time gs_lm_head_logits alone for 16..2048 rows at the workload's d and V")
     ap.add_argument("--no-dependent-launch", action="store_true",

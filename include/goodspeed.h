@@ -203,6 +203,40 @@ gs_status gs_spec_accept(const float* logits, const float* q_probs, const int32_
                          void* ws, size_t ws_bytes, int32_t* d_status, void* stream);
 
 /* --------------------------------------------------------------------------------------------
+ * gs_lm_head_logits_stats + gs_spec_accept_prestats -- Sec. II-A1 and II-A2 as one computation:
+ * P_M = softmax(W h) needs, per verify position, the maximum and the sum of exponentials of the
+ * logits.  gs_spec_accept obtains them by reading every logit once more; here the LM head's epilogue
+ * writes them while it still holds the logits in tensor memory, and the acceptance step starts from
+ * them.
+ *
+ * gs_lm_head_logits_stats: arguments and results as gs_lm_head_logits, plus
+ *   temperature   the softmax temperature the statistics are for (0 = greedy: maxima only)
+ *   stats         device buffer of gs_lm_head_stats_bytes(T) bytes, 16-byte aligned; receives
+ *                 *n_chunk entries per row (one per CTA of the launch; opaque)
+ *   n_chunk       host int, written before the call returns
+ *   bf16 on CTA pairs with T <= 256 only; every other case returns GS_ERR_UNSUPPORTED and launches
+ *   nothing (call gs_lm_head_logits and gs_spec_accept instead).
+ * gs_spec_accept_prestats: arguments and results as gs_spec_accept (same temperature!), plus the
+ *   stats buffer and n_chunk.  Needs V % 4 == 0, 16-byte aligned rows and a vocabulary slice that
+ *   fits shared memory (the cluster kernel); otherwise GS_ERR_UNSUPPORTED and nothing is launched.
+ * Accept decisions and probabilities agree with gs_spec_accept to rounding (the sums of
+ * exponentials are grouped differently).
+ */
+size_t gs_lm_head_stats_bytes(int T);
+gs_status gs_lm_head_logits_stats(const void* H, const void* W, float* logits, int T, int d, int V,
+                                  gs_dtype dt, float temperature, void* stats, size_t stats_bytes,
+                                  int* n_chunk, void* ws, size_t ws_bytes, int32_t* d_status, void* stream);
+gs_status gs_spec_accept_prestats(const float* logits, const float* q_probs, const int32_t* draft_tok,
+                                  const int32_t* cu_q, const float* u_accept, const float* u_sample,
+                                  float temperature, int N, int Tq, int V,
+                                  int32_t* accepted, int32_t* out_tok, int32_t* n_out,
+                                  float* ratio, float* p_tok, float* margin,
+                                  double* alpha_hat, double* X, double eta, double beta,
+                                  double alpha_min, double alpha_max,
+                                  const void* stats, int n_chunk,
+                                  void* ws, size_t ws_bytes, int32_t* d_status, void* stream);
+
+/* --------------------------------------------------------------------------------------------
  * gs_spec_accept_static -- no counterpart in the paper: a convenience of this library.
  *
  * The same computation, arguments and results as gs_spec_accept, for callers that cannot provide

@@ -44,6 +44,12 @@ SIGNATURES = {
     "gs_spec_accept": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _f, _i, _i, _i,
                             _vp, _vp, _vp, _vp, _vp, _vp,
                             _vp, _vp, _d, _d, _d, _d, _vp, _sz, _vp, _vp]),
+    "gs_spec_accept_prestats": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _f, _i, _i, _i,
+                                     _vp, _vp, _vp, _vp, _vp, _vp,
+                                     _vp, _vp, _d, _d, _d, _d, _vp, _i, _vp, _sz, _vp, _vp]),
+    "gs_lm_head_stats_bytes": (_sz, [_i]),
+    "gs_lm_head_logits_stats": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _f, _vp, _sz, C.POINTER(C.c_int),
+                                     _vp, _sz, _vp, _vp]),
     "gs_spec_accept_static_capacity": (_sz, []),
     "gs_spec_accept_static": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _f, _i, _i, _i,
                                    _vp, _vp, _vp, _vp, _vp, _vp,
@@ -194,6 +200,53 @@ def gs_lm_head_logits(H, W, logits, ws, d_status=None):
                                    _ptr(ws), ws.numel() * ws.element_size(),
                                    _ptr(d_status, torch.int32), _stream())
     _check("gs_lm_head_logits", code)
+
+
+GS_ERR_UNSUPPORTED = 3
+
+
+def gs_lm_head_stats_bytes(T) -> int:
+    return lib().gs_lm_head_stats_bytes(int(T))
+
+
+def gs_lm_head_logits_stats(H, W, logits, temperature, stats, ws, d_status=None):
+    """LM head that also writes the rows' softmax statistics.  Returns the number of statistics
+    entries per row, or None if this shape has no such kernel (nothing was launched then)."""
+    T, d = H.shape
+    V = W.shape[1]
+    if W.shape[0] != d or tuple(logits.shape) != (T, V):
+        raise ValueError("shape mismatch")
+    n_chunk = C.c_int(0)
+    code = lib().gs_lm_head_logits_stats(_ptr(H), _ptr(W, H.dtype), _ptr(logits, torch.float32), T, d, V, _dt(H),
+                                         float(temperature), _ptr(stats), stats.numel() * stats.element_size(),
+                                         C.byref(n_chunk), _ptr(ws), ws.numel() * ws.element_size(),
+                                         _ptr(d_status, torch.int32), _stream())
+    if code == GS_ERR_UNSUPPORTED:
+        return None
+    _check("gs_lm_head_logits_stats", code)
+    return int(n_chunk.value)
+
+
+def gs_spec_accept_prestats(logits, q_probs, draft_tok, cu_q, u_accept, u_sample, temperature,
+                            accepted, out_tok, n_out, ratio, p_tok, stats, n_chunk, margin=None,
+                            alpha_hat=None, X=None, eta=0.0, beta=0.0, alpha_min=1e-3, alpha_max=0.999,
+                            ws=None, d_status=None) -> bool:
+    """Acceptance step on statistics from gs_lm_head_logits_stats.  False (nothing launched) if the
+    shape needs the plain gs_spec_accept."""
+    Tq, V = logits.shape
+    N = cu_q.numel() - 1
+    f32, i32, f64 = torch.float32, torch.int32, torch.float64
+    code = lib().gs_spec_accept_prestats(
+        _ptr(logits, f32), _ptr(q_probs, f32), _ptr(draft_tok, i32), _ptr(cu_q, i32),
+        _ptr(u_accept, f32), _ptr(u_sample, f32), float(temperature), N, Tq, V,
+        _ptr(accepted, i32), _ptr(out_tok, i32), _ptr(n_out, i32), _ptr(ratio, f32), _ptr(p_tok, f32),
+        _ptr(margin, f32), _ptr(alpha_hat, f64), _ptr(X, f64), float(eta), float(beta),
+        float(alpha_min), float(alpha_max), _ptr(stats), int(n_chunk),
+        _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(), _ptr(d_status, i32), _stream())
+    if code == GS_ERR_UNSUPPORTED:
+        return False
+    _check("gs_spec_accept_prestats", code)
+    return True
 
 
 def gs_spec_accept_workspace(N, Tq, V) -> int:

@@ -15,6 +15,15 @@ namespace gs {
 
 constexpr int kNumSMsFallback = 148;
 
+// Softmax statistics of one row over one stretch of the vocabulary: maximum, its lowest index, and
+// the sum of 2^((l - m) * log2(e)/tau).  Written by the statistics pass of gs_spec_accept or by the
+// LM-head epilogue, merged by the acceptance pass.
+struct ChunkStat {   // 16 bytes
+  float m;
+  int arg;
+  double z;
+};
+
 // Sticky device status: the first non-zero code wins.
 GS_DEVINL void set_status(int32_t* st, int code) {
   if (st != nullptr) atomicCAS(st, 0, code);

@@ -455,3 +455,32 @@ extern "C" gs_status gs_lm_head_logits(const void* H, const void* W, float* logi
   }
   return launch_lm_head_tc(H, W, logits, T, d, V, d_status, st);
 }
+
+// ------------------------------------------------------------------------------------------------
+// gs_lm_head_logits_stats: the same product, with the softmax statistics of every row (maximum, its
+// lowest index, sum of exponentials at the given temperature, per CTA of the launch) written next to
+// the logits by the epilogue.  gs_spec_accept_prestats consumes them, so the acceptance step does
+// not have to read every logit once more (Sec. II-A1 and II-A2 are adjacent steps of one computation).
+extern "C" size_t gs_lm_head_stats_bytes(int T) {
+  if (T <= 0) return 256;
+  return gs::align_up((size_t)T * (size_t)gs::sm_count() * sizeof(gs::ChunkStat), 256);
+}
+
+extern "C" gs_status gs_lm_head_logits_stats(const void* H, const void* W, float* logits, int T, int d, int V,
+                                             gs_dtype dt, float temperature, void* stats, size_t stats_bytes,
+                                             int* n_chunk, void* ws, size_t ws_bytes, int32_t* d_status,
+                                             void* stream) {
+  using namespace gs;
+  if (T < 0 || d < 0 || V < 0 || !(temperature >= 0.f)) return GS_ERR_INVALID_ARG;
+  if (dt != GS_F32 && dt != GS_BF16) return GS_ERR_INVALID_ARG;
+  if (!H || !W || !logits || !stats || !n_chunk) return GS_ERR_INVALID_ARG;
+  if (T == 0 || V == 0) return GS_ERR_UNSUPPORTED;
+  if (ws == nullptr || ws_bytes < gs_lm_head_workspace(T, d, V, dt)) return GS_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(stats) & 15u) != 0 || stats_bytes < gs_lm_head_stats_bytes(T)) return GS_ERR_WORKSPACE;
+  const bool tma_ok = dt == GS_BF16 && d > 0 && (d % 8 == 0) && (V % 8 == 0) && (reinterpret_cast<uintptr_t>(H) % 16 == 0) &&
+                      (reinterpret_cast<uintptr_t>(W) % 16 == 0);
+  if (!tma_ok || g_head_variant == 1) return GS_ERR_UNSUPPORTED;
+  const float k2 = temperature > 0.f ? 1.4426950408889634f / temperature : 0.f;
+  return launch_lm_head_pair(H, W, logits, T, d, V, d_status, g_head_mt, g_head_stages,
+                             static_cast<cudaStream_t>(stream), static_cast<ChunkStat*>(stats), k2, sm_count(), n_chunk);
+}

@@ -25,8 +25,13 @@ constexpr uint32_t kPairWUnitBytes = 2u * kPairBlockK * 128u;   // one CTA's W s
 constexpr uint32_t kPairMaxSmem = 232448;
 constexpr int kPairMaxUnits = 4;            // widest tile, in units
 
+constexpr int kPairStatRows = 256;          // most rows the epilogue keeps softmax statistics for
+constexpr uint32_t kPairStatBytes = 4u * kPairStatRows * 12u;   // per epilogue warp and row: maximum, its index, sum
+
 struct HeadPairParams {
   float* logits;
+  ChunkStat* stats;      // STATS kernels: [T][gridDim.x], one entry per row and CTA
+  float k2;              // log2(e) / temperature (0 = greedy: maxima only)
   int32_t* d_status;
   int T, d, V;
   int row0;              // first row of H / logits this launch covers
@@ -63,8 +68,21 @@ GS_DEVINL void head_pair_issue(uint32_t d_acc, uint32_t a_hi, uint32_t a_lo_stag
   }
 }
 
+// Floats to unsigned keys that order the same way (0 is below every key of a real number).
+GS_DEVINL uint32_t float_key(float x) {
+  const uint32_t u = __float_as_uint(x);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+GS_DEVINL float key_float(uint32_t k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
 // NT = MMAs along the rows per unit; compile-time so that the issue loop unrolls completely.
-template <int NT>
+// STATS: the epilogue also keeps, per row, the softmax statistics of the logits it writes (what the
+// acceptance pass would otherwise obtain by reading every logit again): a warp reduces the 32
+// columns it holds for 16 rows at a time, one lane per row folds the result into a running entry in
+// shared memory, and at the end of the kernel the CTA's four warps are merged into one entry per row.
+template <int NT, bool STATS = false>
 __global__ void __launch_bounds__(kPairThreads, 1)
 lm_head_pair_kernel(const __grid_constant__ CUtensorMap tmapW, const __grid_constant__ CUtensorMap tmapH,
                     const HeadPairParams P) {
@@ -81,9 +99,16 @@ lm_head_pair_kernel(const __grid_constant__ CUtensorMap tmapW, const __grid_cons
   uint8_t* tail = sm + (bars - base) + 8u * (uint32_t)(2 * S + 4);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 4);
+  // running statistics: [4 epilogue warps][kPairStatRows] maxima, indices, sums
+  float* st_m = reinterpret_cast<float*>(tail + 64);
+  int* st_a = reinterpret_cast<int*>(st_m + 4 * kPairStatRows);
+  float* st_z = reinterpret_cast<float*>(st_a + 4 * kPairStatRows);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_cta_rank();                // 0 = even CTA (issues the MMAs)
+  if (STATS) {
+    for (int i = threadIdx.x; i < 4 * kPairStatRows; i += kPairThreads) { st_m[i] = -INFINITY; st_a[i] = INT_MAX; st_z[i] = 0.f; }
+  }
   const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
   if (threadIdx.x == 0) {
     for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -225,6 +250,65 @@ lm_head_pair_kernel(const __grid_constant__ CUtensorMap tmapW, const __grid_cons
               for (int c = 0; c < 16; ++c)
                 if (t_first + c < P.T) out[(size_t)c * P.V] = __uint_as_float(r[c]);
             }
+            if (STATS) {
+              // 16 rows x this warp's 32 columns: row maxima by integer reduction on order-preserving
+              // keys, lowest column at the maximum by ballot, sums of exponentials by a halving
+              // exchange that leaves row c's sum in lanes 2c and 2c+1.
+              const bool valid = v < P.V;
+              const int c_me = (lane >> 1) & 15;
+              float e[16];
+              float m_me = -INFINITY;
+              int a_me = INT_MAX;
+              if (P.k2 > 0.f) {
+                // The lane sits in the key's five lowest bits, so one integer reduction yields the row
+                // maximum (to 2^-18 relative, from below: all that a reference for the exponentials
+                // has to be, as long as every sum uses the same one) and its lowest column.  A vote
+                // per row, which the exact index would need, costs more than everything else here.
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                  const float x = __uint_as_float(r[c]);
+                  const uint32_t key = valid ? ((float_key(x) & ~31u) | (uint32_t)(31 - lane)) : 0u;
+                  const uint32_t mk = __reduce_max_sync(0xffffffffu, key);
+                  const float mx = (mk == 0u) ? -INFINITY : key_float(mk & ~31u);
+                  e[c] = (valid && mx > -INFINITY) ? fast_exp2((x - mx) * P.k2) : 0.f;
+                  if (c == c_me) { m_me = mx; a_me = mk ? (v - lane) + (31 - (int)(mk & 31u)) : INT_MAX; }
+                }
+              } else {
+                // greedy: the exact maximum and its lowest index, no sums
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                  const float x = __uint_as_float(r[c]);
+                  const uint32_t key = valid ? float_key(x) : 0u;
+                  const uint32_t mk = __reduce_max_sync(0xffffffffu, key);
+                  const uint32_t at = __ballot_sync(0xffffffffu, valid && key == mk);
+                  e[c] = 0.f;
+                  if (c == c_me) { m_me = (mk == 0u) ? -INFINITY : key_float(mk); a_me = at ? (v - lane) + (__ffs(at) - 1) : INT_MAX; }
+                }
+              }
+#pragma unroll
+              for (int h = 8; h >= 1; h >>= 1) {           // lanes with bit (2h) set keep the upper half
+                const bool up = (lane & (2 * h)) != 0;
+#pragma unroll
+                for (int i = 0; i < h; ++i) {
+                  const float send = up ? e[i] : e[i + h];
+                  const float keep = up ? e[i + h] : e[i];
+                  e[i] = keep + __shfl_xor_sync(0xffffffffu, send, 2 * h);
+                }
+              }
+              const float z_me = e[0] + __shfl_xor_sync(0xffffffffu, e[0], 1);
+              const int row = t_first + c_me;
+              if ((lane & 1) == 0 && row < P.T) {
+                const int slot = q * kPairStatRows + row;
+                const float m0 = st_m[slot];
+                if (m_me > -INFINITY) {
+                  const float mn = fmaxf(m0, m_me);
+                  const float z0 = (m0 > -INFINITY) ? st_z[slot] * fast_exp2((m0 - mn) * P.k2) : 0.f;
+                  st_z[slot] = z0 + z_me * fast_exp2((m_me - mn) * P.k2);
+                  if (m_me > m0 || (m_me == m0 && a_me < st_a[slot])) st_a[slot] = a_me;
+                  st_m[slot] = mn;
+                }
+              }
+            }
           }
         }
       }
@@ -238,6 +322,23 @@ lm_head_pair_kernel(const __grid_constant__ CUtensorMap tmapW, const __grid_cons
   __syncthreads();
   cluster_sync_all();
   if (threadIdx.x == 0 && *abort_flag) set_status(P.d_status, GS_ERR_TIMEOUT);
+  if (STATS) {
+    // one entry per row for this CTA: its four warps in order (lowest index wins ties)
+    for (int row = threadIdx.x; row < P.T; row += kPairThreads) {
+      float M = -INFINITY; int arg = INT_MAX;
+#pragma unroll
+      for (int w = 0; w < 4; ++w) argmax_merge(M, arg, st_m[w * kPairStatRows + row], st_a[w * kPairStatRows + row]);
+      double z = 0.0;
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {
+        const float mw = st_m[w * kPairStatRows + row];
+        if (mw > -INFINITY) z += (double)st_z[w * kPairStatRows + row] * (double)fast_exp2((mw - M) * P.k2);
+      }
+      ChunkStat cs;
+      cs.m = M; cs.arg = arg; cs.z = z;
+      P.stats[(size_t)(P.row0 + row) * gridDim.x + blockIdx.x] = cs;
+    }
+  }
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc_pair(tmem_base, P.tmem_cols);
@@ -269,7 +370,8 @@ inline int head_pair_max_clusters(K kernel, size_t smem) {
 }
 
 // Plan for `rows` rows (at most 512) starting at row0.  max_units caps the tile width (0 = widest).
-inline HeadPairPlan head_pair_plan(int rows, int row0, int d, int V, int clusters_avail, int max_units, int max_stages) {
+inline HeadPairPlan head_pair_plan(int rows, int row0, int d, int V, int clusters_avail, int max_units, int max_stages,
+                                   uint32_t reserve = 0) {
   HeadPairPlan pl;
   pl.ok = false;
   HeadPairParams& P = pl.P;
@@ -284,7 +386,7 @@ inline HeadPairPlan head_pair_plan(int rows, int row0, int d, int V, int cluster
   if (max_mt < 1 || clusters_avail < 1) return pl;
   P.h_bytes = (uint32_t)(P.nt * (P.n_tile / 2)) * 128u;
   // widest tile that still leaves a ring of three stages
-  while (max_mt > 1 && 1024u + 3u * ((uint32_t)max_mt * kPairWUnitBytes + P.h_bytes) + 1024u > kPairMaxSmem) --max_mt;
+  while (max_mt > 1 && 1024u + 3u * ((uint32_t)max_mt * kPairWUnitBytes + P.h_bytes) + 1024u + reserve > kPairMaxSmem) --max_mt;
   const int units = (V + (int)kPairUnit - 1) / (int)kPairUnit;
   const int per_cluster = (units + clusters_avail - 1) / clusters_avail;
   const int tiles_per_cluster = (per_cluster + max_mt - 1) / max_mt;
@@ -298,25 +400,29 @@ inline HeadPairPlan head_pair_plan(int rows, int row0, int d, int V, int cluster
   while (cols < (uint32_t)P.n_acc * P.acc_cols) cols <<= 1;
   P.tmem_cols = cols;
   P.stage_bytes = (uint32_t)mt * kPairWUnitBytes + P.h_bytes;
-  int stages = (int)((kPairMaxSmem - 1024u - 1024u) / P.stage_bytes);
+  int stages = (int)((kPairMaxSmem - 1024u - 1024u - reserve) / P.stage_bytes);
   if (stages > 16) stages = 16;
   if (max_stages > 0 && max_stages < stages) stages = max_stages;
   if (stages < 2) return pl;
   P.stages = stages;
   P.k_blocks = (d + (int)kPairBlockK - 1) / (int)kPairBlockK;
-  pl.smem = 1024u + (size_t)stages * P.stage_bytes + 8u * (2u * (uint32_t)stages + 4u) + 64u;
+  pl.smem = 1024u + (size_t)stages * P.stage_bytes + 8u * (2u * (uint32_t)stages + 4u) + 64u + reserve;
   pl.clusters = min(P.num_tiles, clusters_avail);
   pl.ok = true;
   return pl;
 }
 
+// stats != NULL: the kernel variant that also writes per-row softmax statistics, [T][*n_chunk] entries
+// (one MMA along the rows only, i.e. T <= 256; otherwise GS_ERR_UNSUPPORTED and nothing is launched).
 inline gs_status launch_lm_head_pair(const void* H, const void* W, float* logits, int T, int d, int V,
-                                     int32_t* d_status, int max_units, int max_stages, cudaStream_t st) {
+                                     int32_t* d_status, int max_units, int max_stages, cudaStream_t st,
+                                     ChunkStat* stats = nullptr, float k2 = 0.f, int max_chunks = 0, int* n_chunk = nullptr) {
   using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const HeadPairParams);
-  static const KernelFn kernels[2] = {lm_head_pair_kernel<1>, lm_head_pair_kernel<2>};
+  static const KernelFn kernels[3] = {lm_head_pair_kernel<1>, lm_head_pair_kernel<2>, lm_head_pair_kernel<1, true>};
+  if (stats != nullptr && T > kPairStatRows) return GS_ERR_UNSUPPORTED;
   static int clusters_avail = -1;
   if (clusters_avail < 0) {
-    for (int a = 0; a < 2; ++a) {
+    for (int a = 0; a < 3; ++a) {
       if (cudaFuncSetAttribute(kernels[a], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairMaxSmem) != cudaSuccess)
         return GS_ERR_CUDA;
       if (cudaFuncSetAttribute(kernels[a], cudaFuncAttributeNonPortableClusterSizeAllowed, 0) != cudaSuccess)
@@ -327,9 +433,12 @@ inline gs_status launch_lm_head_pair(const void* H, const void* W, float* logits
   }
   for (int row0 = 0; row0 < T; row0 += 512) {
     const int rows = min(512, T - row0);
-    HeadPairPlan pl = head_pair_plan(rows, row0, d, V, clusters_avail, max_units, max_stages);
+    HeadPairPlan pl = head_pair_plan(rows, row0, d, V, clusters_avail, max_units, max_stages,
+                                     stats != nullptr ? kPairStatBytes : 0u);
     if (!pl.ok) return GS_ERR_UNSUPPORTED;
-    pl.P.logits = logits; pl.P.d_status = d_status;
+    if (stats != nullptr && (pl.P.nt != 1 || 2 * pl.clusters > max_chunks)) return GS_ERR_UNSUPPORTED;
+    pl.P.logits = logits; pl.P.d_status = d_status; pl.P.stats = stats; pl.P.k2 = k2;
+    if (n_chunk != nullptr) *n_chunk = 2 * pl.clusters;
     CUtensorMap tmapW, tmapH;
     if (!make_tmap_bf16_2d(&tmapW, W, (uint64_t)d, (uint64_t)V, (uint64_t)V, kPairBlockK, 64)) return GS_ERR_CUDA;
     if (!make_tmap_bf16_2d(&tmapH, H, (uint64_t)T, (uint64_t)d, (uint64_t)d, (uint32_t)(pl.P.n_tile / 2), 64))
@@ -345,7 +454,7 @@ inline gs_status launch_lm_head_pair(const void* H, const void* W, float* logits
     at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at; cfg.numAttrs = dependent_launch_enabled() ? 2 : 1;
-    if (cudaLaunchKernelEx(&cfg, kernels[pl.P.nt - 1], tmapW, tmapH, pl.P) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, kernels[stats != nullptr ? 2 : pl.P.nt - 1], tmapW, tmapH, pl.P) != cudaSuccess) {
       (void)cudaGetLastError();
       return GS_ERR_CUDA;
     }

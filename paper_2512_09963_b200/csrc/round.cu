@@ -12,8 +12,8 @@ namespace gs {
 struct RoundLayout {
   size_t Q, H, q_probs, draft_tok, u_accept, u_sample, cu_q, cu_kv;     // staged inputs
   size_t O, logits, accepted, out_tok, n_out, ratio, p_tok, S_next, status;
-  size_t ws_attn, ws_head, ws_acc;
-  size_t ws_attn_bytes, ws_head_bytes, ws_acc_bytes;
+  size_t ws_attn, ws_head, ws_acc, stats;
+  size_t ws_attn_bytes, ws_head_bytes, ws_acc_bytes, stats_bytes;
   size_t total;
 };
 
@@ -47,6 +47,8 @@ static RoundLayout round_layout(const gs_round_desc& r) {
   L.ws_attn = take(L.ws_attn_bytes);
   L.ws_head = take(L.ws_head_bytes);
   L.ws_acc = take(L.ws_acc_bytes);
+  L.stats_bytes = gs_lm_head_stats_bytes(r.Tq);
+  L.stats = take(L.stats_bytes);
   L.total = off;
   return L;
 }
@@ -137,18 +139,40 @@ extern "C" gs_status gs_verify_round_host(const gs_round_desc* r,
   gs_status s = gs_verify_attn(w + L.Q, d_K, d_V, w + L.O, cu_q, cu_kv, r->N, r->Tq, r->total_kv, r->max_kv_len,
                                r->Hq, r->Hkv, r->hd, r->scale, r->dt, w + L.ws_attn, L.ws_attn_bytes, d_status, st);
   if (s != GS_OK) return s;
-  s = gs_lm_head_logits(w + L.H, d_W, reinterpret_cast<float*>(w + L.logits), r->Tq, r->d, r->V, r->dt,
-                        w + L.ws_head, L.ws_head_bytes, d_status, st);
+  // LM head with the softmax statistics in its epilogue where the shape has that kernel, so that the
+  // acceptance step does not read the logits a second time; the plain pair of calls otherwise.
+  // (Below about 64 verify positions the statistics cost the LM head as much as they save.)
+  int n_chunk = 0;
+  s = GS_ERR_UNSUPPORTED;
+  if (r->Tq >= 64)
+    s = gs_lm_head_logits_stats(w + L.H, d_W, reinterpret_cast<float*>(w + L.logits), r->Tq, r->d, r->V, r->dt,
+                                r->temperature, w + L.stats, L.stats_bytes, &n_chunk, w + L.ws_head, L.ws_head_bytes,
+                                d_status, st);
+  const bool have_stats = (s == GS_OK);
+  if (s == GS_ERR_UNSUPPORTED)
+    s = gs_lm_head_logits(w + L.H, d_W, reinterpret_cast<float*>(w + L.logits), r->Tq, r->d, r->V, r->dt,
+                          w + L.ws_head, L.ws_head_bytes, d_status, st);
   if (s != GS_OK) return s;
   if (cudaStreamWaitEvent(st, side->staged, 0) != cudaSuccess) return GS_ERR_CUDA;
-  s = gs_spec_accept(reinterpret_cast<const float*>(w + L.logits), reinterpret_cast<const float*>(w + L.q_probs),
-                     reinterpret_cast<const int32_t*>(w + L.draft_tok), cu_q,
-                     reinterpret_cast<const float*>(w + L.u_accept), reinterpret_cast<const float*>(w + L.u_sample),
-                     r->temperature, r->N, r->Tq, r->V,
-                     reinterpret_cast<int32_t*>(w + L.accepted), reinterpret_cast<int32_t*>(w + L.out_tok),
-                     reinterpret_cast<int32_t*>(w + L.n_out), reinterpret_cast<float*>(w + L.ratio),
-                     reinterpret_cast<float*>(w + L.p_tok), nullptr, d_alpha_hat, d_X, r->eta, r->beta,
-                     r->alpha_min, r->alpha_max, w + L.ws_acc, L.ws_acc_bytes, d_status, st);
+  const float* lg = reinterpret_cast<const float*>(w + L.logits);
+  const float* qp = reinterpret_cast<const float*>(w + L.q_probs);
+  const int32_t* dtok = reinterpret_cast<const int32_t*>(w + L.draft_tok);
+  const float* ua = reinterpret_cast<const float*>(w + L.u_accept);
+  const float* us = reinterpret_cast<const float*>(w + L.u_sample);
+  int32_t* o_acc = reinterpret_cast<int32_t*>(w + L.accepted);
+  int32_t* o_tok = reinterpret_cast<int32_t*>(w + L.out_tok);
+  int32_t* o_n = reinterpret_cast<int32_t*>(w + L.n_out);
+  float* o_ratio = reinterpret_cast<float*>(w + L.ratio);
+  float* o_p = reinterpret_cast<float*>(w + L.p_tok);
+  s = GS_ERR_UNSUPPORTED;
+  if (have_stats)
+    s = gs_spec_accept_prestats(lg, qp, dtok, cu_q, ua, us, r->temperature, r->N, r->Tq, r->V, o_acc, o_tok, o_n,
+                                o_ratio, o_p, nullptr, d_alpha_hat, d_X, r->eta, r->beta, r->alpha_min, r->alpha_max,
+                                w + L.stats, n_chunk, w + L.ws_acc, L.ws_acc_bytes, d_status, st);
+  if (s == GS_ERR_UNSUPPORTED)
+    s = gs_spec_accept(lg, qp, dtok, cu_q, ua, us, r->temperature, r->N, r->Tq, r->V, o_acc, o_tok, o_n, o_ratio, o_p,
+                       nullptr, d_alpha_hat, d_X, r->eta, r->beta, r->alpha_min, r->alpha_max, w + L.ws_acc,
+                       L.ws_acc_bytes, d_status, st);
   if (s != GS_OK) return s;
   s = gs_schedule(d_X, d_alpha_hat, r->N, r->C, d_s_min, d_s_max, reinterpret_cast<int32_t*>(w + L.S_next),
                   d_status, st);

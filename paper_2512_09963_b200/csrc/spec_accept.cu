@@ -25,12 +25,6 @@ constexpr int kSaChunk = 8192;                   // floats per CTA
 constexpr int kSaPerThread = kSaChunk / kSaThreads;  // 32
 constexpr float kLog2e = 1.4426950408889634f;
 
-struct ChunkStat {   // 16 bytes
-  float m;
-  int arg;
-  double z;
-};
-
 struct SaWorkspace {
   ChunkStat* stats;   // [Tq * n_chunk]
   int* tickets;       // [N] CTAs of a server that have delivered their chunk mass
@@ -152,6 +146,7 @@ struct SaFinishArgs {
   const ChunkStat* stats; int* tickets; double* mass;
   int32_t* d_status;
   int smem_bytes;
+  int stats_from_predecessor;   // the statistics come from the kernel right before this one: read nothing of its output before the wait
 };
 
 // Mass of element v of the selected row: max(0, p - q) or p, in fp64 from an fp32 exponential.
@@ -261,13 +256,21 @@ GS_DEVINL SaDecideSmem sa_decide_carve(unsigned char* raw, int gamma) {
 // First half of the "decide" step: the scalars of every draft position of server i (token, its
 // logit and draft probability -- dependent loads -- and the uniform) go to shared memory.  Reads
 // nothing the statistics pass writes.  The caller synchronises the CTA before sa_decide.
-GS_DEVINL void sa_fetch_scalars(const SaFinishArgs& A, int i, int r0, int gamma, bool writer, const SaDecideSmem& S) {
+// part: 0 = everything, 1 = all but the logits, 2 = the logits only (for the tokens part 1 stored; the
+// same thread handles the same j in both parts).
+GS_DEVINL void sa_fetch_scalars(const SaFinishArgs& A, int i, int r0, int gamma, bool writer, const SaDecideSmem& S,
+                                int part = 0) {
   const int g0 = r0 - i;
   for (int j = threadIdx.x; j < gamma; j += blockDim.x) {
+    if (part == 2) {
+      const int s = S.sTok[j];
+      S.sL[j] = (s >= 0) ? A.logits[(size_t)(r0 + j) * A.V + s] : 0.f;
+      continue;
+    }
     const int s = A.draft_tok[g0 + j];
     const bool in = (s >= 0 && s < A.V);
     S.sTok[j] = in ? s : -1;
-    S.sL[j] = in ? A.logits[(size_t)(r0 + j) * A.V + s] : 0.f;
+    if (part == 0) S.sL[j] = in ? A.logits[(size_t)(r0 + j) * A.V + s] : 0.f;
     S.sQ[j] = in ? A.q_probs[(size_t)(g0 + j) * A.V + s] : 0.f;
     S.sU[j] = A.u_accept[g0 + j];
     if (!in && writer) set_status(A.d_status, GS_ERR_INVALID_ARG);
@@ -541,10 +544,11 @@ __global__ void __launch_bounds__(kFcThreads, 2) sa_finish_cluster(SaFinishArgs 
   bool live = !(r0 < 0 || gamma < 0 || r1 > A.Tq);           // uniform over the cluster
   float* sx = reinterpret_cast<float*>(smem_raw);            // the slice: first the draft row, then the masses in place
   const SaDecideSmem S = sa_decide_carve(smem_raw + (size_t)slice * 4, live ? gamma : 0);
-  if (live) sa_fetch_scalars(A, i, r0, gamma, writer, S);
+  if (live) sa_fetch_scalars(A, i, r0, gamma, writer, S, A.stats_from_predecessor ? 1 : 0);
   const double u = (double)A.u_sample[i];
   pdl_wait();
   pdl_launch_dependents();
+  if (live && A.stats_from_predecessor) sa_fetch_scalars(A, i, r0, gamma, writer, S, 2);   // the logits are the predecessor's output
   __syncthreads();
   if (!live && writer && tid == 0) {
     set_status(A.d_status, GS_ERR_SHAPE);
@@ -738,6 +742,18 @@ extern "C" size_t gs_spec_accept_workspace(int N, int Tq, int V) {
   return gs::sa_layout(N, Tq, V, nullptr, nullptr);
 }
 
+namespace gs {
+static gs_status spec_accept_impl(const float* logits, const float* q_probs, const int32_t* draft_tok,
+                                  const int32_t* cu_q, const float* u_accept, const float* u_sample,
+                                  float temperature, int N, int Tq, int V,
+                                  int32_t* accepted, int32_t* out_tok, int32_t* n_out,
+                                  float* ratio, float* p_tok, float* margin,
+                                  double* alpha_hat, double* X, double eta, double beta,
+                                  double alpha_min, double alpha_max,
+                                  void* ws, size_t ws_bytes, int32_t* d_status, void* stream,
+                                  const ChunkStat* pre_stats, int pre_chunks);
+}
+
 extern "C" gs_status gs_spec_accept(const float* logits, const float* q_probs, const int32_t* draft_tok,
                                     const int32_t* cu_q, const float* u_accept, const float* u_sample,
                                     float temperature, int N, int Tq, int V,
@@ -746,6 +762,36 @@ extern "C" gs_status gs_spec_accept(const float* logits, const float* q_probs, c
                                     double* alpha_hat, double* X, double eta, double beta,
                                     double alpha_min, double alpha_max,
                                     void* ws, size_t ws_bytes, int32_t* d_status, void* stream) {
+  return gs::spec_accept_impl(logits, q_probs, draft_tok, cu_q, u_accept, u_sample, temperature, N, Tq, V, accepted,
+                              out_tok, n_out, ratio, p_tok, margin, alpha_hat, X, eta, beta, alpha_min, alpha_max,
+                              ws, ws_bytes, d_status, stream, nullptr, 0);
+}
+
+/* The acceptance step on statistics that gs_lm_head_logits_stats wrote: no pass over the logits. */
+extern "C" gs_status gs_spec_accept_prestats(const float* logits, const float* q_probs, const int32_t* draft_tok,
+                                             const int32_t* cu_q, const float* u_accept, const float* u_sample,
+                                             float temperature, int N, int Tq, int V,
+                                             int32_t* accepted, int32_t* out_tok, int32_t* n_out,
+                                             float* ratio, float* p_tok, float* margin,
+                                             double* alpha_hat, double* X, double eta, double beta,
+                                             double alpha_min, double alpha_max,
+                                             const void* stats, int n_chunk,
+                                             void* ws, size_t ws_bytes, int32_t* d_status, void* stream) {
+  if (stats == nullptr || n_chunk <= 0) return GS_ERR_INVALID_ARG;
+  return gs::spec_accept_impl(logits, q_probs, draft_tok, cu_q, u_accept, u_sample, temperature, N, Tq, V, accepted,
+                              out_tok, n_out, ratio, p_tok, margin, alpha_hat, X, eta, beta, alpha_min, alpha_max,
+                              ws, ws_bytes, d_status, stream, static_cast<const gs::ChunkStat*>(stats), n_chunk);
+}
+
+static gs_status gs::spec_accept_impl(const float* logits, const float* q_probs, const int32_t* draft_tok,
+                                      const int32_t* cu_q, const float* u_accept, const float* u_sample,
+                                      float temperature, int N, int Tq, int V,
+                                      int32_t* accepted, int32_t* out_tok, int32_t* n_out,
+                                      float* ratio, float* p_tok, float* margin,
+                                      double* alpha_hat, double* X, double eta, double beta,
+                                      double alpha_min, double alpha_max,
+                                      void* ws, size_t ws_bytes, int32_t* d_status, void* stream,
+                                      const ChunkStat* pre_stats, int pre_chunks) {
   using namespace gs;
   if (N < 0 || Tq < 0 || V < 0 || !(temperature >= 0.f)) return GS_ERR_INVALID_ARG;
   if (N == 0) return GS_OK;
@@ -766,7 +812,8 @@ extern "C" gs_status gs_spec_accept(const float* logits, const float* q_probs, c
                    (q_probs == nullptr || reinterpret_cast<uintptr_t>(q_probs) % 16 == 0);
 
   dim3 g1(n_chunk, Tq);
-  if (launch_ex(vec ? sa_row_stats<true> : sa_row_stats<false>, g1, dim3(kSaThreads), 0, st, true, 1,
+  if (pre_stats == nullptr &&
+      launch_ex(vec ? sa_row_stats<true> : sa_row_stats<false>, g1, dim3(kSaThreads), 0, st, true, 1,
                 logits, V, n_chunk, k2, w.stats, w.tickets, N) != cudaSuccess)
     return GS_ERR_CUDA;
 
@@ -778,6 +825,8 @@ extern "C" gs_status gs_spec_accept(const float* logits, const float* q_probs, c
   A.ratio = ratio; A.p_tok = p_tok; A.margin = margin;
   A.alpha_hat = alpha_hat; A.X = X; A.eta = eta; A.beta = beta; A.alpha_min = alpha_min; A.alpha_max = alpha_max;
   A.stats = w.stats; A.tickets = w.tickets; A.mass = w.mass; A.d_status = d_status;
+  A.stats_from_predecessor = 0;
+  if (pre_stats != nullptr) { A.stats = pre_stats; A.n_chunk = pre_chunks; A.stats_from_predecessor = 1; }
   // rows of one server are bounded by Tq - (N-1); size the dynamic shared memory for that
   const size_t max_rows = (size_t)(Tq - N + 1);
   const size_t smem = sa_decide_bytes(max_rows);
@@ -797,9 +846,10 @@ extern "C" gs_status gs_spec_accept(const float* logits, const float* q_probs, c
       (void)cudaGetLastError();
       return GS_ERR_CUDA;
     }
-    count_launches(2);
+    count_launches(pre_stats == nullptr ? 2 : 1);
     return launch_status();
   }
+  if (pre_stats != nullptr) return GS_ERR_UNSUPPORTED;     // only the cluster kernel takes foreign statistics
   if (smem > 160 * 1024) return GS_ERR_UNSUPPORTED;
   A.smem_bytes = (int)smem;
   if (smem > 40 * 1024) {

@@ -49,6 +49,7 @@ class VerifyRound:
         self.ws_attn = _ws(B.gs_verify_attn_workspace(N, Tq, total_kv, max_kv_len, Hq, Hkv, hd, dt), dev)
         self.ws_head = _ws(B.gs_lm_head_workspace(Tq, d, V, dt), dev)
         self.ws_acc = _ws(B.gs_spec_accept_workspace(N, Tq, V), dev)
+        self.stats = _ws(B.gs_lm_head_stats_bytes(Tq), dev)
         self.scale = 1.0 / math.sqrt(hd)
 
     # the four steps, separately callable (the benchmark times them one by one as well)
@@ -67,15 +68,39 @@ class VerifyRound:
                          self.eta, self.beta, self.alpha_min, self.alpha_max,
                          ws=self.ws_acc, d_status=self.d_status)
 
+    def head_accept_fused(self, H, W, q_probs, draft_tok, cu_q, u_accept, u_sample, tau, update=True) -> bool:
+        """LM head with the softmax statistics in its epilogue, then the acceptance step on them (no
+        second pass over the logits).  Shapes without such kernels run the two plain calls.  Returns
+        whether the fused kernels ran."""
+        n_chunk = B.gs_lm_head_logits_stats(H, W, self.logits, tau, self.stats, self.ws_head, self.d_status)
+        if n_chunk is not None:
+            if B.gs_spec_accept_prestats(self.logits, q_probs, draft_tok, cu_q, u_accept, u_sample, tau,
+                                         self.accepted, self.out_tok, self.n_out, self.ratio, self.p_tok,
+                                         self.stats, n_chunk, self.margin,
+                                         self.alpha_hat if update else None, self.X if update else None,
+                                         self.eta, self.beta, self.alpha_min, self.alpha_max,
+                                         ws=self.ws_acc, d_status=self.d_status):
+                return True
+            self.accept(q_probs, draft_tok, cu_q, u_accept, u_sample, tau, update=update)
+            return False
+        self.head(H, W)
+        self.accept(q_probs, draft_tok, cu_q, u_accept, u_sample, tau, update=update)
+        return False
+
     def schedule(self, s_min: Optional[torch.Tensor] = None, s_max: Optional[torch.Tensor] = None):
         B.gs_schedule(self.X, self.alpha_hat, self.C, self.S_next, s_min, s_max, self.d_status)
 
-    def run(self, inp, s_min=None, s_max=None):
-        """Enqueue the whole round for the input dict made by workloads.make_step."""
+    def run(self, inp, s_min=None, s_max=None, fused=False):
+        """Enqueue the whole round for the input dict made by workloads.make_step.  fused=True uses
+        the LM head that writes the softmax statistics where the shape has one."""
         self.attn(inp["Q"], inp["K"], inp["V"], inp["cu_q"], inp["cu_kv"])
-        self.head(inp["H"], inp["W"])
-        self.accept(inp["q_probs"], inp["draft_tok"], inp["cu_q"], inp["u_accept"], inp["u_sample"],
-                    inp["tau"])
+        if fused:
+            self.head_accept_fused(inp["H"], inp["W"], inp["q_probs"], inp["draft_tok"], inp["cu_q"],
+                                   inp["u_accept"], inp["u_sample"], inp["tau"])
+        else:
+            self.head(inp["H"], inp["W"])
+            self.accept(inp["q_probs"], inp["draft_tok"], inp["cu_q"], inp["u_accept"], inp["u_sample"],
+                        inp["tau"])
         self.schedule(s_min, s_max)
 
     @classmethod

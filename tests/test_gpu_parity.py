@@ -432,18 +432,72 @@ def test_attention_bad_offsets_are_flagged():
     assert st == 2
 
 
+# ------------------------------------------------------------------ LM head + acceptance, statistics fused
+@pytest.mark.parametrize("T_extra,d,V,tau", [(0, 512, 9000, 0.7), (0, 256, 20000, 1.0), (0, 320, 4104, 0.0),
+                                             (150, 256, 8192, 0.7)],
+                         ids=["ragged-V", "wide", "greedy", "many-rows"])
+def test_fused_head_statistics_match_two_pass(T_extra, d, V, tau):
+    """gs_lm_head_logits_stats + gs_spec_accept_prestats against the oracle, and against the plain
+    pair of calls: logits bit-identical, counts and tokens equal (the statistics group their sums
+    differently, so probabilities agree to rounding)."""
+    cfg = wl.shrink(wl.CONFIGS["cfg2"], d=d, V=V, prefix_scale=0.02, name=f"fused_{d}_{V}")
+    gamma = [8, 1, 3, 0, 6, 2, 7, 4]
+    if T_extra:
+        cfg = wl.shrink(cfg, N=24, name=cfg.name + "_24")
+        gamma = list(np.random.default_rng(5).integers(3, 9, 24))
+    inp = wl.make_step(cfg, tau=tau, gamma=gamma)
+    dev = to_dev(inp)
+    plain = VerifyRound.for_inputs(dev, C=4 * cfg.N)
+    plain.run(dev)
+    fused = VerifyRound.for_inputs(dev, C=4 * cfg.N)
+    fused.attn(dev["Q"], dev["K"], dev["V"], dev["cu_q"], dev["cu_kv"])
+    ran = fused.head_accept_fused(dev["H"], dev["W"], dev["q_probs"], dev["draft_tok"], dev["cu_q"],
+                                  dev["u_accept"], dev["u_sample"], inp["tau"])
+    fused.schedule()
+    torch.cuda.synchronize()
+    assert ran, "this shape has the fused kernels"
+    assert int(fused.d_status.item()) == 0 and int(plain.d_status.item()) == 0
+    assert torch.equal(fused.logits, plain.logits)
+    t32 = tau32(inp["tau"])
+    ref_logits = orc.ref_lm_head(inp["H"], inp["W"])
+    ref = orc.ref_spec_accept(ref_logits, inp["q_probs"], inp["draft_tok"], inp["cu_q"], inp["u_accept"],
+                              inp["u_sample"], t32)
+    slack = pu.chain_slack(fused.logits, ref_logits, t32)
+    pu.compare_accept(pu.gpu_accept_dict(fused), ref, ref_logits, inp["q_probs"], inp["cu_q"].numpy(),
+                      inp["u_sample"], t32, V, slack=slack)
+    a, b = pu.gpu_accept_dict(fused), pu.gpu_accept_dict(plain)
+    assert np.array_equal(a["accepted"], b["accepted"]) and np.array_equal(a["out_tok"], b["out_tok"])
+    np.testing.assert_allclose(a["ratio"], b["ratio"], atol=2e-6)
+    np.testing.assert_allclose(a["p_tok"], b["p_tok"], atol=2e-6)
+
+
+def test_fused_head_statistics_unsupported_shapes_fall_back():
+    """More than 256 rows: no fused kernel, the runner uses the two plain calls and says so."""
+    cfg = wl.shrink(wl.CONFIGS["cfg3"], d=128, V=4096, prefix_scale=0.02, name="fused_fallback")
+    inp = wl.make_step(cfg, allocator=orc.ref_schedule_greedy)
+    dev = to_dev(inp)
+    assert dev["H"].shape[0] > 256
+    rnd = VerifyRound.for_inputs(dev, C=256)
+    ran = rnd.head_accept_fused(dev["H"], dev["W"], dev["q_probs"], dev["draft_tok"], dev["cu_q"],
+                                dev["u_accept"], dev["u_sample"], inp["tau"])
+    torch.cuda.synchronize()
+    assert not ran and int(rnd.d_status.item()) == 0
+    pu.assert_close_rel(rnd.logits, orc.ref_lm_head(inp["H"], inp["W"]), "fallback logits")
+
+
 # ------------------------------------------------------------------ the round from host buffers
-def test_verify_round_host_matches_device_path():
+@pytest.mark.parametrize("gamma", [[3, 1, 8, 2, 5, 4, 7, 6], [8, 8, 8, 8, 8, 8, 8, 8]], ids=["44-positions", "72-positions"])
+def test_verify_round_host_matches_device_path(gamma):
     """gs_verify_round_host (inputs in pinned host memory, draft distributions copied on the
     library's copy stream while attention and the LM head run) gives what the four calls give on
     device-resident inputs; two rounds back to back with different drafts reuse the staging area."""
     cfg = wl.shrink(wl.CONFIGS["cfg2"], d=256, V=16384, prefix_scale=0.1, name="host_round")
     for round_idx in (0, 1):
-        inp = wl.make_step(cfg, round_idx=round_idx, gamma=[3, 1, 8, 2, 5, 4, 7, 6])     # same shapes, new drafts
+        inp = wl.make_step(cfg, round_idx=round_idx, gamma=gamma)     # same shapes, new drafts
         d = to_dev(inp)
         N, Tq = cfg.N, int(inp["cu_q"][-1])
         rnd = VerifyRound.for_inputs(d, C=4 * N)
-        rnd.run(d)
+        rnd.run(d, fused=Tq >= 64)     # the host-buffer round takes the same kernels (statistics from the LM head from 64 positions on)
         torch.cuda.synchronize()
         assert int(rnd.d_status.item()) == 0
         desc = B.RoundDesc(N=N, Tq=Tq, total_kv=d["K"].shape[0], max_kv_len=rnd.max_kv_len, Hq=cfg.Hq, Hkv=cfg.Hkv,
