@@ -94,6 +94,7 @@ class ClosedLoop:
                                                          cfg.hd, gsdt))
         self.ws_head = ws(B.gs_lm_head_workspace(Tq_max, cfg.d, cfg.V, gsdt))
         self.ws_acc = ws(B.gs_spec_accept_workspace(N, Tq_max, cfg.V))
+        self.stats = ws(B.gs_lm_head_stats_bytes(Tq_max))
 
     # ---------------------------------------------------------------- inputs of round t
     def true_alpha(self, t):
@@ -195,10 +196,25 @@ class ClosedLoop:
         else:
             B.gs_verify_attn(inp["Q"], inp["K"], inp["V"], O, inp["cu_q"], inp["cu_kv"], self.max_kv_len,
                              1.0 / math.sqrt(cfg.hd), self.ws_attn, self.d_status)
-        B.gs_lm_head_logits(inp["H"], inp["W"], logits, self.ws_head, self.d_status)
-        B.gs_spec_accept(logits, inp["q_probs"], inp["draft_tok"], inp["cu_q"], inp["u_accept"], inp["u_sample"],
-                         inp["tau"], self.accepted, self.out_tok[:Tq], self.n_out, self.ratio[:G], self.p_tok[:G],
-                         None, self.alpha_hat, self.X, self.eta, self.beta, ws=self.ws_acc, d_status=self.d_status)
+        # from 64 verify positions on the LM head writes the softmax statistics itself (when the shape
+        # has that kernel) and the acceptance step skips its pass over the logits
+        n_chunk = None
+        if Tq >= 64:
+            n_chunk = B.gs_lm_head_logits_stats(inp["H"], inp["W"], logits, inp["tau"], self.stats, self.ws_head,
+                                                self.d_status)
+        done = False
+        if n_chunk is not None:
+            done = B.gs_spec_accept_prestats(logits, inp["q_probs"], inp["draft_tok"], inp["cu_q"], inp["u_accept"],
+                                             inp["u_sample"], inp["tau"], self.accepted, self.out_tok[:Tq], self.n_out,
+                                             self.ratio[:G], self.p_tok[:G], self.stats, n_chunk, None,
+                                             self.alpha_hat, self.X, self.eta, self.beta, ws=self.ws_acc,
+                                             d_status=self.d_status)
+        else:
+            B.gs_lm_head_logits(inp["H"], inp["W"], logits, self.ws_head, self.d_status)
+        if not done:
+            B.gs_spec_accept(logits, inp["q_probs"], inp["draft_tok"], inp["cu_q"], inp["u_accept"], inp["u_sample"],
+                             inp["tau"], self.accepted, self.out_tok[:Tq], self.n_out, self.ratio[:G], self.p_tok[:G],
+                             None, self.alpha_hat, self.X, self.eta, self.beta, ws=self.ws_acc, d_status=self.d_status)
         B.gs_schedule(self.X, self.alpha_hat, self.C, self.S_next, self.s_min, self.s_max, self.d_status)
         return O, logits
 
