@@ -183,6 +183,14 @@ GS_DEVINL uint32_t pack_bf16_pos(float lo, float hi) {
   return __byte_perm(__float_as_uint(lo) + 0x8000u, __float_as_uint(hi) + 0x8000u, 0x7632);
 }
 
+// Clears the tickets.  The attention kernel is launched behind it as its programmatic dependent: it
+// starts at once (this kernel only began after everything earlier on the stream had finished, so the
+// inputs are complete) and waits for this grid only where it first touches a ticket.
+__global__ void attn_zero_kernel(int* p, int n) {
+  pdl_launch_dependents();
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) p[i] = 0;
+}
+
 __global__ void __launch_bounds__(kAtThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant__ CUtensorMap tmapV,
                const AttnTcParams P) {
@@ -222,8 +230,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // The next kernel on the stream may set itself up on idle SMs right away (it still waits for this
-  // grid to finish before it touches global memory).  This kernel follows a memset and has no
-  // programmatic predecessor of its own.
+  // grid to finish before it touches global memory).
   pdl_launch_dependents();
   if ((base & 1023u) != 0) {                     // the operand layouts need a 1024-byte aligned base
     if (threadIdx.x == 0) set_status(P.d_status, GS_ERR_CUDA);
@@ -625,8 +632,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
       if (!single) {
         if (row_ok) { out[kAtHd] = m_run; out[kAtHd + 1] = l_run; }
         // One ticket per group: the CTA that takes the last one finds the other splits' rows
-        // complete (their writers fenced before taking theirs) and merges them.  The 128 softmax
-        // threads meet on mbarriers with the usual bounded wait.
+        // complete (their writers fenced before taking theirs) and merges them.  The tickets were
+        // cleared by the kernel this one was launched behind: make sure that has finished.
+        // The 128 epilogue threads meet on mbarriers with the usual bounded wait.
+        pdl_wait();
         __threadfence();
         mbar_arrive(bar(kEpiA));
         if (!mbar_wait(bar(kEpiA), (uint32_t)n_ticket & 1u, abort_flag)) { ok = false; break; }
@@ -807,10 +816,14 @@ inline gs_status launch_attn_tc(const void* Q, const void* K, const void* V, voi
   if (!make_tmap_bf16_2d(&tmK, K, kv_rows, (uint64_t)Hkv * kAtHd, (uint64_t)Hkv * kAtHd, kAtTile, 64) ||
       !make_tmap_bf16_2d(&tmV, V, kv_rows, (uint64_t)Hkv * kAtHd, (uint64_t)Hkv * kAtHd, kAtTile, 64))
     return GS_ERR_CUDA;
-  if (cudaMemsetAsync(P.tickets, 0, pl.ticket_bytes, st) != cudaSuccess) return GS_ERR_CUDA;
-  attn_tc_kernel<<<pl.grid, kAtThreads, kAtSmem, st>>>(tmK, tmV, P);
+  const int n_ticket = (int)(pl.ticket_bytes / sizeof(int));
+  attn_zero_kernel<<<(n_ticket + 1023) / 1024 > 64 ? 64 : (n_ticket + 1023) / 1024, 1024, 0, st>>>(P.tickets, n_ticket);
   if (cudaGetLastError() != cudaSuccess) return GS_ERR_CUDA;
-  count_launches(1);
+  if (launch_ex(attn_tc_kernel, dim3(pl.grid), dim3(kAtThreads), kAtSmem, st, true, 1, tmK, tmV, P) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return GS_ERR_CUDA;
+  }
+  count_launches(2);
   return launch_status();
 }
 
