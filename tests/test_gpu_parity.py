@@ -90,6 +90,30 @@ def test_cfg1_matches_stored_golden():
         assert rnd.S_next.cpu().tolist() == gold[tau_key]["S_next"]
 
 
+def test_round_without_dependent_launch_is_bit_identical():
+    """Programmatic dependent launch only moves kernel start-up earlier: a whole round (split
+    attention with tickets included) gives the same bits with the attribute switched off."""
+    cfg = wl.shrink(wl.CONFIGS["cfg2"], d=256, V=8192, prefix_scale=0.25, name="round_pdl")
+    inp = wl.make_step(cfg)
+    d = to_dev(inp)
+    B.gs_verify_attn_configure(2)                 # two-tile splits: partial results, tickets, merges
+    try:
+        outs = []
+        for on in (True, False):
+            B.gs_set_dependent_launch(on)
+            rnd = VerifyRound.for_inputs(d, C=4 * cfg.N)
+            rnd.run(d, fused=True)
+            torch.cuda.synchronize()
+            assert int(rnd.d_status.item()) == 0
+            outs.append({k: getattr(rnd, k).clone() for k in ("O", "logits", "accepted", "out_tok", "ratio", "S_next")})
+    finally:
+        B.gs_set_dependent_launch(True)
+        B.gs_verify_attn_configure(0)
+    for k in outs[0]:
+        assert torch.equal(outs[0][k], outs[1][k]), k
+    pu.assert_close_rel(outs[0]["O"], orc.ref_attention(inp["Q"], inp["K"], inp["V"], inp["cu_q"], inp["cu_kv"]), "attention")
+
+
 # ------------------------------------------------------------------ spec_accept
 ACCEPT_CASES = [
     # name, base cfg, V, tau   (V spans several 4096-chunks plus a ragged tail, or breaks the 16-byte path)
