@@ -15,7 +15,10 @@
 // softmax warps and the loads of later tiles overlap.  An item whose server needs a single KV split normalises and
 // stores its rows directly; otherwise it writes an unnormalised partial (m, l, O) to the workspace
 // and takes a ticket, and the last split of a (server, position block, KV head) to finish merges
-// them (nobody waits).  CTAs are persistent and stride over the items.
+// them (nobody waits).  Four more warps do that epilogue, one item behind the softmax warps, so
+// stores, tickets and merges overlap the next item's tiles.  CTAs are persistent and stride over the
+// items, which are enumerated longest cache first.  The caches may be contiguous or pages of a pool
+// named by a block table (a page is one tile).
 #pragma once
 #include "common.cuh"
 #include "sm100_ptx.cuh"

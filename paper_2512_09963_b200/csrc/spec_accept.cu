@@ -4,15 +4,20 @@
 // Two launches on one stream:
 //   1. sa_row_stats   every logit row is cut into chunks of 8192 floats; one CTA per (chunk,row)
 //                     streams its chunk once with 16-byte loads and writes (max, argmax, sum exp).
-//   2. sa_finish      one CTA per (chunk, server).  Every CTA of a server first repeats the small
-//                     "decide" step (a warp per row merges that row's chunk statistics, evaluates
-//                     p(s_j), q(s_j), the ratio; one thread scans for the first rejection), which
-//                     selects the one row the last token is drawn from; the CTA then sums the mass
-//                     of its chunk of that row (max(0, p - q) after a rejection, p for the bonus
-//                     row).  The last CTA of a server to finish (an atomic ticket, nobody waits)
-//                     scans the chunk masses in order, finds the chunk that holds u * total and
-//                     does an ordered prefix scan inside it.  CTA (0, server) writes the outputs
-//                     and the estimator update.
+//                     (Not launched by gs_spec_accept_prestats: the LM head's epilogue wrote the
+//                     statistics.)
+//   2. the finish step.  Every CTA of a server first repeats the small "decide" step (a warp per row
+//                     merges that row's chunk statistics, evaluates p(s_j), q(s_j), the ratio; one
+//                     thread scans for the first rejection), which selects the one row the last token
+//                     is drawn from (max(0, p - q) after a rejection, p for the bonus row).
+//      sa_finish_cluster (default) one thread-block cluster per server, CTA k owning the k-th slice of
+//                     the vocabulary: slice masses in shared memory, slice totals exchanged through
+//                     distributed shared memory, the owner of u * total scans its own slice.
+//      sa_finish      (V not a multiple of 4, or a slice too large for shared memory) one CTA per
+//                     (chunk, server): chunk masses through the workspace; the last CTA of a server
+//                     to finish (an atomic ticket, nobody waits) scans them, finds the chunk that
+//                     holds u * total and does an ordered prefix scan inside it.
+//                     CTA 0 of a server writes the outputs and the estimator update.
 // Only one row per server is read a second time.  All cross-thread sums are fp64 in a fixed
 // order, so two runs give identical bits.
 #include "common.cuh"
