@@ -524,7 +524,11 @@ constexpr uint32_t kFcPiece = 16384;               // bytes per bulk copy
 
 inline int fc_slice(int V) { return ((V + kFcCluster - 1) / kFcCluster + 3) / 4 * 4; }
 
-__global__ void __launch_bounds__(kFcThreads, 2) sa_finish_cluster(SaFinishArgs A, int slice) {
+// LOADS = 16-byte loads of logits a thread keeps in flight: 4 lets two clusters share an SM (64
+// registers a thread); 10 covers a whole slice of up to 20480 logits in one round trip to L2 and is
+// used when the batch is small enough for every CTA to have an SM of its own.
+template <int LOADS>
+__global__ void __launch_bounds__(kFcThreads, LOADS > 4 ? 1 : 2) sa_finish_cluster(SaFinishArgs A, int slice) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __shared__ __align__(8) uint64_t s_bar;
   __shared__ int s_acc, s_abort, s_found, s_lastpos;
@@ -606,15 +610,15 @@ __global__ void __launch_bounds__(kFcThreads, 2) sa_finish_cluster(SaFinishArgs 
   bool q_here = !resid;
   auto fill_masses = [&](bool res) {
     const int n4 = len >> 2;
-    for (int f0 = tid; f0 < n4; f0 += 4 * kFcThreads) {
-      float4 l[4];
+    for (int f0 = tid; f0 < n4; f0 += LOADS * kFcThreads) {
+      float4 l[LOADS];
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
+      for (int k = 0; k < LOADS; ++k) {
         const int f = f0 + k * kFcThreads;
         l[k] = (f < n4) ? __ldg(l4 + f) : make_float4(0.f, 0.f, 0.f, 0.f);
       }
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
+      for (int k = 0; k < LOADS; ++k) {
         l[k].x = fast_exp2(fmaf(l[k].x, A.k2, negMk)) * invZf;
         l[k].y = fast_exp2(fmaf(l[k].y, A.k2, negMk)) * invZf;
         l[k].z = fast_exp2(fmaf(l[k].z, A.k2, negMk)) * invZf;
@@ -625,7 +629,7 @@ __global__ void __launch_bounds__(kFcThreads, 2) sa_finish_cluster(SaFinishArgs 
         q_here = true;
       }
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
+      for (int k = 0; k < LOADS; ++k) {
         const int f = f0 + k * kFcThreads;
         if (f < n4) {
           float4* dst = reinterpret_cast<float4*>(sx) + f;
@@ -841,12 +845,16 @@ static gs_status gs::spec_accept_impl(const float* logits, const float* q_probs,
   if (vec && g_sa_finish_variant != 1 && smem_fc <= 200 * 1024) {
     static bool attr_set = false;
     if (!attr_set) {
-      if (cudaFuncSetAttribute(sa_finish_cluster, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
+      if (cudaFuncSetAttribute(sa_finish_cluster<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess ||
+          cudaFuncSetAttribute(sa_finish_cluster<10>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
         return GS_ERR_CUDA;
       attr_set = true;
     }
     A.smem_bytes = (int)smem_fc;
-    if (launch_ex(sa_finish_cluster, dim3(kFcCluster, N), dim3(kFcThreads), smem_fc, st, true, kFcCluster, A, slice) !=
+    // every CTA on an SM of its own (with room to spare for the placement of whole clusters)?
+    const bool roomy = (long long)N * kFcCluster * 3 <= (long long)sm_count() * 2 && slice <= 10 * kFcThreads * 4;
+    if ((roomy ? launch_ex(sa_finish_cluster<10>, dim3(kFcCluster, N), dim3(kFcThreads), smem_fc, st, true, kFcCluster, A, slice)
+               : launch_ex(sa_finish_cluster<4>, dim3(kFcCluster, N), dim3(kFcThreads), smem_fc, st, true, kFcCluster, A, slice)) !=
         cudaSuccess) {
       (void)cudaGetLastError();
       return GS_ERR_CUDA;
