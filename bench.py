@@ -38,8 +38,9 @@ ETA, BETA = 0.1, 0.5
 # per launch), keyed by the sha256 of the kernel source it was taken on; a changed kernel reports null.
 # cfg2's full launch is within ncu's single-pass size rule only for the launch list, so the counters
 # were taken on a smaller vocabulary and scale with the units processed (see profiles/).
-# small case (V = 32768): 336.067 MB read + 3.770 MB written per launch, times 151936/32768
-NCU_TRAFFIC = {"26b8c6888d7758e0": {"cfg2": 1575730630}}
+# small case (V = 32768), the kernel with the statistics epilogue: 336.085 MB read + 6.565 MB written
+# per launch, times 151936/32768
+NCU_TRAFFIC = {"26b8c6888d7758e0": {"cfg2": 1588769825}}
 
 
 def _kernel_hash():
@@ -229,10 +230,10 @@ def run_ours(args, cfg, rank, world, local_rank):
     # Does this shape have the LM head that writes the softmax statistics in its epilogue (then the
     # acceptance step does not read the logits a second time)?
     # Measured on B200: the statistics cost the LM head 4-5 us (they sit in the epilogue of its last,
-    # not overlapped, tile) and save the acceptance step its pass over T_q x V logits; that pays from
-    # about 64 verify positions on (cfg4: -2.7 % per step, cfg2 with 46 positions: +0.4 %).
+    # not overlapped, tile) and save the acceptance step its pass over T_q x V logits: -0.5 % per step
+    # at 28 and 46 verify positions, -2.7 % at 87.
     fused = False
-    if not args.no_fused_stats and (Tq >= 64 or args.fused_stats):
+    if not args.no_fused_stats:
         fused = rnd.head_accept_fused(inp["H"], inp["W"], inp["q_probs"], inp["draft_tok"], inp["cu_q"],
                                       inp["u_accept"], inp["u_sample"], inp["tau"], update=False)
         torch.cuda.synchronize()
@@ -399,7 +400,7 @@ def run_ours(args, cfg, rank, world, local_rank):
     flops_head = 2.0 * Tq * d * V
     ach = bytes_head / (k_us["lm_head_logits"] * 1e-6) / 1e9
     khash = _kernel_hash()
-    roofline = {"kernel": "lm_head_pair_kernel", "bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s",
+    roofline = {"kernel": "lm_head_pair_kernel<1, true> (statistics epilogue)" if fused else "lm_head_pair_kernel", "bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s",
                 "frac": ach / peak, "peak_source": f"{peak_kind} (MEASURED_PEAKS.json hbm_gbs)" if peak_kind == "measured"
                 else "fallback 6650 GB/s", "traffic": NCU_TRAFFIC.get(khash, {}).get(cfg.name),
                 "algorithmic_bytes": bytes_head, "duration_us": k_us["lm_head_logits"],
@@ -547,8 +548,6 @@ def main():
     ap.add_argument("--rounds", type=int, default=1000, help="rounds of the closed loop (--config cfg5)")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
-    ap.add_argument("--fused-stats", action="store_true",
-                    help="softmax statistics from the LM head's epilogue even below 64 verify positions")
     ap.add_argument("--no-fused-stats", action="store_true",
                     help="plain gs_lm_head_logits + gs_spec_accept even where the LM head could write the softmax statistics")
     ap.add_argument("--head-sweep", action="store_true",

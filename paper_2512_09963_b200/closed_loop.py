@@ -196,12 +196,10 @@ class ClosedLoop:
         else:
             B.gs_verify_attn(inp["Q"], inp["K"], inp["V"], O, inp["cu_q"], inp["cu_kv"], self.max_kv_len,
                              1.0 / math.sqrt(cfg.hd), self.ws_attn, self.d_status)
-        # from 64 verify positions on the LM head writes the softmax statistics itself (when the shape
-        # has that kernel) and the acceptance step skips its pass over the logits
-        n_chunk = None
-        if Tq >= 64:
-            n_chunk = B.gs_lm_head_logits_stats(inp["H"], inp["W"], logits, inp["tau"], self.stats, self.ws_head,
-                                                self.d_status)
+        # the LM head writes the softmax statistics itself (when the shape has that kernel) and the
+        # acceptance step skips its pass over the logits
+        n_chunk = B.gs_lm_head_logits_stats(inp["H"], inp["W"], logits, inp["tau"], self.stats, self.ws_head,
+                                            self.d_status)
         done = False
         if n_chunk is not None:
             done = B.gs_spec_accept_prestats(logits, inp["q_probs"], inp["draft_tok"], inp["cu_q"], inp["u_accept"],

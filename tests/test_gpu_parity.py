@@ -521,7 +521,7 @@ def test_verify_round_host_matches_device_path(gamma):
         d = to_dev(inp)
         N, Tq = cfg.N, int(inp["cu_q"][-1])
         rnd = VerifyRound.for_inputs(d, C=4 * N)
-        rnd.run(d, fused=Tq >= 64)     # the host-buffer round takes the same kernels (statistics from the LM head from 64 positions on)
+        rnd.run(d, fused=True)         # the host-buffer round takes the same kernels (statistics from the LM head)
         torch.cuda.synchronize()
         assert int(rnd.d_status.item()) == 0
         desc = B.RoundDesc(N=N, Tq=Tq, total_kv=d["K"].shape[0], max_kv_len=rnd.max_kv_len, Hq=cfg.Hq, Hkv=cfg.Hkv,
