@@ -181,8 +181,10 @@ gs_status gs_lm_head_logits(const void* H, const void* W, float* logits, int T, 
  * Estimators (alpha_hat, X: [N] fp64 in/out, both NULL to skip):
  *   alpha_hat_i <- clamp((1-eta) alpha_hat_i + eta * mean_j ratio_j, alpha_min, alpha_max)
  *                  (unchanged when gamma_i = 0);  X_i <- (1-beta) X_i + beta (a_i + 1).
- * Errors: INVALID_ARG, SHAPE (T_q < N), WORKSPACE.  Device status: GS_ERR_SHAPE for decreasing
- * offsets, GS_ERR_INVALID_ARG for a draft token outside [0, V) (it is then rejected).
+ * Errors: INVALID_ARG, SHAPE (T_q < N), WORKSPACE.  Device status: GS_ERR_SHAPE for a server whose
+ * offsets leave it without a row, or leave a server before or after it without one (decreasing
+ * offsets, cu_q[N] > T_q): that server gets accepted = n_out = 0 and nothing else of it is read or
+ * written; GS_ERR_INVALID_ARG for a draft token outside [0, V) (it is then rejected).
  */
 size_t gs_spec_accept_workspace(int N, int Tq, int V);
 /* Kernel choice of the second pass (process-wide, not thread-safe): 0 = automatic: one thread-block
@@ -214,7 +216,7 @@ gs_status gs_spec_accept(const float* logits, const float* q_probs, const int32_
  *   stats         device buffer of gs_lm_head_stats_bytes(T) bytes, 16-byte aligned; receives
  *                 *n_chunk entries per row (one per CTA of the launch; opaque)
  *   n_chunk       host int, written before the call returns
- *   bf16 on CTA pairs with T <= 256 only; every other case returns GS_ERR_UNSUPPORTED and launches
+ *   bf16 on CTA pairs with T <= 512 only; every other case returns GS_ERR_UNSUPPORTED and launches
  *   nothing (call gs_lm_head_logits and gs_spec_accept instead).
  * gs_spec_accept_prestats: arguments and results as gs_spec_accept (same temperature!), plus the
  *   stats buffer and n_chunk.  Needs V % 4 == 0, 16-byte aligned rows and a vocabulary slice that
@@ -288,6 +290,16 @@ gs_status gs_schedule(const double* X, const double* alpha_hat, int N, int C,
  * Errors: INVALID_ARG. */
 gs_status gs_schedule_select(int variant);
 
+/* gs_schedule_host -- the same GoodSpeed-sched allocation (Eq. goodspeed_sched, Sec. III-C) for
+ * estimator state in HOST memory: every pointer is a host pointer, no CUDA call is made, the result
+ * is in S_out when the call returns.  Same marginal-allocation steps and the same chain of fp64
+ * multiplications as gs_schedule, so the two give identical allocations for identical inputs.  Meant
+ * for a scheduler that runs beside the GPU or on ranks that have exchanged their estimates; cost
+ * O(N * C).  Errors: INVALID_ARG (null/negative), UNSUPPORTED (N > 2^20), SHAPE if sum s_min > C (the
+ * floors are then returned as they are). */
+gs_status gs_schedule_host(const double* X, const double* alpha_hat, int N, int C,
+                           const int32_t* s_min, const int32_t* s_max, int32_t* S_out);
+
 /* --------------------------------------------------------------------------------------------
  * gs_verify_round_host -- Algorithm 1, the verification-server steps of one round (batching,
  * verification, estimator update, GoodSpeed-sched), for a caller whose per-round data is in HOST
@@ -329,6 +341,19 @@ gs_status gs_verify_round_host(const gs_round_desc* r,
                                void* d_ws, size_t ws_bytes,
                                int32_t* h_accepted, int32_t* h_out_tok, int32_t* h_n_out,
                                int32_t* h_S_next, int32_t* h_status, void* stream);
+
+/* --------------------------------------------------------------------------------------------
+ * gs_selftest_wait_timeout -- no counterpart in the paper: a check of the library's failure path.
+ * Every device-side wait of this library (on an mbarrier a TMA load, an MMA or another warp
+ * completes) is bounded: when it runs out the kernel raises an abort flag, all its roles leave their
+ * loops, GS_ERR_TIMEOUT goes to *d_status and the kernel ends normally, so the context stays usable.
+ * This call launches one warp that waits, with that same wait routine, for a barrier nothing ever
+ * completes, with a limit of limit_us microseconds (1 .. 1 000 000) instead of the production 2 s.
+ *   d_status     device int32 (required): receives GS_ERR_TIMEOUT (sticky like every device status)
+ *   d_waited_ns  device uint64, nullable: how long the wait lasted
+ * Errors: INVALID_ARG.  Nothing faults and nothing waits beyond the limit. */
+gs_status gs_selftest_wait_timeout(unsigned int limit_us, int32_t* d_status, unsigned long long* d_waited_ns,
+                                   void* stream);
 
 /* Number of CUDA kernels the library has launched so far in this process (host-side counter). */
 unsigned long long gs_launch_count(void);

@@ -55,6 +55,8 @@ SIGNATURES = {
                                    _vp, _vp, _vp, _vp, _vp, _vp,
                                    _vp, _vp, _d, _d, _d, _d, _vp, _vp]),
     "gs_schedule": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp]),
+    "gs_schedule_host": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp]),
+    "gs_selftest_wait_timeout": (_i, [C.c_uint, _vp, _vp, _vp]),
     "gs_verify_round_workspace": (_sz, [_vp]),
     "gs_verify_round_host": (_i, [_vp] + [_vp] * 8 + [_vp] * 7 + [_vp, _sz] + [_vp] * 5 + [_vp]),
     "gs_launch_count": (C.c_ulonglong, []),
@@ -277,6 +279,28 @@ def gs_schedule(X, alpha_hat, C_budget, S_out, s_min=None, s_max=None, d_status=
     code = lib().gs_schedule(_ptr(X, f64), _ptr(alpha_hat, f64), N, int(C_budget), _ptr(s_min, i32),
                              _ptr(s_max, i32), _ptr(S_out, i32), _ptr(d_status, i32), _stream())
     _check("gs_schedule", code)
+
+
+def gs_schedule_host(X, alpha_hat, C_budget, S_out, s_min=None, s_max=None):
+    """gs_schedule on host arrays (CPU tensors); no CUDA call.  GS_ERR_SHAPE (floors above the
+    budget) raises like every other error, after S_out has received the floors."""
+    N = X.numel()
+    i32, f64 = torch.int32, torch.float64
+    hp = lambda t, dt: _ptr(t, dt, cuda=False)
+    for t in (X, alpha_hat, S_out, s_min, s_max):
+        if t is not None and t.is_cuda:
+            raise ValueError("gs_schedule_host takes host tensors")
+    code = lib().gs_schedule_host(hp(X, f64), hp(alpha_hat, f64), N, int(C_budget), hp(s_min, i32), hp(s_max, i32),
+                                  hp(S_out, i32))
+    _check("gs_schedule_host", code)
+
+
+def gs_selftest_wait_timeout(limit_us, d_status, d_waited_ns=None):
+    """One warp waits limit_us microseconds for a barrier nothing completes, then reports
+    GS_ERR_TIMEOUT in d_status (see the header)."""
+    _check("gs_selftest_wait_timeout",
+           lib().gs_selftest_wait_timeout(int(limit_us), _ptr(d_status, torch.int32), _ptr(d_waited_ns, torch.int64),
+                                          _stream()))
 
 
 def gs_launch_count() -> int:

@@ -40,7 +40,11 @@ attn_generic_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T* _
   const int i = find_server(cu_q, N, r);
   const int q0 = cu_q[i], n_new = cu_q[i + 1] - q0;
   const int k0 = cu_kv[i], Lkv = cu_kv[i + 1] - k0;
-  if (n_new <= 0 || Lkv < n_new || Lkv > max_kv_len || k0 < 0 || k0 + Lkv > total_kv) {
+  // the same per-server checks as the tensor-core kernel, plus: this row must lie inside the server the
+  // search returned (offsets that do not start at 0 or that decrease would otherwise hand it another
+  // server's keys).  Such rows are flagged and left unwritten.
+  if (n_new <= 0 || Lkv < n_new || Lkv > max_kv_len || k0 < 0 || k0 + Lkv > total_kv || q0 < 0 ||
+      q0 + n_new > Tq || r < q0 || r >= q0 + n_new) {
     if (tid == 0) set_status(d_status, GS_ERR_SHAPE);
     return;
   }

@@ -255,7 +255,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
   if (warp == 1) {
     tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kAtTmemCols);
     tmem_relinquish();
-  } else if (cached) {
+  }
+  // The barrier and tensor-memory set-up above overlaps the tail of whatever runs before this kernel
+  // on the stream; global memory is touched only after that work has finished.
+  pdl_wait();
+  if (warp != 1 && cached) {
     const int t = (warp == 0) ? (int)threadIdx.x : (int)threadIdx.x - 32;      // every thread but the allocating warp's
     for (int i = t; i <= P.N; i += kAtThreads - 32) {
       const int q0 = P.cu_q[i], k0 = P.cu_kv[i];
@@ -793,11 +797,12 @@ inline gs_status launch_attn_tc(const void* Q, const void* K, const void* V, voi
                                 const int32_t* cu_kv, int N, int Tq, int total_kv, int max_kv_len, int Hq, int Hkv,
                                 float scale, void* ws, int32_t* d_status, cudaStream_t st,
                                 const int32_t* block_table = nullptr, int max_pages = 0, int n_pages = 0) {
-  static bool attr_set = false;
-  if (!attr_set) {
+  static PerDeviceOnce attr_set;
+  const int slot = device_slot();
+  if (attr_set.needed(slot)) {
     if (cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAtSmem) != cudaSuccess)
       return GS_ERR_CUDA;
-    attr_set = true;
+    attr_set.mark(slot);
   }
   const AttnTcPlan pl = attn_tc_plan(N, Tq, total_kv, max_kv_len, Hq, Hkv);
   AttnTcParams P;

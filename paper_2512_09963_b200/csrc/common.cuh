@@ -71,17 +71,32 @@ inline cudaError_t launch_ex(void (*kernel)(KArgs...), dim3 grid, dim3 block, si
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
+// Per-device host state (function attributes set, SM counts, addresses of __device__ arrays) is kept
+// in tables indexed by the CUDA device that is current when the entry point is called.
+constexpr int kMaxDevices = 64;
+inline int device_slot() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+  return dev;
+}
+
+// True once per device: the caller then sets its kernels' attributes (cudaFuncSetAttribute applies to
+// the current device only) and calls mark() when that succeeded.
+struct PerDeviceOnce {
+  bool done[kMaxDevices] = {};
+  bool needed(int slot) const { return slot < 0 || !done[slot]; }
+  void mark(int slot) { if (slot >= 0) done[slot] = true; }
+};
+
 inline int sm_count() {
-  static int cached = 0;
-  if (cached == 0) {
-    int dev = 0, n = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess &&
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
-      cached = n;
-    else
-      cached = kNumSMsFallback;
-  }
-  return cached;
+  static int cached[kMaxDevices] = {};
+  const int slot = device_slot();
+  if (slot >= 0 && cached[slot] > 0) return cached[slot];
+  int n = 0;
+  if (slot < 0 || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, slot) != cudaSuccess || n <= 0)
+    return kNumSMsFallback;
+  cached[slot] = n;
+  return n;
 }
 
 // 2^x by the special-function unit (relative error about 2 ulp); 2^-inf = 0.

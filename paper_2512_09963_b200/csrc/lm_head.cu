@@ -336,14 +336,15 @@ inline gs_status launch_lm_head_tc(const void* H, const void* W, float* logits, 
       {lm_head_tc_kernel<16, 1>, lm_head_tc_kernel<16, 2>},
       {lm_head_tc_kernel<32, 1>, lm_head_tc_kernel<32, 2>},
       {lm_head_tc_kernel<64, 1>, lm_head_tc_kernel<64, 2>}};
-  static bool attr_set = false;
-  if (!attr_set) {
+  static PerDeviceOnce attr_set;
+  const int slot = device_slot();
+  if (attr_set.needed(slot)) {
     for (int a = 0; a < 3; ++a)
       for (int b = 0; b < 2; ++b)
         if (cudaFuncSetAttribute(kernels[a][b], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem) !=
             cudaSuccess)
           return GS_ERR_CUDA;
-    attr_set = true;
+    attr_set.mark(slot);
   }
   const int sms = sm_count();
   const int units = (V + (int)kTileM - 1) / (int)kTileM;

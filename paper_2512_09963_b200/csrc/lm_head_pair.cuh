@@ -25,8 +25,10 @@ constexpr uint32_t kPairWUnitBytes = 2u * kPairBlockK * 128u;   // one CTA's W s
 constexpr uint32_t kPairMaxSmem = 232448;
 constexpr int kPairMaxUnits = 4;            // widest tile, in units
 
-constexpr int kPairStatRows = 256;          // most rows the epilogue keeps softmax statistics for
-constexpr uint32_t kPairStatBytes = 4u * kPairStatRows * 12u;   // per epilogue warp and row: maximum, its index, sum
+constexpr int kPairStatRows = 512;          // most rows the epilogue keeps softmax statistics for (two MMAs along the rows)
+// Shared memory of the running statistics for a launch with `nt` MMAs along the rows: per epilogue warp
+// and row a maximum, its index and a sum.
+constexpr uint32_t pair_stat_bytes(int nt) { return 4u * (uint32_t)(nt * 256) * 12u; }
 
 struct HeadPairParams {
   float* logits;
@@ -99,15 +101,16 @@ lm_head_pair_kernel(const __grid_constant__ CUtensorMap tmapW, const __grid_cons
   uint8_t* tail = sm + (bars - base) + 8u * (uint32_t)(2 * S + 4);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 4);
-  // running statistics: [4 epilogue warps][kPairStatRows] maxima, indices, sums
+  // running statistics: [4 epilogue warps][SR] maxima, indices, sums
+  constexpr int SR = NT * 256;
   float* st_m = reinterpret_cast<float*>(tail + 64);
-  int* st_a = reinterpret_cast<int*>(st_m + 4 * kPairStatRows);
-  float* st_z = reinterpret_cast<float*>(st_a + 4 * kPairStatRows);
+  int* st_a = reinterpret_cast<int*>(st_m + 4 * SR);
+  float* st_z = reinterpret_cast<float*>(st_a + 4 * SR);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_cta_rank();                // 0 = even CTA (issues the MMAs)
   if (STATS) {
-    for (int i = threadIdx.x; i < 4 * kPairStatRows; i += kPairThreads) { st_m[i] = -INFINITY; st_a[i] = INT_MAX; st_z[i] = 0.f; }
+    for (int i = threadIdx.x; i < 4 * SR; i += kPairThreads) { st_m[i] = -INFINITY; st_a[i] = INT_MAX; st_z[i] = 0.f; }
   }
   const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
   if (threadIdx.x == 0) {
@@ -298,7 +301,7 @@ lm_head_pair_kernel(const __grid_constant__ CUtensorMap tmapW, const __grid_cons
               const float z_me = e[0] + __shfl_xor_sync(0xffffffffu, e[0], 1);
               const int row = t_first + c_me;
               if ((lane & 1) == 0 && row < P.T) {
-                const int slot = q * kPairStatRows + row;
+                const int slot = q * SR + row;
                 const float m0 = st_m[slot];
                 if (m_me > -INFINITY) {
                   const float mn = fmaxf(m0, m_me);
@@ -327,12 +330,12 @@ lm_head_pair_kernel(const __grid_constant__ CUtensorMap tmapW, const __grid_cons
     for (int row = threadIdx.x; row < P.T; row += kPairThreads) {
       float M = -INFINITY; int arg = INT_MAX;
 #pragma unroll
-      for (int w = 0; w < 4; ++w) argmax_merge(M, arg, st_m[w * kPairStatRows + row], st_a[w * kPairStatRows + row]);
+      for (int w = 0; w < 4; ++w) argmax_merge(M, arg, st_m[w * SR + row], st_a[w * SR + row]);
       double z = 0.0;
 #pragma unroll
       for (int w = 0; w < 4; ++w) {
-        const float mw = st_m[w * kPairStatRows + row];
-        if (mw > -INFINITY) z += (double)st_z[w * kPairStatRows + row] * (double)fast_exp2((mw - M) * P.k2);
+        const float mw = st_m[w * SR + row];
+        if (mw > -INFINITY) z += (double)st_z[w * SR + row] * (double)fast_exp2((mw - M) * P.k2);
       }
       ChunkStat cs;
       cs.m = M; cs.arg = arg; cs.z = z;
@@ -413,30 +416,34 @@ inline HeadPairPlan head_pair_plan(int rows, int row0, int d, int V, int cluster
 }
 
 // stats != NULL: the kernel variant that also writes per-row softmax statistics, [T][*n_chunk] entries
-// (one MMA along the rows only, i.e. T <= 256; otherwise GS_ERR_UNSUPPORTED and nothing is launched).
+// (one launch only, i.e. T <= 512; otherwise GS_ERR_UNSUPPORTED and nothing is launched).
 inline gs_status launch_lm_head_pair(const void* H, const void* W, float* logits, int T, int d, int V,
                                      int32_t* d_status, int max_units, int max_stages, cudaStream_t st,
                                      ChunkStat* stats = nullptr, float k2 = 0.f, int max_chunks = 0, int* n_chunk = nullptr) {
   using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const HeadPairParams);
-  static const KernelFn kernels[3] = {lm_head_pair_kernel<1>, lm_head_pair_kernel<2>, lm_head_pair_kernel<1, true>};
+  static const KernelFn kernels[4] = {lm_head_pair_kernel<1>, lm_head_pair_kernel<2>, lm_head_pair_kernel<1, true>,
+                                      lm_head_pair_kernel<2, true>};
   if (stats != nullptr && T > kPairStatRows) return GS_ERR_UNSUPPORTED;
-  static int clusters_avail = -1;
-  if (clusters_avail < 0) {
-    for (int a = 0; a < 3; ++a) {
+  static int clusters_per_device[kMaxDevices] = {};
+  const int slot = device_slot();
+  if (slot < 0) return GS_ERR_CUDA;
+  int& clusters_avail = clusters_per_device[slot];
+  if (clusters_avail <= 0) {
+    for (int a = 0; a < 4; ++a) {
       if (cudaFuncSetAttribute(kernels[a], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairMaxSmem) != cudaSuccess)
         return GS_ERR_CUDA;
       if (cudaFuncSetAttribute(kernels[a], cudaFuncAttributeNonPortableClusterSizeAllowed, 0) != cudaSuccess)
         (void)cudaGetLastError();
     }
     clusters_avail = head_pair_max_clusters(kernels[1], kPairMaxSmem);
-    if (clusters_avail < 1) { clusters_avail = -1; return GS_ERR_UNSUPPORTED; }
+    if (clusters_avail < 1) { clusters_avail = 0; return GS_ERR_UNSUPPORTED; }
   }
   for (int row0 = 0; row0 < T; row0 += 512) {
     const int rows = min(512, T - row0);
     HeadPairPlan pl = head_pair_plan(rows, row0, d, V, clusters_avail, max_units, max_stages,
-                                     stats != nullptr ? kPairStatBytes : 0u);
+                                     stats != nullptr ? pair_stat_bytes((rows + 255) / 256) : 0u);
     if (!pl.ok) return GS_ERR_UNSUPPORTED;
-    if (stats != nullptr && (pl.P.nt != 1 || 2 * pl.clusters > max_chunks)) return GS_ERR_UNSUPPORTED;
+    if (stats != nullptr && 2 * pl.clusters > max_chunks) return GS_ERR_UNSUPPORTED;
     pl.P.logits = logits; pl.P.d_status = d_status; pl.P.stats = stats; pl.P.k2 = k2;
     if (n_chunk != nullptr) *n_chunk = 2 * pl.clusters;
     CUtensorMap tmapW, tmapH;
@@ -454,7 +461,7 @@ inline gs_status launch_lm_head_pair(const void* H, const void* W, float* logits
     at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at; cfg.numAttrs = dependent_launch_enabled() ? 2 : 1;
-    if (cudaLaunchKernelEx(&cfg, kernels[stats != nullptr ? 2 : pl.P.nt - 1], tmapW, tmapH, pl.P) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, kernels[(stats != nullptr ? 2 : 0) + pl.P.nt - 1], tmapW, tmapH, pl.P) != cudaSuccess) {
       (void)cudaGetLastError();
       return GS_ERR_CUDA;
     }

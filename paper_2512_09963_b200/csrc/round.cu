@@ -60,10 +60,9 @@ struct RoundSide {
   bool ok = false;
 };
 static RoundSide* round_side() {
-  constexpr int kMaxDevices = 64;
-  static RoundSide side[kMaxDevices];
-  int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  static RoundSide side[gs::kMaxDevices];
+  const int dev = gs::device_slot();
+  if (dev < 0) return nullptr;
   RoundSide& s = side[dev];
   if (!s.ok) {
     if (cudaStreamCreateWithFlags(&s.copy, cudaStreamNonBlocking) != cudaSuccess ||

@@ -13,6 +13,7 @@
 //   * schedule_kernel: the greedy itself, one block-wide arg-max per token; any N <= 1024, and the
 //     path taken when an alpha_hat lies outside [0, 1] (gains no longer non-increasing).
 #include "common.cuh"
+#include <new>
 
 namespace gs {
 
@@ -210,12 +211,13 @@ extern "C" gs_status gs_schedule(const double* X, const double* alpha_hat, int N
   if (N > 1024) return GS_ERR_UNSUPPORTED;
   const size_t table = (size_t)N * (size_t)(C > 0 ? C : 1) * 8;
   if (N <= 32 && table <= 160 * 1024 && gs::g_schedule_variant != 1) {
-    static bool attr_set = false;
-    if (!attr_set) {
+    static gs::PerDeviceOnce attr_set;
+    const int slot = gs::device_slot();
+    if (attr_set.needed(slot)) {
       if (cudaFuncSetAttribute(gs::schedule_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024) !=
           cudaSuccess)
         return GS_ERR_CUDA;
-      attr_set = true;
+      attr_set.mark(slot);
     }
     if (gs::launch_ex(gs::schedule_rank_kernel, dim3(1), dim3(32 * N), table, static_cast<cudaStream_t>(stream), true, 1,
                       X, alpha_hat, N, C, s_min, s_max, S_out, d_status) != cudaSuccess) {
@@ -233,4 +235,47 @@ extern "C" gs_status gs_schedule(const double* X, const double* alpha_hat, int N
   }
   gs::count_launches(1);
   return GS_OK;
+}
+
+
+// The same allocation for estimator state that lives in host memory (a scheduler that runs beside
+// the GPU, or ranks that have just exchanged their estimates): plain C++, no CUDA call.  The gains
+// follow the device kernels bit for bit: alpha_hat / X, then one fp64 multiplication per step
+// (nothing here can contract into a fused multiply-add), negative or NaN gains count as zero, the
+// lowest index wins ties, an eligible zero gain still beats "no server left".
+extern "C" gs_status gs_schedule_host(const double* X, const double* alpha_hat, int N, int C,
+                                      const int32_t* s_min, const int32_t* s_max, int32_t* S_out) {
+  if (N < 0 || C < 0) return GS_ERR_INVALID_ARG;
+  if (N == 0) return GS_OK;
+  if (!X || !alpha_hat || !S_out) return GS_ERR_INVALID_ARG;
+  if (N > (1 << 20)) return GS_ERR_UNSUPPORTED;
+  double* gain = new (std::nothrow) double[N];
+  int32_t* cap = new (std::nothrow) int32_t[N];
+  if (gain == nullptr || cap == nullptr) { delete[] gain; delete[] cap; return GS_ERR_INVALID_ARG; }
+  long long used = 0;
+  for (int i = 0; i < N; ++i) {
+    const double a = alpha_hat[i];
+    int S = s_min ? s_min[i] : 0;
+    if (S < 0) S = 0;
+    cap[i] = s_max ? s_max[i] : C;
+    double g = a / X[i];
+    for (int k = 0; k < S; ++k) g = g * a;
+    gain[i] = (g >= 0.0) ? g : 0.0;
+    S_out[i] = S;
+    used += S;
+  }
+  gs_status rc = GS_OK;
+  long long budget = (long long)C - used;
+  if (budget < 0) { rc = GS_ERR_SHAPE; budget = 0; }      // floors above the budget: returned as they are
+  for (long long step = 0; step < budget; ++step) {
+    int best = -1;
+    for (int i = 0; i < N; ++i)
+      if (S_out[i] < cap[i] && (best < 0 || gain[i] > gain[best])) best = i;
+    if (best < 0) break;                                    // every server is at its cap
+    S_out[best] += 1;
+    gain[best] = gain[best] * alpha_hat[best];
+  }
+  delete[] gain;
+  delete[] cap;
+  return rc;
 }

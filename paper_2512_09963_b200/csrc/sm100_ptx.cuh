@@ -46,7 +46,7 @@ GS_DEVINL bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // another thread of the CTA already gave up) it raises *abort_flag and returns false, so every
 // role of the kernel leaves its loop and the kernel ends; no wait in this library is unbounded.
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
-GS_DEVINL bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+GS_DEVINL bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint64_t limit_ns = kWaitLimitNs) {
   uint64_t t0 = 0;
   for (uint32_t spin = 1;; ++spin) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -54,7 +54,7 @@ GS_DEVINL bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag
       if (*abort_flag) return false;
       const uint64_t now = global_timer_ns();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+      else if (now - t0 > limit_ns) { *abort_flag = 1; return false; }
     }
   }
 }
@@ -72,8 +72,9 @@ GS_DEVINL bool elect_one() {
   return pred != 0;
 }
 // Whole-warp wait: every lane polls, the verdict is made uniform.
-GS_DEVINL bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag)) != 0;
+GS_DEVINL bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                              uint64_t limit_ns = kWaitLimitNs) {
+  return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, limit_ns)) != 0;
 }
 
 // ------------------------------------------------------------------ TMA (per-CTA loads only)

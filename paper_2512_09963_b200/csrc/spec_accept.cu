@@ -258,6 +258,14 @@ GS_DEVINL SaDecideSmem sa_decide_carve(unsigned char* raw, int gamma) {
   return S;
 }
 
+// Offsets of server i that keep every access of the finish step inside its arrays: at least one row,
+// at least one row left for each server before it (its per-draft offset r0 - i is then >= 0) and for
+// each server after it (its last draft entry r1 - 2 - i then lies below Gamma = Tq - N, and its
+// r1 - r0 rows fit the shared memory sized for Tq - N + 1).  Any other server is skipped and flagged.
+GS_DEVINL bool sa_server_ok(int i, int r0, int r1, int N, int Tq) {
+  return r0 >= i && r1 > r0 && r1 <= Tq - (N - 1 - i);
+}
+
 // First half of the "decide" step: the scalars of every draft position of server i (token, its
 // logit and draft probability -- dependent loads -- and the uniform) go to shared memory.  Reads
 // nothing the statistics pass writes.  The caller synchronises the CTA before sa_decide.
@@ -387,7 +395,7 @@ __global__ void __launch_bounds__(kSaThreads) sa_finish(SaFinishArgs A) {
   const bool writer = (c == 0);           // one CTA per server owns the outputs
   const int r0 = A.cu_q[i], r1 = A.cu_q[i + 1];
   const int gamma = r1 - r0 - 1;
-  if (r0 < 0 || gamma < 0 || r1 > A.Tq) {
+  if (!sa_server_ok(i, r0, r1, A.N, A.Tq)) {
     if (writer && tid == 0) {
       set_status(A.d_status, GS_ERR_SHAPE);
       A.accepted[i] = 0; A.n_out[i] = 0;
@@ -550,7 +558,7 @@ __global__ void __launch_bounds__(kFcThreads, LOADS > 4 ? 1 : 2) sa_finish_clust
   const bool writer = (rank == 0);
   const int r0 = A.cu_q[i], r1 = A.cu_q[i + 1];
   const int gamma = r1 - r0 - 1;
-  bool live = !(r0 < 0 || gamma < 0 || r1 > A.Tq);           // uniform over the cluster
+  bool live = sa_server_ok(i, r0, r1, A.N, A.Tq);            // uniform over the cluster
   float* sx = reinterpret_cast<float*>(smem_raw);            // the slice: first the draft row, then the masses in place
   const SaDecideSmem S = sa_decide_carve(smem_raw + (size_t)slice * 4, live ? gamma : 0);
   if (live) sa_fetch_scalars(A, i, r0, gamma, writer, S, A.stats_from_predecessor ? 1 : 0);
@@ -843,12 +851,13 @@ static gs_status gs::spec_accept_impl(const float* logits, const float* q_probs,
   const int slice = fc_slice(V);
   const size_t smem_fc = (size_t)slice * 4 + smem;
   if (vec && g_sa_finish_variant != 1 && smem_fc <= 200 * 1024) {
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceOnce attr_set;
+    const int slot = device_slot();
+    if (attr_set.needed(slot)) {
       if (cudaFuncSetAttribute(sa_finish_cluster<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess ||
           cudaFuncSetAttribute(sa_finish_cluster<10>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
         return GS_ERR_CUDA;
-      attr_set = true;
+      attr_set.mark(slot);
     }
     A.smem_bytes = (int)smem_fc;
     // every CTA on an SM of its own (with room to spare for the placement of whole clusters)?
@@ -893,10 +902,9 @@ static __device__ __align__(256) unsigned char g_sa_static_scratch[kSaStaticByte
 // In host code the symbol above is only a handle; the device address has to be asked for, once
 // per device, with that device current.
 static void* sa_static_scratch_ptr(gs_status* err) {
-  constexpr int kMaxDevices = 64;
   static void* cached[kMaxDevices] = {};
-  int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { *err = GS_ERR_CUDA; return nullptr; }
+  const int dev = device_slot();
+  if (dev < 0) { *err = GS_ERR_CUDA; return nullptr; }
   if (cached[dev] == nullptr) {
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, g_sa_static_scratch) != cudaSuccess || p == nullptr) { *err = GS_ERR_CUDA; return nullptr; }

@@ -7,7 +7,7 @@ the oracle itself flags as near-ties:
   * a correction/bonus draw where u lies within 1e-5 (in CDF units) of the interval of the
     token the library emitted, measured on the oracle's fp64 CDF.
 After a logged accept/reject flip the rest of that server's outputs legitimately diverge and
-are skipped.  Probabilities are compared to 1e-5 absolute, attention outputs and logits to
+are skipped.  Every such decision is printed (pytest -s shows the lines) and returned in the log.  Probabilities are compared to 1e-5 absolute, attention outputs and logits to
 2e-2 relative to max(|ref|, rms(ref row)).
 """
 from __future__ import annotations
@@ -78,6 +78,8 @@ def compare_accept(gpu, ref, logits, q_probs, cu_q, u_sample, tau, V, slack=0.0)
             assert marg < NEAR_TIE_, (f"server {i}: accepted {a_g} vs oracle {a_r}, decision {j} has "
                                      f"|u - p/q| = {marg:.3e}")
             log["accept_near_ties"].append((i, j, float(marg)))
+            print(f"near-tie (accept): server {i} draft position {j}: |u - p/q| = {marg:.3e}; "
+                  f"library accepted {a_g}, oracle {a_r}")
             continue
         assert np.array_equal(seg[:a_g], ref["out_tok"][r0:r0 + a_g]), f"server {i}: accepted tokens"
         tok_g, tok_r = int(seg[a_g]), int(ref["out_tok"][r0 + a_r])
@@ -96,7 +98,18 @@ def compare_accept(gpu, ref, logits, q_probs, cu_q, u_sample, tau, V, slack=0.0)
             f"server {i}: emitted {tok_g}, oracle {tok_r}; u={u_sample[i]:.8f} is {dist:.3e} away from "
             f"the emitted token's CDF interval [{lo:.8f},{hi:.8f}]")
         log["sample_near_ties"].append((i, tok_g, tok_r, float(dist)))
+        print(f"near-tie (draw): server {i}: library token {tok_g}, oracle token {tok_r}; u is {dist:.3e} "
+              f"(CDF units) from the library token's interval")
     return log
+
+
+def log_for_json(log):
+    """The near-tie log as plain lists: which decisions differed from the oracle's, and by how little."""
+    return {"servers": log["servers"], "sample_exact": log["sample_exact"],
+            "accept_near_ties": [{"server": int(i), "draft_position": int(j), "abs_u_minus_ratio": m}
+                                 for i, j, m in log["accept_near_ties"]],
+            "sample_near_ties": [{"server": int(i), "library_token": int(a), "oracle_token": int(b),
+                                  "cdf_distance": d} for i, a, b, d in log["sample_near_ties"]]}
 
 
 def gpu_accept_dict(rnd):

@@ -224,6 +224,97 @@ def test_spec_accept_estimators_and_device_status():
     assert int(r3.d_status.item()) == 2      # GS_ERR_SHAPE
 
 
+@pytest.mark.parametrize("V", [20000, 8, 4099], ids=["slices", "tiny-V", "odd-V"])
+def test_spec_accept_residual_without_mass_draws_from_target(V, finish_variant):
+    """A rejected draft row with q >= p everywhere (q = 1.5 p, unnormalised on purpose): the ratio is
+    2/3 for every token, u_accept = 0.95 rejects, max(0, p - q) has no mass and the correction token
+    is drawn from p itself -- the second pass of the cluster kernel, the whole-row scan of the ticket
+    kernel.  Servers 0, 2 and 5 take that path at their first draft position; the others run as usual."""
+    cfg = wl.shrink(wl.CONFIGS["cfg2"], V=V, d=64, prefix_scale=0.01, name=f"acc_nomass_{V}")
+    inp = wl.make_step(cfg, tau=0.7, gamma=[3, 1, 8, 2, 5, 4, 7, 6], synthetic_logits=True)
+    tau = tau32(inp["tau"])
+    cu_q = inp["cu_q"].numpy()
+    for k in ("q_probs", "u_accept", "draft_tok"):
+        inp[k] = inp[k].clone()
+    for i in (0, 2, 5):
+        r0, g0 = int(cu_q[i]), int(cu_q[i]) - i
+        p = torch.softmax(inp["target_logits_f32"][r0].double() / tau, dim=0)
+        inp["q_probs"][g0] = (1.5 * p).float()
+        inp["u_accept"][g0] = 0.95
+        inp["draft_tok"][g0] = int(torch.argmax(p))          # a token with mass, so that p/q is 2/3 and not 0/0
+    rnd = run_accept_only(inp)
+    ref, log = check_accept(inp, rnd)
+    for i in (0, 2, 5):
+        r0, g0 = int(cu_q[i]), int(cu_q[i]) - i
+        p = orc.ref_softmax_T(pu.np64(inp["target_logits_f32"][r0]), tau)
+        assert np.maximum(p - pu.np64(inp["q_probs"][g0]), 0.0).sum() == 0.0      # the case is really reached
+        assert ref["accepted"][i] == 0 and ref["resampled"][i] == 1
+        assert int(rnd.accepted[i].item()) == 0
+        assert abs(float(rnd.ratio[g0].item()) - 2.0 / 3.0) < 1e-5
+    assert not log["accept_near_ties"]
+    # the three fall-back draws follow p's CDF: they equal the oracle's tokens unless flagged as near-ties
+    assert log["sample_exact"] + len(log["sample_near_ties"]) == cfg.N
+
+
+def _padded(n, dtype, fill):
+    """A tensor of n elements in the middle of a canary-filled buffer: (view, whole buffer)."""
+    buf = torch.full((n + 128,), fill, dtype=dtype, device=DEV)
+    return buf[64:64 + n], buf
+
+
+@pytest.mark.parametrize("bad", ["all-rows-in-server-0", "no-rows-in-server-0"])
+def test_spec_accept_malformed_offsets_touch_nothing(bad, finish_variant):
+    """Offsets that do not decrease but leave a server without a row must only set the device status: no read or write outside the arrays.  Outputs sit inside canary-filled
+    buffers, which must come back untouched apart from accepted / n_out = 0 of the skipped servers."""
+    cfg = wl.shrink(wl.CONFIGS["cfg2"], V=8192, d=64, N=2, prefix_scale=0.01, name="acc_badcu")
+    inp = wl.make_step(cfg, gamma=[3, 4], synthetic_logits=True)
+    d = to_dev(inp)
+    logits = d["target_logits_f32"].contiguous()
+    Tq, V = logits.shape
+    N, G = 2, Tq - 2
+    cu = {"all-rows-in-server-0": [0, Tq, Tq], "no-rows-in-server-0": [0, 0, Tq]}[bad]
+    cu_q = torch.tensor(cu, dtype=torch.int32, device=DEV)
+    i32, f32 = torch.int32, torch.float32
+    acc, acc_b = _padded(N, i32, -77)
+    tok, tok_b = _padded(Tq, i32, -77)
+    nout, nout_b = _padded(N, i32, -77)
+    ratio, ratio_b = _padded(G, f32, -77.0)
+    ptok, ptok_b = _padded(G, f32, -77.0)
+    marg, marg_b = _padded(G + N, f32, -77.0)
+    st = torch.zeros(1, dtype=i32, device=DEV)
+    ws = torch.empty(B.gs_spec_accept_workspace(N, Tq, V), dtype=torch.uint8, device=DEV)
+    B.gs_spec_accept(logits, d["q_probs"], d["draft_tok"], cu_q, d["u_accept"], d["u_sample"], 0.7,
+                     acc, tok, nout, ratio, ptok, marg, None, None, ws=ws, d_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 2                                   # GS_ERR_SHAPE
+    for view, buf, n in ((acc, acc_b, N), (tok, tok_b, Tq), (nout, nout_b, N), (ratio, ratio_b, G),
+                         (ptok, ptok_b, G), (marg, marg_b, G + N)):
+        assert bool((buf[:64] == -77).all()) and bool((buf[64 + n:] == -77).all())
+    assert acc.tolist() == [0, 0] and nout.tolist() == [0, 0]
+    assert bool((tok == -77).all()) and bool((ratio == -77).all()) and bool((ptok == -77).all())
+
+
+def test_bounded_wait_runs_out_and_reports_timeout():
+    """A device-side wait that nothing will ever complete gives up after its limit: the kernel writes
+    GS_ERR_TIMEOUT to the device status and ends normally; the context stays usable (a scheduler call
+    right after it gives the right answer)."""
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    waited = torch.zeros(1, dtype=torch.int64, device=DEV)
+    B.gs_selftest_wait_timeout(3000, st, waited)                 # 3 ms
+    torch.cuda.synchronize()
+    assert int(st.item()) == 6                                   # GS_ERR_TIMEOUT
+    assert 3_000_000 <= int(waited.item()) < 500_000_000
+    assert "wait" in B.gs_status_str(6)
+    X = torch.tensor([1.0, 2.0, 4.0], dtype=torch.float64, device=DEV)
+    al = torch.tensor([0.5, 0.9, 0.7], dtype=torch.float64, device=DEV)
+    S = torch.empty(3, dtype=torch.int32, device=DEV)
+    st2 = torch.zeros(1, dtype=torch.int32, device=DEV)
+    B.gs_schedule(X, al, 12, S, None, None, st2)
+    torch.cuda.synchronize()
+    assert int(st2.item()) == 0
+    assert np.array_equal(S.cpu().numpy(), orc.ref_schedule_greedy(X.cpu().numpy(), al.cpu().numpy(), 12))
+
+
 # ------------------------------------------------------------------ scheduler
 @pytest.fixture(params=[0, 1], ids=["rank-kernel", "greedy-kernel"])
 def schedule_variant(request):
@@ -458,17 +549,22 @@ def test_attention_bad_offsets_are_flagged():
 
 # ------------------------------------------------------------------ LM head + acceptance, statistics fused
 @pytest.mark.parametrize("T_extra,d,V,tau", [(0, 512, 9000, 0.7), (0, 256, 20000, 1.0), (0, 320, 4104, 0.0),
-                                             (150, 256, 8192, 0.7)],
-                         ids=["ragged-V", "wide", "greedy", "many-rows"])
+                                             (150, 256, 8192, 0.7), (288, 256, 8200, 1.0), (512, 192, 4104, 0.7),
+                                             (300, 128, 4096, 0.0)],
+                         ids=["ragged-V", "wide", "greedy", "many-rows", "288-rows", "512-rows", "greedy-300-rows"])
 def test_fused_head_statistics_match_two_pass(T_extra, d, V, tau):
     """gs_lm_head_logits_stats + gs_spec_accept_prestats against the oracle, and against the plain
     pair of calls: logits bit-identical, counts and tokens equal (the statistics group their sums
     differently, so probabilities agree to rounding)."""
     cfg = wl.shrink(wl.CONFIGS["cfg2"], d=d, V=V, prefix_scale=0.02, name=f"fused_{d}_{V}")
     gamma = [8, 1, 3, 0, 6, 2, 7, 4]
-    if T_extra:
+    if T_extra == 150:
         cfg = wl.shrink(cfg, N=24, name=cfg.name + "_24")
         gamma = list(np.random.default_rng(5).integers(3, 9, 24))
+    elif T_extra:                                     # exactly T_extra verify positions: two MMAs along the rows
+        cfg = wl.shrink(cfg, N=32, name=cfg.name + f"_{T_extra}")
+        gamma = np.random.default_rng(T_extra).multinomial(T_extra - 32, np.ones(32) / 32)
+        assert gamma.sum() + 32 == T_extra
     inp = wl.make_step(cfg, tau=tau, gamma=gamma)
     dev = to_dev(inp)
     plain = VerifyRound.for_inputs(dev, C=4 * cfg.N)
@@ -496,11 +592,11 @@ def test_fused_head_statistics_match_two_pass(T_extra, d, V, tau):
 
 
 def test_fused_head_statistics_unsupported_shapes_fall_back():
-    """More than 256 rows: no fused kernel, the runner uses the two plain calls and says so."""
+    """More than 512 rows: no fused kernel, the runner uses the two plain calls and says so."""
     cfg = wl.shrink(wl.CONFIGS["cfg3"], d=128, V=4096, prefix_scale=0.02, name="fused_fallback")
-    inp = wl.make_step(cfg, allocator=orc.ref_schedule_greedy)
+    inp = wl.make_step(cfg, gamma=np.full(32, 16))
     dev = to_dev(inp)
-    assert dev["H"].shape[0] > 256
+    assert dev["H"].shape[0] > 512
     rnd = VerifyRound.for_inputs(dev, C=256)
     ran = rnd.head_accept_fused(dev["H"], dev["W"], dev["q_probs"], dev["draft_tok"], dev["cu_q"],
                                 dev["u_accept"], dev["u_sample"], inp["tau"])

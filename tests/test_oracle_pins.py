@@ -254,6 +254,40 @@ def test_inverse_cdf_convention():
     assert orc.ref_inverse_cdf(7.0 * w, 0.35)[0] == 3
 
 
+def test_inverse_cdf_without_an_index_takes_the_last_token_with_mass():
+    """Threshold at (or, by rounding, beyond) the total mass: no prefix sum exceeds it, and the draw
+    is the last token that has mass, never a trailing zero-mass token.  Expected values by hand."""
+    w = np.array([0.0, 0.2, 0.0, 0.3, 0.5, 0.0])           # prefix sums .0 .2 .2 .5 1. 1.: none > 1.0
+    v, m = orc.ref_inverse_cdf(w, 1.0)
+    assert v == 4 and m == 0.0
+    assert orc.ref_inverse_cdf(np.array([3.0, 1.0, 0.0, 0.0]), 1.0)[0] == 1
+    assert orc.ref_inverse_cdf(np.array([0.0, 0.0, 2.0]), 1.0)[0] == 2
+    # a threshold beyond the total (u > 1 stands in for rounding) behaves the same
+    assert orc.ref_inverse_cdf(w, 1.0 + 1e-9)[0] == 4
+
+
+def test_residual_without_mass_falls_back_to_the_target_distribution():
+    """A draft row with q >= p everywhere leaves max(0, p - q) without mass; the correction token is
+    then drawn from p itself.  q = 1.5 p (unnormalised on purpose) gives ratio 2/3 for every token."""
+    p = np.array([0.2, 0.3, 0.5])
+    q = 1.5 * p
+    np.testing.assert_array_equal(orc.ref_residual(p, q), p)
+    np.testing.assert_array_equal(orc.ref_residual(p, p), p)           # q == p: the same fall-back
+    # one element with mass left: the ordinary residual, not the fall-back
+    np.testing.assert_allclose(orc.ref_residual(p, np.array([0.3, 0.45, 0.4])), [0.0, 0.0, 0.1], atol=1e-15)
+    # through the whole acceptance pass: u_accept = 0.9 > 2/3 rejects the first draft token, and the
+    # correction token follows p's CDF (.2, .5, 1.)
+    p2 = [0.6, 0.3, 0.1]
+    for u_smp, want in ((0.1, 0), (0.35, 1), (0.6, 2), (0.999, 2)):
+        out = _one_server([p, p2], [q], [1], [0.9], u_smp)
+        assert out["accepted"][0] == 0 and out["resampled"][0] == 1
+        np.testing.assert_allclose(out["ratio"], [2.0 / 3.0], rtol=1e-12)
+        assert list(out["out_tok"]) == [want, -1]
+    # u_accept below 2/3 accepts and the bonus token comes from the second row
+    out = _one_server([p, p2], [q], [1], [0.6], 0.65)
+    assert out["accepted"][0] == 1 and list(out["out_tok"]) == [1, 1]
+
+
 def _exact_output_law(p1, q1, p2_of, q2_of, V):
     """P(first output token = x) and P(s1 accepted, second output token = y), obtained by
     integrating the oracle's own decisions over the uniforms exactly: accept has measure
