@@ -158,6 +158,19 @@ def make_host_inputs(cfg, device):
 
 
 # ------------------------------------------------------------------------------------------------
+def config_dict(cfg, inp, n_gpus):
+    """What the workload is: the same keys and values in both arms."""
+    N = cfg.N
+    Tq = int(inp["cu_q"][-1])
+    return {"workload": cfg.name, "servers_per_gpu": N, "draft_tokens_per_gpu": int(inp["gamma"].sum()),
+            "verify_positions": Tq, "prefix": int(inp["prefix"][0]) if cfg.prefix_mode == "fixed" else
+            f"{int(inp['prefix'].min())}..{int(inp['prefix'].max())}", "d": cfg.d, "V": cfg.V,
+            "heads": f"{cfg.Hq}q/{cfg.Hkv}kv x {cfg.hd}", "temperature": float(inp["tau"]),
+            "parallelism": f"dp{n_gpus} over draft servers",
+            "l2": "inputs larger than L2: the head weight (1.5-2.1 GB) streams through L2 every step and evicts "
+                  "the KV cache and logits"}
+
+
 def run_reference(args, cfg, rank, world):
     """The CPU oracle as it stands, on a bounded sample of the same workload."""
     if rank != 0:
@@ -186,7 +199,8 @@ def run_reference(args, cfg, rank, world):
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": cfg.name, "note": "fp64 CPU oracle on host cores"},
+            "config": config_dict(cfg, host, args.gpus),
+            "arm": "fp64 CPU oracle on host cores, bounded sample of the workload (see cpu_baseline.sample)",
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -194,18 +208,35 @@ def run_reference(args, cfg, rank, world):
 
 
 # ------------------------------------------------------------------------------------------------
-def run_ours(args, cfg, rank, world, local_rank):
+def head_roofline(T, d, V, es, us, peak_hbm, peaks):
+    """The LM head against the roofline that binds it: time / max(t_HBM, t_tensor), with both raw
+    fractions.  Tensor peak: the measured bf16 burst figure (the kernel is timed alone, for tens of
+    milliseconds); the sustained figure is quoted beside it."""
+    by = d * V * es + T * V * 4 + T * d * es
+    fl = 2.0 * T * d * V
+    tf_burst = float(peaks.get("bf16_tflops", 1590.0))
+    tf_sust = float(peaks.get("bf16_tflops_sustained", 1400.0))
+    t_hbm = by / (peak_hbm * 1e9) * 1e6              # us
+    t_tc = fl / (tf_burst * 1e12) * 1e6
+    gbs, tfs = by / us / 1e3, fl / us / 1e6
+    tensor = t_tc > t_hbm
+    return {"bound": "tensor" if tensor else "hbm",
+            "achieved": tfs if tensor else gbs, "peak": tf_burst if tensor else peak_hbm,
+            "unit": "TFLOP/s" if tensor else "GB/s", "frac": (tfs / tf_burst) if tensor else (gbs / peak_hbm),
+            "frac_of_binding_roofline": max(t_hbm, t_tc) / us,
+            "frac_hbm": gbs / peak_hbm, "frac_bf16_burst": tfs / tf_burst, "frac_bf16_sustained": tfs / tf_sust,
+            "t_hbm_us": t_hbm, "t_tensor_us": t_tc, "duration_us": us, "algorithmic_bytes": by, "flops": fl,
+            "gbs": gbs, "tensor_tflops": tfs}
+
+
+def measure_config(args, cfg, rank, world, local_rank, steps, warmup, detail):
+    """One workload on this rank's GPU: W warm-up steps, K timed steps, per-kernel durations.
+    detail=True adds the end-to-end leg, the CPU baseline and the parity check (single GPU only)."""
     from paper_2512_09963_b200 import binding as B
-    from paper_2512_09963_b200 import build as gs_build
     from paper_2512_09963_b200.runner import VerifyRound
+    from paper_2512_09963_b200.sharded import ShardedScheduler, aggregate_throughput
     import torch.distributed as dist
 
-    if rank == 0:
-        gs_build.build()
-    if world > 1:
-        dist.barrier()
-    B.lib()
-    B.gs_set_dependent_launch(not args.no_dependent_launch)
     dev = torch.device("cuda", local_rank)
     cfg_r = dataclasses.replace(cfg, seed_tag=f"/rank{rank}") if world > 1 else cfg
     inp, host = make_host_inputs(cfg_r, dev)
@@ -214,15 +245,10 @@ def run_ours(args, cfg, rank, world, local_rank):
     C = cfg.C if cfg.C else 8 * N
     rnd = VerifyRound.for_inputs(inp, C=C, eta=ETA, beta=BETA)
     s_min = torch.ones(N * world, dtype=torch.int32, device=dev)
-    s_max = torch.full((N * world,), 8, dtype=torch.int32, device=dev)
+    s_max = torch.full((N * world,), max(8, cfg.gamma_hi), dtype=torch.int32, device=dev)
     # multi-GPU: servers are sharded over ranks; only the scheduler couples them, through an
     # all-gather of the estimator state (16 bytes per server) before every rank runs the same greedy.
-    if world > 1:
-        est_local = torch.empty(2 * N, dtype=torch.float64, device=dev)
-        est_all = torch.empty(2 * N * world, dtype=torch.float64, device=dev)
-        X_all = torch.empty(N * world, dtype=torch.float64, device=dev)
-        a_all = torch.empty(N * world, dtype=torch.float64, device=dev)
-        S_all = torch.empty(N * world, dtype=torch.int32, device=dev)
+    sharded = ShardedScheduler(N, rank, world, C * world, dev, s_min, s_max) if world > 1 else None
 
     def reset_state():
         rnd.alpha_hat.fill_(0.5)
@@ -230,9 +256,6 @@ def run_ours(args, cfg, rank, world, local_rank):
 
     # Does this shape have the LM head that writes the softmax statistics in its epilogue (then the
     # acceptance step does not read the logits a second time)?
-    # Measured on B200: the statistics cost the LM head 4-5 us (they sit in the epilogue of its last,
-    # not overlapped, tile) and save the acceptance step its pass over T_q x V logits: -0.5 % per step
-    # at 28 and 46 verify positions, -2.7 % at 87.
     fused = False
     if not args.no_fused_stats:
         fused = rnd.head_accept_fused(inp["H"], inp["W"], inp["q_probs"], inp["draft_tok"], inp["cu_q"],
@@ -266,14 +289,7 @@ def run_ours(args, cfg, rank, world, local_rank):
         if world == 1:
             rnd.schedule(s_min, s_max)
         else:
-            est_local[:N].copy_(rnd.alpha_hat)
-            est_local[N:].copy_(rnd.X)
-            dist.all_gather_into_tensor(est_all, est_local)
-            g = est_all.view(world, 2, N)
-            a_all.copy_(g[:, 0, :].reshape(-1))
-            X_all.copy_(g[:, 1, :].reshape(-1))
-            B.gs_schedule(X_all, a_all, C * world, S_all, s_min, s_max, rnd.d_status)
-            rnd.S_next.copy_(S_all[rank * N:(rank + 1) * N])
+            sharded.step(rnd.alpha_hat, rnd.X, rnd.S_next, rnd.d_status)
 
     # ---- launches per step and a first (eager) run
     reset_state()
@@ -298,7 +314,7 @@ def run_ours(args, cfg, rank, world, local_rank):
     run_step = graph.replay if graph is not None else step
 
     # ---- timed region: W warm-up steps, then exactly K steps between barriers/synchronisations
-    for _ in range(args.warmup):
+    for _ in range(warmup):
         run_step()
     torch.cuda.synchronize()
     if world > 1:
@@ -308,32 +324,22 @@ def run_ours(args, cfg, rank, world, local_rank):
     torch.cuda.synchronize()
     t_wall0 = time.time()
     e0.record()
-    for _ in range(args.steps):
+    for _ in range(steps):
         run_step()
     e1.record()
     torch.cuda.synchronize()
     t_wall1 = time.time()
     if world > 1:
         dist.barrier()
-    ms_total = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
-        g = torch.tensor([Gamma], dtype=torch.int64, device=dev)
-        dist.all_reduce(g)
-        gamma_all = int(g.item())
-    else:
-        gamma_all = Gamma
-    ms_step = ms_total / args.steps
+    ms_total, gamma_all = aggregate_throughput(e0.elapsed_time(e1), Gamma, dev)
+    ms_step = ms_total / steps
     clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
 
     # ---- per-kernel durations.  The LM head is long enough to be timed eagerly with events around
     # the call inside a running step sequence.  The short calls are timed as CUDA-graph replays of
     # [L2 flush; call] minus replays of [L2 flush] alone, so that neither the host's launch cost nor a
     # warm L2 enters the figure.
-    n_k = min(args.steps, 30)
-    names = ("verify_attn", "lm_head_logits", "spec_accept", "gs_schedule")
+    n_k = min(steps, 30)
     calls = {
         "verify_attn": lambda: rnd.attn(inp["Q"], inp["K"], inp["V"], inp["cu_q"], inp["cu_kv"]),
         "lm_head_logits": head_call,
@@ -384,40 +390,52 @@ def run_ours(args, cfg, rank, world, local_rank):
     base_us = replay_us(graph_of(None))
     for nme in ("verify_attn", "spec_accept", "gs_schedule"):
         k_us[nme] = max(replay_us(graph_of(calls[nme])) - base_us, 0.0)
-    k_us["lm_head_graph"] = max(replay_us(graph_of(calls["lm_head_logits"])) - base_us, 0.0)
     del flush_buf, flush_sink
 
-    if rank != 0:
-        return
     # ---- rooflines
     peak, peak_kind, peaks = _peaks()
     d, V = cfg.d, cfg.V
     es = 2 if cfg.dtype == "bf16" else 4
     total_kv = int(inp["K"].shape[0])
-    bytes_head = d * V * es + Tq * V * 4 + Tq * d * es
     bytes_attn = 2 * total_kv * cfg.Hkv * cfg.hd * es + 2 * Tq * cfg.Hq * cfg.hd * es
     # with the statistics from the LM head's epilogue the pass over all logits is gone
     bytes_acc = N * V * 8 if fused else Tq * V * 4 + N * V * 8
-    flops_head = 2.0 * Tq * d * V
-    ach = bytes_head / (k_us["lm_head_logits"] * 1e-6) / 1e9
+    bytes_acc_two_pass = Tq * V * 4 + N * V * 8
+    head = head_roofline(Tq, d, V, es, k_us["lm_head_logits"], peak, peaks)
     khash = _kernel_hash()
-    roofline = {"kernel": "lm_head_pair_kernel<1, true> (statistics epilogue)" if fused else "lm_head_pair_kernel", "bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s",
-                "frac": ach / peak, "peak_source": f"{peak_kind} (MEASURED_PEAKS.json hbm_gbs)" if peak_kind == "measured"
-                else "fallback 6650 GB/s", "traffic": NCU_TRAFFIC.get(khash, {}).get(cfg.name),
-                "algorithmic_bytes": bytes_head, "duration_us": k_us["lm_head_logits"],
-                "tensor_tflops": flops_head / (k_us["lm_head_logits"] * 1e-6) / 1e12}
+    roofline = {"kernel": ("lm_head_pair_kernel with the statistics epilogue" if fused else "lm_head_pair_kernel"),
+                "bound": head["bound"], "achieved": head["achieved"], "peak": head["peak"], "unit": head["unit"],
+                "frac": head["frac"],
+                "peak_source": (f"{peak_kind} (MEASURED_PEAKS.json " + ("bf16_tflops, burst" if head["bound"] == "tensor" else "hbm_gbs") + ")")
+                if peak_kind == "measured" else "fallback 6650 GB/s / 1590 TFLOP/s",
+                "traffic": NCU_TRAFFIC.get(khash, {}).get(cfg.name),
+                "algorithmic_bytes": head["algorithmic_bytes"], "duration_us": head["duration_us"],
+                "frac_of_binding_roofline": head["frac_of_binding_roofline"], "frac_hbm": head["frac_hbm"],
+                "frac_bf16_burst": head["frac_bf16_burst"], "frac_bf16_sustained": head["frac_bf16_sustained"],
+                "t_hbm_us": head["t_hbm_us"], "t_tensor_us": head["t_tensor_us"], "tensor_tflops": head["tensor_tflops"]}
     kernels = {
         "verify_attn": {"us": k_us["verify_attn"], "algorithmic_bytes": bytes_attn,
                         "gbs": bytes_attn / k_us["verify_attn"] / 1e3, "frac_hbm": bytes_attn / k_us["verify_attn"] / 1e3 / peak},
-        "lm_head_logits": {"us": k_us["lm_head_logits"], "algorithmic_bytes": bytes_head, "gbs": ach, "frac_hbm": ach / peak},
+        "lm_head_logits": {"us": k_us["lm_head_logits"], "algorithmic_bytes": head["algorithmic_bytes"], "gbs": head["gbs"],
+                           "bound": head["bound"], "frac_of_binding_roofline": head["frac_of_binding_roofline"],
+                           "frac_hbm": head["frac_hbm"], "frac_bf16_burst": head["frac_bf16_burst"],
+                           "frac_bf16_sustained": head["frac_bf16_sustained"]},
         "spec_accept": {"us": k_us["spec_accept"], "algorithmic_bytes": bytes_acc,
-                        "gbs": bytes_acc / k_us["spec_accept"] / 1e3, "frac_hbm": bytes_acc / k_us["spec_accept"] / 1e3 / peak},
+                        "gbs": bytes_acc / k_us["spec_accept"] / 1e3, "frac_hbm": bytes_acc / k_us["spec_accept"] / 1e3 / peak,
+                        "two_pass_bytes": bytes_acc_two_pass,
+                        "frac_hbm_on_two_pass_bytes": bytes_acc_two_pass / k_us["spec_accept"] / 1e3 / peak},
         "gs_schedule": {"us": k_us["gs_schedule"]},
     }
+    out = {"cfg": cfg, "inp": inp, "host": host, "rnd": rnd, "first": first, "N": N, "Tq": Tq, "Gamma": Gamma, "C": C,
+           "ms_step": ms_step, "gamma_all": gamma_all, "clocks": clocks, "kernels": kernels, "roofline": roofline,
+           "fused": fused, "graph": graph is not None, "launches_per_step": int(launches_per_step), "khash": khash,
+           "s_min": s_min, "s_max": s_max, "step": step, "reset_state": reset_state, "total_kv": total_kv,
+           "e2e": None, "cpu": None, "parity": None}
+    if not detail or world > 1:
+        return out
 
     # ---- end to end through the host-buffer entry point (pinned inputs, results read back each step)
-    e2e = None
-    if world == 1 and not args.profile_small:
+    if not args.profile_small:
         desc = B.RoundDesc(N=N, Tq=Tq, total_kv=total_kv, max_kv_len=rnd.max_kv_len, Hq=cfg.Hq, Hkv=cfg.Hkv,
                            hd=cfg.hd, d=d, V=V, C=C, dt=B.GS_BF16 if cfg.dtype == "bf16" else B.GS_F32,
                            scale=cfg.hd ** -0.5, temperature=float(inp["tau"]), eta=ETA, beta=BETA,
@@ -441,26 +459,25 @@ def run_ours(args, cfg, rank, world, local_rank):
         e2e_step()
         e2e_ok = (int(outs["status"][0]) == 0 and torch.equal(outs["accepted"], first["accepted"].cpu())
                   and torch.equal(outs["out_tok"], first["out_tok"].cpu()))
-        n_e = min(args.steps, 30)
+        n_e = min(steps, 30)
         for _ in range(3):
             e2e_step()
         t0 = time.time()
         for _ in range(n_e):
             e2e_step()
         dt = (time.time() - t0) / n_e
-        e2e = {"value": Gamma / dt, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-               "ms_per_step": dt * 1e3, "matches_device_path": bool(e2e_ok)}
+        out["e2e"] = {"value": Gamma / dt, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                      "ms_per_step": dt * 1e3, "matches_device_path": bool(e2e_ok)}
+        del ws
 
     # ---- CPU baseline = the oracle on the host cores, and a parity check of this launch configuration
-    cpu = None
-    parity = None
-    if world == 1 and not args.skip_cpu_baseline:
+    if not args.skip_cpu_baseline:
         import parity_utils as pu
         t0 = time.time()
         ref = oracle_round(host, N, C)
         dt = time.time() - t0
-        cpu = {"value": Gamma / dt, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "seconds": dt,
-               "sample": f"the whole {cfg.name} step once ({Gamma} draft tokens, {Tq} verify positions)"}
+        out["cpu"] = {"value": Gamma / dt, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "seconds": dt,
+                      "sample": f"the whole {cfg.name} step once ({Gamma} draft tokens, {Tq} verify positions)"}
         got = {k: first[k].cpu().numpy() for k in ("accepted", "out_tok", "n_out")}
         reset_state()
         step()
@@ -474,28 +491,111 @@ def run_ours(args, cfg, rank, world, local_rank):
             with contextlib.redirect_stdout(sys.stderr):       # the near-tie lines go to stderr; stdout carries the JSON line only
                 log = pu.compare_accept(got, ref, ref["logits"], host["q_probs"], host["cu_q"].numpy(),
                                         host["u_sample"], tau, V, slack=slack)
-            parity = {"status": "ok", "near_tie_band": pu.NEAR_TIE + slack, **pu.log_for_json(log)}
+            out["parity"] = {"status": "ok", "near_tie_band": pu.NEAR_TIE + slack, **pu.log_for_json(log)}
         except AssertionError as ex:
-            parity = {"status": "FAILED", "detail": str(ex)[:300]}
+            out["parity"] = {"status": "FAILED", "detail": str(ex)[:300]}
+    return out
 
+
+def run_ours(args, cfg, rank, world, local_rank):
+    from paper_2512_09963_b200 import binding as B
+    from paper_2512_09963_b200 import build as gs_build
+    import torch.distributed as dist
+
+    if rank == 0:
+        gs_build.build()
+    if world > 1:
+        dist.barrier()
+    B.lib()
+    B.gs_set_dependent_launch(not args.no_dependent_launch)
+    m = measure_config(args, cfg, rank, world, local_rank, args.steps, args.warmup, detail=True)
+    ms_step, first, inp = m["ms_step"], m["first"], m["inp"]
     goodput = float(first["n_out"].sum().item()) * world / (ms_step * 1e-3)
+    config = config_dict(cfg, m["host"], world)
+    launch_info = {"launch": "CUDA graph replay of the four calls" if m["graph"] else "eager, four calls per step",
+                   "softmax_statistics": "LM-head epilogue (gs_lm_head_logits_stats + gs_spec_accept_prestats)" if m["fused"]
+                   else "statistics pass of gs_spec_accept"}
+    # ---- the other single-GPU workloads, on the same box in the same run: step time and per-kernel rooflines
+    others = {}
+    extra = [] if (world > 1 or args.profile_small or args.only_headline) else [c for c in ("cfg3", "cfg4") if c != cfg.name]
+    del m["inp"], m["host"], m["rnd"], m["step"], m["reset_state"]
+    inp = None
+    for name in extra:
+        torch.cuda.empty_cache()
+        c2 = wl.CONFIGS[name]
+        k = min(args.steps, 300)
+        m2 = measure_config(args, c2, rank, world, local_rank, k, args.warmup, detail=False)
+        others[name] = {"config": config_dict(c2, m2["host"], 1), "steps": k, "ms_per_step": m2["ms_step"],
+                        "value": m2["gamma_all"] / (m2["ms_step"] * 1e-3), "unit": UNIT,
+                        "goodput_tokens_per_s": float(m2["first"]["n_out"].sum().item()) / (m2["ms_step"] * 1e-3),
+                        "kernels": m2["kernels"], "lm_head_roofline": m2["roofline"], "clocks": m2["clocks"],
+                        "softmax_statistics": "LM-head epilogue" if m2["fused"] else "statistics pass of gs_spec_accept",
+                        "launches_per_step": m2["launches_per_step"]}
+        del m2
+    if rank != 0:
+        return
     line = {
-        "metric": METRIC, "value": gamma_all / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+        "metric": METRIC, "value": m["gamma_all"] / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
-        "config": {"workload": cfg.name, "servers_per_gpu": N, "draft_tokens_per_gpu": Gamma, "verify_positions": Tq,
-                   "prefix": int(inp["prefix"][0]), "d": d, "V": V, "heads": f"{cfg.Hq}q/{cfg.Hkv}kv x {cfg.hd}",
-                   "temperature": float(inp["tau"]), "parallelism": f"dp{world} over draft servers",
-                   "l2": "inputs larger than L2: the 1.56 GB head weight streams through L2 every step and evicts the KV cache and logits",
-                   "launch": "CUDA graph replay of the four calls" if graph is not None else "eager, four calls per step",
-                   "softmax_statistics": "LM-head epilogue (gs_lm_head_logits_stats + gs_spec_accept_prestats)" if fused
-                   else "statistics pass of gs_spec_accept"},
+        "config": config, "launch_info": launch_info,
         "goodput_tokens_per_s": goodput,
-        "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu, "e2e": e2e,
-        "gpu_launches": int(launches_per_step) * args.steps, "launches_per_step": int(launches_per_step),
-        "clocks": clocks, "parity_vs_oracle": parity, "kernel_source_hash": khash,
+        "roofline": m["roofline"], "kernels": m["kernels"], "cpu_baseline": m["cpu"], "e2e": m["e2e"],
+        "gpu_launches": m["launches_per_step"] * args.steps, "launches_per_step": m["launches_per_step"],
+        "clocks": m["clocks"], "parity_vs_oracle": m["parity"], "kernel_source_hash": m["khash"],
+        "configs": others,
     }
     print(json.dumps(line), flush=True)
+
+
+def run_rank_check(args, rank, world):
+    """`--rank-check`: the rank plumbing without the GPU work.  Every rank joins the process group
+    (gloo on host tensors when there is no CUDA device), runs the estimator exchange of
+    paper_2512_09963_b200.sharded on seeded estimates and rank 0 prints what it saw."""
+    import torch.distributed as dist
+    from paper_2512_09963_b200 import build as gs_build
+    from paper_2512_09963_b200.sharded import ShardedScheduler
+    use_cuda = torch.cuda.is_available() and torch.cuda.device_count() >= world
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    os.environ.setdefault("MASTER_PORT", "29511")
+    if world > 1:
+        dist.init_process_group("nccl" if use_cuda else "gloo", rank=rank, world_size=world)
+    if rank == 0:
+        gs_build.build()
+    if world > 1:
+        dist.barrier()
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0"))) if use_cuda else torch.device("cpu")
+    n, C = 8, 64
+    r = np.random.default_rng(7 + rank)
+    alpha = torch.from_numpy(r.uniform(0.3, 0.95, n)).to(dev)
+    X = torch.from_numpy(r.uniform(1.0, 6.0, n)).to(dev)
+    sched = ShardedScheduler(n, rank, world, C * world, dev)
+    mine = torch.empty(n, dtype=torch.int32, device=dev)
+    S_all = sched.step(alpha, X, mine)
+    seen = torch.zeros(world, dtype=torch.int64, device=dev)
+    seen[rank] = 1
+    if world > 1:
+        dist.all_reduce(seen)
+    if rank == 0:
+        print(json.dumps({"rank_check": True, "n_gpus": args.gpus, "world_size": world, "backend": "nccl" if use_cuda else "gloo",
+                          "ranks_seen": [i for i in range(world) if int(seen[i]) == 1], "servers_per_rank": n,
+                          "budget_total": C * world, "allocation": S_all.cpu().tolist(),
+                          "allocation_sum": int(S_all.sum().item())}), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def spawn_ranks(n):
+    """`--gpus N` without a launcher around it: start N ranks of this very command under torch's
+    launcher on this node and hand their exit code back."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *sys.argv[1:]]
+    return subprocess.call(cmd)
 
 
 def run_head_sweep(args, cfg, local_rank):
@@ -555,6 +655,11 @@ def main():
                     help="time gs_lm_head_logits alone for 16..2048 rows at the workload's d and V")
     ap.add_argument("--no-dependent-launch", action="store_true",
                     help="launch the kernels without the programmatic-dependent-launch attribute")
+    ap.add_argument("--only-headline", action="store_true",
+                    help="time the named workload only (the default run also times cfg3 and cfg4 at --gpus 1)")
+    ap.add_argument("--rank-check", action="store_true",
+                    help="start the ranks, run the estimator exchange of the sharded path on seeded estimates and "
+                         "print what rank 0 saw; no GPU work (gloo on host tensors when there is no CUDA device)")
     ap.add_argument("--profile-small", action="store_true",
                     help="profiling case: vocabulary cut to 32768 (W = 336 MB, still larger than L2), eager "
                          "launches, no CPU baseline and no end-to-end leg; for ncu --set full captures")
@@ -562,9 +667,14 @@ def main():
     if args.steps is None:
         args.steps = 2000 if args.impl == "ours" else 20
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and (args.impl == "ours" or args.rank_check):
+        sys.exit(spawn_ranks(args.gpus))             # no launcher around this process: start the ranks here
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.rank_check:
+        run_rank_check(args, rank, world)
+        return
     cfg = wl.CONFIGS[args.config]
     if args.profile_small:
         cfg = wl.shrink(cfg, V=32768, name=cfg.name + "_V32768")
