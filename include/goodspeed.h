@@ -95,6 +95,14 @@ size_t gs_verify_attn_workspace(int N, int Tq, int total_kv, int max_kv_len, int
  * splitting.  Results agree to rounding.  The workspace size depends
  * on it: set it before gs_verify_attn_workspace.  Errors: INVALID_ARG. */
 gs_status gs_verify_attn_configure(int tiles_per_split);
+/* Kernel choice of the tensor-core path (process-wide, not thread-safe).  0 = automatic: a batch with
+ * few (server, block of positions, KV head) groups runs one thread-block cluster of 2, 4 or 8 CTAs per
+ * group (each CTA takes a part of the group's keys, the parts are merged through distributed shared
+ * memory; the workspace is not touched), every other batch -- and any batch while a split size is
+ * forced by gs_verify_attn_configure -- runs persistent CTAs that walk the batch's items and merge
+ * KV splits through the workspace.  1 = always the persistent kernel; 2, 4, 8 = always clusters of that
+ * size.  Results agree to rounding.  Errors: INVALID_ARG. */
+gs_status gs_verify_attn_select(int variant);
 gs_status gs_verify_attn(const void* Q, const void* K, const void* V, void* O,
                          const int32_t* cu_q, const int32_t* cu_kv,
                          int N, int Tq, int total_kv, int max_kv_len, int Hq, int Hkv, int hd,
@@ -225,6 +233,10 @@ gs_status gs_spec_accept(const float* logits, const float* q_probs, const int32_
  * exponentials are grouped differently).
  */
 size_t gs_lm_head_stats_bytes(int T);
+/* 1 where the statistics epilogue is expected to make the round shorter than the separate statistics
+ * pass of gs_spec_accept (up to 256 rows: the extra epilogue work hides under the next tile's MMAs), 0
+ * where it is not (more rows: a single accumulator, every epilogue holds up the tensor core). */
+int gs_lm_head_stats_pays(int T);
 gs_status gs_lm_head_logits_stats(const void* H, const void* W, float* logits, int T, int d, int V,
                                   gs_dtype dt, float temperature, void* stats, size_t stats_bytes,
                                   int* n_chunk, void* ws, size_t ws_bytes, int32_t* d_status, void* stream);

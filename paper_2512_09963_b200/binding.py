@@ -37,6 +37,7 @@ SIGNATURES = {
     "gs_lm_head_select": (_i, [_i]),
     "gs_spec_accept_select": (_i, [_i]),
     "gs_verify_attn_configure": (_i, [_i]),
+    "gs_verify_attn_select": (_i, [_i]),
     "gs_schedule_select": (_i, [_i]),
     "gs_set_dependent_launch": (_i, [_i]),
     "gs_lm_head_logits": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _vp, _sz, _vp, _vp]),
@@ -48,6 +49,7 @@ SIGNATURES = {
                                      _vp, _vp, _vp, _vp, _vp, _vp,
                                      _vp, _vp, _d, _d, _d, _d, _vp, _i, _vp, _sz, _vp, _vp]),
     "gs_lm_head_stats_bytes": (_sz, [_i]),
+    "gs_lm_head_stats_pays": (_i, [_i]),
     "gs_lm_head_logits_stats": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _f, _vp, _sz, C.POINTER(C.c_int),
                                      _vp, _sz, _vp, _vp]),
     "gs_spec_accept_static_capacity": (_sz, []),
@@ -138,6 +140,10 @@ def gs_verify_attn_configure(tiles_per_split: int = 0):
     _check("gs_verify_attn_configure", lib().gs_verify_attn_configure(int(tiles_per_split)))
 
 
+def gs_verify_attn_select(variant: int = 0):
+    _check("gs_verify_attn_select", lib().gs_verify_attn_select(int(variant)))
+
+
 def gs_verify_attn(Q, K, V, O, cu_q, cu_kv, max_kv_len, scale, ws, d_status=None):
     Tq, Hq, hd = Q.shape
     total_kv, Hkv, _ = K.shape
@@ -209,6 +215,11 @@ GS_ERR_UNSUPPORTED = 3
 
 def gs_lm_head_stats_bytes(T) -> int:
     return lib().gs_lm_head_stats_bytes(int(T))
+
+
+def gs_lm_head_stats_pays(T) -> bool:
+    """Whether the statistics epilogue is expected to beat the separate statistics pass at T rows."""
+    return bool(lib().gs_lm_head_stats_pays(int(T)))
 
 
 def gs_lm_head_logits_stats(H, W, logits, temperature, stats, ws, d_status=None):

@@ -198,8 +198,10 @@ class ClosedLoop:
                              1.0 / math.sqrt(cfg.hd), self.ws_attn, self.d_status)
         # the LM head writes the softmax statistics itself (when the shape has that kernel) and the
         # acceptance step skips its pass over the logits
-        n_chunk = B.gs_lm_head_logits_stats(inp["H"], inp["W"], logits, inp["tau"], self.stats, self.ws_head,
-                                            self.d_status)
+        n_chunk = None
+        if B.gs_lm_head_stats_pays(Tq):
+            n_chunk = B.gs_lm_head_logits_stats(inp["H"], inp["W"], logits, inp["tau"], self.stats, self.ws_head,
+                                                self.d_status)
         done = False
         if n_chunk is not None:
             done = B.gs_spec_accept_prestats(logits, inp["q_probs"], inp["draft_tok"], inp["cu_q"], inp["u_accept"],

@@ -19,6 +19,14 @@
 // stores, tickets and merges overlap the next item's tiles.  CTAs are persistent and stride over the
 // items, which are enumerated longest cache first.  The caches may be contiguous or pages of a pool
 // named by a block table (a page is one tile).
+//
+// Small batches (fewer (server, position block, KV head) groups than half the SMs) run the CLUSTER
+// instantiation instead: one thread-block cluster of 2, 4 or 8 CTAs per group, CTA k taking the k-th
+// part of the group's visible tiles, exactly one item per CTA.  Each CTA leaves its unnormalised
+// (O, m, l) rows in its own shared memory (the K/V ring is free by then), the cluster meets at one
+// barrier, and CTA 0 merges the parts through distributed shared memory and stores the rows: no
+// workspace, no tickets, no clearing kernel, and a set-up that finds the CTA's one item with a single
+// round of loads.
 #pragma once
 #include "common.cuh"
 #include "sm100_ptx.cuh"
@@ -64,6 +72,7 @@ struct AttnTcParams {
   int tiles_per_chunk;      // KV tiles per split (upper bound; splits of a server are balanced)
   int min_split_tiles;      // a server is split only into parts of at least this many tiles
   int max_items;
+  int cluster;              // CLUSTER kernel: CTAs per group (2, 4 or 8); 0 for the persistent kernel
   float scale_log2;         // scale * log2(e)
 };
 
@@ -166,6 +175,133 @@ GS_DEVINL AttnItem attn_find_item(const AttnTcParams& P, const int32_t* cu_q, co
 
 static_assert(sizeof(AttnItem) * kAtItemCache <= kAtItemCacheBytes, "item cache too small");
 
+// CLUSTER kernel: part `split` of group `grp` of server i, whose first group is `gbase` (groups are
+// numbered server -> position block -> KV head).  Only the tiles that hold a key the block can see are
+// shared out, as evenly as possible; the first n_used = min(cluster, visible tiles) parts get one.
+GS_DEVINL AttnItem attn_cluster_item(const AttnTcParams& P, int i, int q0, int n_new, int k0, int Lkv, int gbase,
+                                     int grp, int split) {
+  AttnItem it;
+  const int rem = grp - gbase;
+  it.g = rem % P.Hkv; it.tg = rem / P.Hkv; it.split = split; it.server = i;
+  it.item_base = 0; it.nsplit = P.cluster; it.group = grp;
+  it.q_row0 = q0 + it.tg * P.TB;
+  it.n_t = min(P.TB, n_new - it.tg * P.TB);
+  it.kv0 = k0; it.Lkv = Lkv; it.L = Lkv - n_new;
+  const int last_key = it.L + it.tg * P.TB + it.n_t - 1;
+  const int vis = last_key / kAtTile + 1;
+  const int tb = vis / P.cluster, tr = vis % P.cluster;
+  it.tile0 = split * tb + min(split, tr);
+  it.n_tiles = tb + (split < tr ? 1 : 0);
+  it.n_used = min(P.cluster, vis);
+  it.valid = 1;
+  return it;
+}
+
+// Whole warp: finds the server that owns group `grp` (32 servers per step: one round of loads, a
+// shuffle scan of the servers' group counts, a vote) and writes the CTA's item.
+GS_DEVINL void attn_cluster_find_item(const AttnTcParams& P, int grp, int split, int lane, AttnItem* out) {
+  int carry = 0;
+  bool found = false;
+  for (int c = 0; c < P.N && !found; c += 32) {
+    const int i = c + lane;
+    int q0 = 0, n_new = 0, k0 = 0, Lkv = 0, groups = 0;
+    if (i < P.N) {
+      q0 = P.cu_q[i]; k0 = P.cu_kv[i];
+      n_new = P.cu_q[i + 1] - q0; Lkv = P.cu_kv[i + 1] - k0;
+      if (attn_server_ok(P, q0, n_new, k0, Lkv)) groups = ((n_new + P.TB - 1) / P.TB) * P.Hkv;
+    }
+    int inc = groups;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int a = __shfl_up_sync(0xffffffffu, inc, d);
+      if (lane >= d) inc += a;
+    }
+    const int excl = carry + inc - groups;
+    const bool mine = groups > 0 && grp >= excl && grp < excl + groups;
+    if (__ballot_sync(0xffffffffu, mine) != 0u) {
+      if (mine) *out = attn_cluster_item(P, i, q0, n_new, k0, Lkv, excl, grp, split);
+      found = true;
+    }
+    carry += __shfl_sync(0xffffffffu, inc, 31);
+  }
+  if (!found && lane == 0) out->valid = 0;
+}
+
+GS_DEVINL float4 ld_cluster_f32x4(uint32_t cluster_addr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(cluster_addr) : "memory");
+  return v;
+}
+GS_DEVINL float2 ld_cluster_f32x2(uint32_t cluster_addr) {
+  float2 v;
+  asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(cluster_addr) : "memory");
+  return v;
+}
+
+// CLUSTER kernel, after the first cluster barrier: this CTA's share of the merge of a group's parts.
+// The n_used CTAs that hold a part share the rows out: CTA k merges rows k, k + n_used, ...; its warp w
+// the w-th, (w + 10)-th ... of those; lane c4 owns 4 of the 128 head dims, so a row of one part is one
+// 512-byte access to that CTA's shared memory.  Every warp fetches all its rows (at most UN), arrives
+// at the second cluster barrier (its reads of the peers are done), then does the arithmetic and the
+// stores.  (Inlined on purpose: as a real call its stack frame lives in local memory, which is cold,
+// and the merge took 8 us longer.)
+template <int KMAX, int UN>
+GS_DEVINL void attn_cluster_merge(int R, int n_used, int G, int Hq, __nv_bfloat16* O, int q_row0, int g,
+                                                int rank, int warp, int lane, const uint8_t* smem_raw) {
+  constexpr int kWarps = kAtThreads / 32;
+  const uint32_t stage = smem_u32(smem_raw);
+  float4 v[UN][KMAX];
+  float2 ml[UN][KMAX];
+#pragma unroll
+  for (int u = 0; u < UN; ++u) {
+    const int row = rank + n_used * (warp + kWarps * u);
+#pragma unroll
+    for (int k = 0; k < KMAX; ++k) {
+      v[u][k] = make_float4(0.f, 0.f, 0.f, 0.f);
+      ml[u][k] = make_float2(-INFINITY, 0.f);
+      if (row < R && k < n_used) {          // warp-uniform
+        if (k == rank) {                       // this CTA's own part: plain shared-memory loads
+          const float* mine = reinterpret_cast<const float*>(smem_raw) + (size_t)row * kAtPartStride;
+          v[u][k] = *reinterpret_cast<const float4*>(mine + lane * 4);
+          ml[u][k] = *reinterpret_cast<const float2*>(mine + kAtHd);
+        } else {
+          const uint32_t a = map_to_cta(stage, (uint32_t)k) + (uint32_t)row * (kAtPartStride * 4u);
+          v[u][k] = ld_cluster_f32x4(a + (uint32_t)lane * 16u);
+          ml[u][k] = ld_cluster_f32x2(a + kAtHd * 4u);
+        }
+      }
+    }
+  }
+  cluster_arrive_release();
+#pragma unroll
+  for (int u = 0; u < UN; ++u) {
+    const int row = rank + n_used * (warp + kWarps * u);
+    if (row < R) {
+      float M = -INFINITY;
+#pragma unroll
+      for (int k = 0; k < KMAX; ++k) if (k < n_used) M = fmaxf(M, ml[u][k].x);
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      float L = 0.f;
+#pragma unroll
+      for (int k = 0; k < KMAX; ++k) {
+        if (k < n_used && ml[u][k].x > -INFINITY) {
+          const float wk = fast_exp2(ml[u][k].x - M);
+          L += ml[u][k].y * wk;
+          acc.x += v[u][k].x * wk; acc.y += v[u][k].y * wk; acc.z += v[u][k].z * wk; acc.w += v[u][k].w * wk;
+        }
+      }
+      const float inv = 1.f / L;
+      __nv_bfloat162 b0 = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
+      __nv_bfloat162 b1 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+      uint2 pk;
+      pk.x = *reinterpret_cast<uint32_t*>(&b0); pk.y = *reinterpret_cast<uint32_t*>(&b1);
+      __nv_bfloat16* orow2 = O + ((size_t)(q_row0 + row / G) * Hq + g * G + (row % G)) * kAtHd;
+      *reinterpret_cast<uint2*>(orow2 + lane * 4) = pk;
+    }
+  }
+}
+
 // 2^x on the FMA pipe (x <= 127): floor by the 1.5*2^23 trick, a cubic for 2^f on [0,1] (relative
 // error 9e-5, far below bf16 resolution) and an integer add to the exponent.  One softmax thread
 // needs 128 exponentials per tile and the special-function unit delivers 4 per clock per SM
@@ -194,6 +330,7 @@ __global__ void attn_zero_kernel(int* p, int n) {
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) p[i] = 0;
 }
 
+template <bool CLUSTER>
 __global__ void __launch_bounds__(kAtThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant__ CUtensorMap tmapV,
                const AttnTcParams P) {
@@ -216,7 +353,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
   // The offsets are read by every role for every item: keep them in shared memory when they fit.
   float* s_ml = reinterpret_cast<float*>(smem_raw + kAtStages * kAtKvBytes + 256);     // [128][2] row maximum, row sum
   int32_t* s_cu = reinterpret_cast<int32_t*>(smem_raw + kAtStages * kAtKvBytes + 256 + 1024);
-  const bool cached = P.N <= kAtMaxCached;
+  const bool cached = !CLUSTER && P.N <= kAtMaxCached;
   const int32_t* cu_q = cached ? s_cu : P.cu_q;
   const int32_t* cu_kv = cached ? s_cu + (P.N + 1) : P.cu_kv;
   // first item and first group of every server (exclusive prefix sums; entry N = number of items)
@@ -228,16 +365,25 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
   int32_t* s_order_w = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(s_gbase_w + (kAtMaxCached + 1)) + kAtItemCacheBytes);
   int32_t* s_tmp_cnt = s_order_w + kAtSortMax;
   int32_t* s_tmp_grp = s_tmp_cnt + kAtSortMax;
-  const bool sorted = P.N <= kAtSortMax;
+  const bool sorted = !CLUSTER && P.N <= kAtSortMax;
   const int32_t* s_order = sorted ? s_order_w : nullptr;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // The k-th item of this CTA.  The items are enumerated longest cache first and dealt out in rounds of
+  // gridDim.x; every other round runs backwards, so that the CTA that got the longest item of one round
+  // gets the shortest of the next (a plain stride would hand CTA 0 the longest item of every round).
+  // Ids past the end of the enumeration only occur in the last round, so the first one ends a CTA's walk.
+  auto item_id = [&](int k) -> long long {
+    const long long b = (k & 1) ? (long long)gridDim.x - 1 - blockIdx.x : (long long)blockIdx.x;
+    return (long long)k * gridDim.x + b;
+  };
   // The next kernel on the stream may set itself up on idle SMs right away (it still waits for this
   // grid to finish before it touches global memory).
   pdl_launch_dependents();
-  if ((base & 1023u) != 0) {                     // the operand layouts need a 1024-byte aligned base
+  const bool misaligned = (base & 1023u) != 0;   // the operand layouts need a 1024-byte aligned base
+  if (misaligned) {
     if (threadIdx.x == 0) set_status(P.d_status, GS_ERR_CUDA);
-    return;
+    if (!CLUSTER) return;                        // a cluster's CTAs all go on to the cluster barriers, without an item
   }
   if (threadIdx.x == 0) {
     mbar_init(bar(0), 4); mbar_init(bar(1), 4);
@@ -259,6 +405,39 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
   // The barrier and tensor-memory set-up above overlaps the tail of whatever runs before this kernel
   // on the stream; global memory is touched only after that work has finished.
   pdl_wait();
+  AttnItem* s_items = reinterpret_cast<AttnItem*>(s_gbase_w + (kAtMaxCached + 1));
+  // K and V of tile j of an item into ring stage st (one elected lane of the producer warp).
+  auto issue_tile = [&](const AttnItem& it, int j, uint32_t st) {
+    mbar_arrive_expect_tx(bar(kKvFull + st), kAtKvBytes);
+    const uint32_t dst = kv_base + st * kAtKvBytes;
+    // contiguous caches: the server's rows follow one another; paged caches: tile = page
+    const int key = (P.block_table == nullptr)
+                        ? it.kv0 + (it.tile0 + j) * kAtTile
+                        : P.block_table[(size_t)it.server * P.max_pages + it.tile0 + j] * kAtTile;
+    const int col = it.g * kAtHd;
+    tma_load_2d(dst, &tmapK, col, key, bar(kKvFull + st));
+    tma_load_2d(dst + kAtHalfBytes, &tmapK, col + 64, key, bar(kKvFull + st));
+    tma_load_2d(dst + 2 * kAtHalfBytes, &tmapV, col, key, bar(kKvFull + st));
+    tma_load_2d(dst + 3 * kAtHalfBytes, &tmapV, col + 64, key, bar(kKvFull + st));
+  };
+  int pre_issued = 0;          // CLUSTER: 1 once the producer warp has started the first tile's loads, before the CTA's first barrier
+  if (CLUSTER && warp == 0) {
+    // Exactly one item per CTA: part (blockIdx.x % cluster) of group (blockIdx.x / cluster), found with
+    // one round of loads.  The same warp initialised the barriers (its lane 0, above), so it starts the
+    // loads of the first tile at once, without waiting for the other warps (only the first: measured,
+    // asking for three tiles at once delays the one the first scores wait for).
+    __syncwarp();
+    if (misaligned) { if (lane == 0) s_items[0].valid = 0; }
+    else attn_cluster_find_item(P, (int)blockIdx.x / P.cluster, (int)blockIdx.x % P.cluster, lane, &s_items[0]);
+    __syncwarp();
+    const AttnItem it = s_items[0];
+    if (it.valid) {
+      pre_issued = min(it.n_tiles, 1);
+      if (elect_one())
+        for (int j = 0; j < pre_issued; ++j) issue_tile(it, j, (uint32_t)j);
+      __syncwarp();
+    }
+  }
   if (warp != 1 && cached) {
     const int t = (warp == 0) ? (int)threadIdx.x : (int)threadIdx.x - 32;      // every thread but the allocating warp's
     for (int i = t; i <= P.N; i += kAtThreads - 32) {
@@ -306,18 +485,19 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
       gcarry += __shfl_sync(0xffffffffu, ginc, 31);
     }
   }
-  __syncthreads();
-  // The descriptors of this CTA's first items, one thread each: a descriptor costs a dozen integer
-  // divisions, which every role would otherwise repeat, one after the other, at every item.
-  AttnItem* s_items = reinterpret_cast<AttnItem*>(s_gbase_w + (kAtMaxCached + 1));
-  if (warp == 3) {
-    const long long id = (long long)blockIdx.x + (long long)lane * gridDim.x;
-    AttnItem it;
-    it.valid = 0;
-    if (id < P.max_items) it = attn_find_item(P, cu_q, cu_kv, s_base, s_gbase, s_order, (int)id);
-    s_items[lane] = it;
+  if (!CLUSTER) {
+    __syncthreads();
+    // The descriptors of this CTA's first items, one thread each: a descriptor costs a dozen integer
+    // divisions, which every role would otherwise repeat, one after the other, at every item.
+    if (warp == 3) {
+      const long long id = item_id(lane);
+      AttnItem it;
+      it.valid = 0;
+      if (id < P.max_items) it = attn_find_item(P, cu_q, cu_kv, s_base, s_gbase, s_order, (int)id);
+      s_items[lane] = it;
+    }
+    __syncthreads();
   }
-  __syncthreads();
   auto item_at = [&](int k, int id) -> AttnItem {
     return k < kAtItemCache ? s_items[k] : attn_find_item(P, cu_q, cu_kv, s_base, s_gbase, s_order, id);
   };
@@ -326,48 +506,38 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
   const uint32_t tmem_Q = tmem_base + kAtColQ;
 
   // Every role walks the same item sequence and recomputes the item from the offsets.
-  if (warp == 0) {
-    if (blockIdx.x == 0 && lane > 0) {
-      // offsets only the device can vouch for: such servers are skipped everywhere and flagged here
-      for (int i = lane - 1; i < P.N; i += 31) {
-        const int q0 = P.cu_q[i], n_new = P.cu_q[i + 1] - q0;
-        const int k0 = P.cu_kv[i], Lkv = P.cu_kv[i + 1] - k0;
-        if (!attn_server_ok(P, q0, n_new, k0, Lkv)) {
-          set_status(P.d_status, GS_ERR_SHAPE);
-        } else if (P.block_table != nullptr) {
-          // every tile of the server must name a page of the pool (a bad entry would only read the
-          // tensor map's fill value, but the result would be meaningless)
-          for (int t = 0; t < (Lkv + kAtTile - 1) / kAtTile; ++t) {
-            const int pg = P.block_table[(size_t)i * P.max_pages + t];
-            if (pg < 0 || pg >= P.n_pages) set_status(P.d_status, GS_ERR_INVALID_ARG);
-          }
+  if (blockIdx.x == 0 && warp == 9) {
+    // offsets only the device can vouch for: such servers are skipped everywhere and flagged here, by a
+    // warp that has nothing to do until the first item ends
+    for (int i = lane; i < P.N; i += 32) {
+      const int q0 = P.cu_q[i], n_new = P.cu_q[i + 1] - q0;
+      const int k0 = P.cu_kv[i], Lkv = P.cu_kv[i + 1] - k0;
+      if (!attn_server_ok(P, q0, n_new, k0, Lkv)) {
+        set_status(P.d_status, GS_ERR_SHAPE);
+      } else if (P.block_table != nullptr) {
+        // every tile of the server must name a page of the pool (a bad entry would only read the
+        // tensor map's fill value, but the result would be meaningless)
+        for (int t = 0; t < (Lkv + kAtTile - 1) / kAtTile; ++t) {
+          const int pg = P.block_table[(size_t)i * P.max_pages + t];
+          if (pg < 0 || pg >= P.n_pages) set_status(P.d_status, GS_ERR_INVALID_ARG);
         }
       }
     }
     __syncwarp();
+  }
+  if (warp == 0) {
     // ------------------------------------------------ TMA producer (whole warp in the loops, one elected lane issues)
     {
-      uint32_t st = 0, ph = 0;
+      // CLUSTER: the first tiles are already on their way (stages 0 .. pre_issued-1)
+      uint32_t st = (uint32_t)pre_issued % kAtStages, ph = (pre_issued == kAtStages) ? 1u : 0u;
       bool ok = true;
-      for (int id = blockIdx.x, k_item = 0; id < P.max_items && ok; id += gridDim.x, ++k_item) {
-        const AttnItem it = item_at(k_item, id);
+      for (long long k_item = 0, id = item_id(0); id < P.max_items && ok && (!CLUSTER || k_item == 0); ++k_item, id = item_id((int)k_item)) {
+        const AttnItem it = item_at((int)k_item, (int)id);
         if (!it.valid) break;
         if (it.n_tiles == 0) continue;
-        for (int j = 0; j < it.n_tiles; ++j) {
+        for (int j = pre_issued; j < it.n_tiles; ++j) {
           if (!mbar_wait_warp(bar(kKvEmpty + st), ph ^ 1u, abort_flag)) { ok = false; break; }
-          if (elect_one()) {
-            mbar_arrive_expect_tx(bar(kKvFull + st), kAtKvBytes);
-            const uint32_t dst = kv_base + st * kAtKvBytes;
-            // contiguous caches: the server's rows follow one another; paged caches: tile = page
-            const int key = (P.block_table == nullptr)
-                                ? it.kv0 + (it.tile0 + j) * kAtTile
-                                : P.block_table[(size_t)it.server * P.max_pages + it.tile0 + j] * kAtTile;
-            const int col = it.g * kAtHd;
-            tma_load_2d(dst, &tmapK, col, key, bar(kKvFull + st));
-            tma_load_2d(dst + kAtHalfBytes, &tmapK, col + 64, key, bar(kKvFull + st));
-            tma_load_2d(dst + 2 * kAtHalfBytes, &tmapV, col, key, bar(kKvFull + st));
-            tma_load_2d(dst + 3 * kAtHalfBytes, &tmapV, col + 64, key, bar(kKvFull + st));
-          }
+          if (elect_one()) issue_tile(it, j, st);
           __syncwarp();
           if (++st == kAtStages) { st = 0; ph ^= 1u; }
         }
@@ -400,8 +570,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
       }
       __syncwarp();
     };
-    for (int id = blockIdx.x, k_item = 0; id < P.max_items && ok; id += gridDim.x, ++k_item) {
-      const AttnItem it = item_at(k_item, id);
+    for (long long k_item = 0, id = item_id(0); id < P.max_items && ok && (!CLUSTER || k_item == 0); ++k_item, id = item_id((int)k_item)) {
+      const AttnItem it = item_at((int)k_item, (int)id);
       if (!it.valid) break;
       if (it.n_tiles == 0) continue;
       // Q of this item sits in tensor memory (written by the softmax warps after they have
@@ -452,8 +622,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
     int n_item = 0, n_tile_total = 0;
     bool ok = true;
-    for (int id = blockIdx.x, k_item = 0; id < P.max_items && ok; id += gridDim.x, ++k_item) {
-      const AttnItem it = item_at(k_item, id);
+    for (long long k_item = 0, id = item_id(0); id < P.max_items && ok && (!CLUSTER || k_item == 0); ++k_item, id = item_id((int)k_item)) {
+      const AttnItem it = item_at((int)k_item, (int)id);
       if (!it.valid) break;
       if (it.n_tiles == 0) continue;
       const int R = it.n_t * P.G;
@@ -593,8 +763,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
     int n_item = 0, n_ticket = 0;
     bool ok = true;
-    for (int id = blockIdx.x, k_item = 0; id < P.max_items && ok; id += gridDim.x, ++k_item) {
-      const AttnItem it = item_at(k_item, id);
+    for (long long k_item = 0, id = item_id(0); id < P.max_items && ok && (!CLUSTER || k_item == 0); ++k_item, id = item_id((int)k_item)) {
+      const AttnItem it = item_at((int)k_item, (int)id);
       if (!it.valid) break;
       if (it.n_tiles == 0) continue;
       const int R = it.n_t * P.G;
@@ -604,7 +774,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
       if (!mbar_wait(bar(kOFull), (uint32_t)n_item & 1u, abort_flag)) { ok = false; break; }
       tc_fence_after();
       __nv_bfloat16* orow = P.O + ((size_t)(it.q_row0 + r / P.G) * P.Hq + it.g * P.G + (r % P.G)) * kAtHd;
-      float* out = P.part + ((size_t)id * kAtRows + r) * kAtPartStride;
+      // partial rows go to the workspace, or (CLUSTER) to this CTA's own shared memory: every tile of
+      // the item has been consumed by now, so the K/V ring is free
+      float* out = CLUSTER ? reinterpret_cast<float*>(smem_raw) + (size_t)r * kAtPartStride
+                           : P.part + ((size_t)id * kAtRows + r) * kAtPartStride;
       const bool single = (it.n_used == 1);            // the only split of its group: normalise and store
       const float inv1 = single ? 1.f / l_run : 1.f;
 #pragma unroll
@@ -636,8 +809,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(kODrained));          // the statistics were read before this point too
-      if (!single) {
-        if (row_ok) { out[kAtHd] = m_run; out[kAtHd + 1] = l_run; }
+      if (!single && row_ok) { out[kAtHd] = m_run; out[kAtHd + 1] = l_run; }
+      if (!CLUSTER && !single) {
         // One ticket per group: the CTA that takes the last one finds the other splits' rows
         // complete (their writers fenced before taking theirs) and merges them.  The tickets were
         // cleared by the kernel this one was launched behind: make sure that has finished.
@@ -737,6 +910,26 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
   }
   tc_fence_before();
   __syncthreads();
+  if (CLUSTER) {
+    // Every CTA of the cluster arrives here (every wait above is bounded), with its part of the group
+    // in its shared memory.  CTA 0 merges the parts that saw keys and stores the rows; the others
+    // stay until it has read them.
+    cluster_arrive_release();
+    cluster_wait_acquire();
+    const AttnItem it = s_items[0];
+    const int rank = (int)cluster_cta_rank();
+    const bool merging = it.valid && it.n_used > 1 && rank < it.n_used;      // uniform over the CTA
+    if (merging) {
+      // rows of a CTA: at most 128 / n_used; of a warp: a tenth of that, rounded up
+      const int R = it.n_t * P.G;
+      if (it.n_used <= 2) attn_cluster_merge<2, 7>(R, it.n_used, P.G, P.Hq, P.O, it.q_row0, it.g, rank, warp, lane, smem_raw);
+      else if (it.n_used <= 4) attn_cluster_merge<4, 5>(R, it.n_used, P.G, P.Hq, P.O, it.q_row0, it.g, rank, warp, lane, smem_raw);
+      else attn_cluster_merge<8, 3>(R, it.n_used, P.G, P.Hq, P.O, it.q_row0, it.g, rank, warp, lane, smem_raw);
+    } else {
+      cluster_arrive_release();
+    }
+    cluster_wait_acquire();
+  }
   if (threadIdx.x == 0 && *abort_flag) set_status(P.d_status, GS_ERR_TIMEOUT);
   if (warp == 1) {
     tc_fence_after();
@@ -751,10 +944,54 @@ inline int& attn_tiles_per_split_override() {
   return v;
 }
 
+// Kernel choice forced by gs_verify_attn_select: 0 = automatic, 1 = the persistent kernel, 2 / 4 / 8 =
+// the CLUSTER kernel with that many CTAs per group.
+inline int& attn_variant_override() {
+  static int v = 0;
+  return v;
+}
+
 struct AttnTcPlan {
   int TB, tiles_per_chunk, min_split_tiles, max_items, max_groups, grid;
+  int cluster;              // CTAs per group of the CLUSTER kernel, 0 = the persistent kernel
   size_t ticket_bytes, ws_bytes;
 };
+
+// Both kernels need more dynamic shared memory than the default limit: raised once per device.
+inline bool attn_set_attributes() {
+  static PerDeviceOnce attr_set;
+  const int slot = device_slot();
+  if (attr_set.needed(slot)) {
+    if (cudaFuncSetAttribute(attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAtSmem) != cudaSuccess ||
+        cudaFuncSetAttribute(attn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAtSmem) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return false;
+    }
+    attr_set.mark(slot);
+  }
+  return true;
+}
+
+// Clusters of `cs` attention CTAs (one CTA per SM) the device can hold at once; cached per device.
+inline int attn_max_clusters(int cs) {
+  static int cached[kMaxDevices][4] = {};
+  const int slot = device_slot();
+  const int idx = cs == 2 ? 0 : cs == 4 ? 1 : 2;
+  if (slot >= 0 && cached[slot][idx] != 0) return max(cached[slot][idx], 0);
+  if (!attn_set_attributes()) return 0;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(cs * sm_count()));
+  cfg.blockDim = dim3(kAtThreads);
+  cfg.dynamicSmemBytes = kAtSmem;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = (unsigned)cs; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, attn_tc_kernel<true>, &cfg) != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
+  if (slot >= 0) cached[slot][idx] = n > 0 ? n : -1;
+  return n;
+}
 
 inline bool attn_tc_supported(int Hq, int Hkv, int hd, gs_dtype dt) {
   if (dt != GS_BF16 || hd != kAtHd || Hkv <= 0 || Hq % Hkv != 0) return false;
@@ -787,6 +1024,18 @@ inline AttnTcPlan attn_tc_plan(int N, int Tq, int total_kv, int max_kv_len, int 
   pl.max_groups = (int)min((long long)Hkv * blocks, (long long)INT_MAX / 2);
   pl.ticket_bytes = align_up((size_t)pl.max_groups * sizeof(int), 256);
   pl.ws_bytes = pl.ticket_bytes + (size_t)pl.max_items * kAtRows * kAtPartStride * sizeof(float);
+  // Few groups (a small batch): one cluster per group, as wide as still lets every cluster of the
+  // expected number of groups be resident at once, and no wider than leaves a part two tiles.
+  pl.cluster = 0;
+  const int forced = attn_variant_override();
+  if (forced == 2 || forced == 4 || forced == 8) {
+    pl.cluster = forced;
+  } else if (forced == 0 && attn_tiles_per_split_override() == 0) {
+    const int avg_new = (Tq + max(1, N) - 1) / max(1, N);
+    const long long groups_est = (long long)N * Hkv * ((avg_new + pl.TB - 1) / pl.TB);
+    for (int cs = 8; cs >= 2 && pl.cluster == 0; cs >>= 1)
+      if (tiles_avg >= 2 * cs && groups_est * cs <= (long long)attn_max_clusters(cs) * cs) pl.cluster = cs;
+  }
   return pl;
 }
 
@@ -797,13 +1046,7 @@ inline gs_status launch_attn_tc(const void* Q, const void* K, const void* V, voi
                                 const int32_t* cu_kv, int N, int Tq, int total_kv, int max_kv_len, int Hq, int Hkv,
                                 float scale, void* ws, int32_t* d_status, cudaStream_t st,
                                 const int32_t* block_table = nullptr, int max_pages = 0, int n_pages = 0) {
-  static PerDeviceOnce attr_set;
-  const int slot = device_slot();
-  if (attr_set.needed(slot)) {
-    if (cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAtSmem) != cudaSuccess)
-      return GS_ERR_CUDA;
-    attr_set.mark(slot);
-  }
+  if (!attn_set_attributes()) return GS_ERR_CUDA;
   const AttnTcPlan pl = attn_tc_plan(N, Tq, total_kv, max_kv_len, Hq, Hkv);
   AttnTcParams P;
   P.cu_q = cu_q; P.cu_kv = cu_kv; P.d_status = d_status;
@@ -815,6 +1058,7 @@ inline gs_status launch_attn_tc(const void* Q, const void* K, const void* V, voi
   P.N = N; P.Tq = Tq; P.total_kv = total_kv; P.max_kv_len = max_kv_len; P.Hq = Hq; P.Hkv = Hkv;
   P.G = Hq / Hkv; P.TB = pl.TB; P.tiles_per_chunk = pl.tiles_per_chunk; P.min_split_tiles = pl.min_split_tiles;
   P.max_items = pl.max_items;
+  P.cluster = 0;
   P.scale_log2 = scale * kAtLog2e;
   auto enc = tensor_map_encoder();
   if (enc == nullptr) return GS_ERR_CUDA;
@@ -824,10 +1068,23 @@ inline gs_status launch_attn_tc(const void* Q, const void* K, const void* V, voi
   if (!make_tmap_bf16_2d(&tmK, K, kv_rows, (uint64_t)Hkv * kAtHd, (uint64_t)Hkv * kAtHd, kAtTile, 64) ||
       !make_tmap_bf16_2d(&tmV, V, kv_rows, (uint64_t)Hkv * kAtHd, (uint64_t)Hkv * kAtHd, kAtTile, 64))
     return GS_ERR_CUDA;
+  if (pl.cluster > 0 && (long long)pl.max_groups * pl.cluster < (long long)INT_MAX / 2) {
+    // one cluster per (server, position block, KV head) group, one item per CTA; groups beyond the
+    // batch's real number (the host only knows a bound) find no item and leave at once
+    P.cluster = pl.cluster;
+    P.max_items = pl.max_groups * pl.cluster;
+    if (launch_ex(attn_tc_kernel<true>, dim3((unsigned)P.max_items), dim3(kAtThreads), kAtSmem, st, true, pl.cluster, tmK, tmV,
+                  P) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return GS_ERR_CUDA;
+    }
+    count_launches(1);
+    return launch_status();
+  }
   const int n_ticket = (int)(pl.ticket_bytes / sizeof(int));
   attn_zero_kernel<<<(n_ticket + 1023) / 1024 > 64 ? 64 : (n_ticket + 1023) / 1024, 1024, 0, st>>>(P.tickets, n_ticket);
   if (cudaGetLastError() != cudaSuccess) return GS_ERR_CUDA;
-  if (launch_ex(attn_tc_kernel, dim3(pl.grid), dim3(kAtThreads), kAtSmem, st, true, 1, tmK, tmV, P) != cudaSuccess) {
+  if (launch_ex(attn_tc_kernel<false>, dim3(pl.grid), dim3(kAtThreads), kAtSmem, st, true, 1, tmK, tmV, P) != cudaSuccess) {
     (void)cudaGetLastError();
     return GS_ERR_CUDA;
   }

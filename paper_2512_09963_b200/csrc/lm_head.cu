@@ -467,6 +467,13 @@ extern "C" size_t gs_lm_head_stats_bytes(int T) {
   return gs::align_up((size_t)T * (size_t)gs::sm_count() * sizeof(gs::ChunkStat), 256);
 }
 
+/* Whether taking the statistics from the LM-head epilogue is expected to beat the separate statistics
+ * pass.  Up to 256 rows the accumulators are double-buffered and the extra epilogue work hides under
+ * the next tile's MMAs (measured: the round gets 0.5-3 % shorter); from 257 rows on the accumulator is
+ * single and every tile's epilogue, statistics included, holds up the tensor core (measured at 288 rows:
+ * LM head +104 us against 32 us saved in the acceptance step). */
+extern "C" int gs_lm_head_stats_pays(int T) { return (T > 0 && T <= 256) ? 1 : 0; }
+
 extern "C" gs_status gs_lm_head_logits_stats(const void* H, const void* W, float* logits, int T, int d, int V,
                                              gs_dtype dt, float temperature, void* stats, size_t stats_bytes,
                                              int* n_chunk, void* ws, size_t ws_bytes, int32_t* d_status,

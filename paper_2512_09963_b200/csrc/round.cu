@@ -141,9 +141,11 @@ extern "C" gs_status gs_verify_round_host(const gs_round_desc* r,
   // LM head with the softmax statistics in its epilogue where the shape has that kernel, so that the
   // acceptance step does not read the logits a second time; the plain pair of calls otherwise.
   int n_chunk = 0;
-  s = gs_lm_head_logits_stats(w + L.H, d_W, reinterpret_cast<float*>(w + L.logits), r->Tq, r->d, r->V, r->dt,
-                              r->temperature, w + L.stats, L.stats_bytes, &n_chunk, w + L.ws_head, L.ws_head_bytes,
-                              d_status, st);
+  s = GS_ERR_UNSUPPORTED;
+  if (gs_lm_head_stats_pays(r->Tq))
+    s = gs_lm_head_logits_stats(w + L.H, d_W, reinterpret_cast<float*>(w + L.logits), r->Tq, r->d, r->V, r->dt,
+                                r->temperature, w + L.stats, L.stats_bytes, &n_chunk, w + L.ws_head, L.ws_head_bytes,
+                                d_status, st);
   const bool have_stats = (s == GS_OK);
   if (s == GS_ERR_UNSUPPORTED)
     s = gs_lm_head_logits(w + L.H, d_W, reinterpret_cast<float*>(w + L.logits), r->Tq, r->d, r->V, r->dt,

@@ -10,6 +10,12 @@ extern "C" gs_status gs_verify_attn_configure(int tiles_per_split) {
   return GS_OK;
 }
 
+extern "C" gs_status gs_verify_attn_select(int variant) {
+  if (variant != 0 && variant != 1 && variant != 2 && variant != 4 && variant != 8) return GS_ERR_INVALID_ARG;
+  gs::attn_variant_override() = variant;
+  return GS_OK;
+}
+
 extern "C" size_t gs_verify_attn_workspace(int N, int Tq, int total_kv, int max_kv_len, int Hq, int Hkv,
                                            int hd, gs_dtype dt) {
   using namespace gs;

@@ -68,11 +68,15 @@ class VerifyRound:
                          self.eta, self.beta, self.alpha_min, self.alpha_max,
                          ws=self.ws_acc, d_status=self.d_status)
 
-    def head_accept_fused(self, H, W, q_probs, draft_tok, cu_q, u_accept, u_sample, tau, update=True) -> bool:
+    def head_accept_fused(self, H, W, q_probs, draft_tok, cu_q, u_accept, u_sample, tau, update=True,
+                          force=False) -> bool:
         """LM head with the softmax statistics in its epilogue, then the acceptance step on them (no
-        second pass over the logits).  Shapes without such kernels run the two plain calls.  Returns
-        whether the fused kernels ran."""
-        n_chunk = B.gs_lm_head_logits_stats(H, W, self.logits, tau, self.stats, self.ws_head, self.d_status)
+        second pass over the logits).  Shapes without such kernels, and shapes where the library
+        expects the separate statistics pass to be faster (gs_lm_head_stats_pays; force=True overrides
+        that), run the two plain calls.  Returns whether the fused kernels ran."""
+        n_chunk = None
+        if force or B.gs_lm_head_stats_pays(H.shape[0]):
+            n_chunk = B.gs_lm_head_logits_stats(H, W, self.logits, tau, self.stats, self.ws_head, self.d_status)
         if n_chunk is not None:
             if B.gs_spec_accept_prestats(self.logits, q_probs, draft_tok, cu_q, u_accept, u_sample, tau,
                                          self.accepted, self.out_tok, self.n_out, self.ratio, self.p_tok,

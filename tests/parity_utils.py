@@ -56,8 +56,7 @@ def compare_accept(gpu, ref, logits, q_probs, cu_q, u_sample, tau, V, slack=0.0)
     cu_q = np.asarray(cu_q, dtype=np.int64)
     N = len(cu_q) - 1
     log = {"accept_near_ties": [], "sample_near_ties": [], "sample_exact": 0, "servers": N}
-    logits64, q64 = np64(logits), np64(q_probs)
-    u_sample = np64(u_sample)
+    u_sample = np64(u_sample)      # logits and q_probs rows are widened only where a draw has to be re-examined
     for i in range(N):
         r0 = cu_q[i]
         gamma = int(cu_q[i + 1] - r0 - 1)
@@ -87,8 +86,8 @@ def compare_accept(gpu, ref, logits, q_probs, cu_q, u_sample, tau, V, slack=0.0)
             log["sample_exact"] += 1
             continue
         # not the oracle's token: is u within NEAR_TIE of the emitted token's CDF interval?
-        p = orc.ref_softmax_T(logits64[r0 + a_r], tau)
-        w = orc.ref_residual(p, q64[g0 + a_r]) if a_r < gamma else p
+        p = orc.ref_softmax_T(np64(logits[r0 + a_r]), tau)
+        w = orc.ref_residual(p, np64(q_probs[g0 + a_r])) if a_r < gamma else p
         F = np.cumsum(w)
         R = F[-1]
         lo = (F[tok_g - 1] if tok_g > 0 else 0.0) / R

@@ -425,6 +425,57 @@ def test_attention_small(name, cfg, attn_splits):
     assert torch.equal(O, O2)                     # deterministic
 
 
+@pytest.fixture(params=[2, 4, 8], ids=["clusters-of-2", "clusters-of-4", "clusters-of-8"])
+def attn_cluster(request):
+    """The cluster kernel forced for any batch: one cluster of that many CTAs per (server, position
+    block, KV head) group, parts merged through distributed shared memory."""
+    B.gs_verify_attn_select(request.param)
+    yield request.param
+    B.gs_verify_attn_select(0)
+
+
+@pytest.mark.parametrize("name,cfg", ATTN_CASES)
+def test_attention_cluster_kernel(name, cfg, attn_cluster):
+    inp = attn_case(cfg)
+    O, st = run_attn(inp)
+    assert st == 0
+    ref = orc.ref_attention(inp["Q"], inp["K"], inp["V"], inp["cu_q"], inp["cu_kv"])
+    pu.assert_close_rel(O, ref, f"attention {name}, clusters of {attn_cluster}")
+    O2, _ = run_attn(inp)
+    assert torch.equal(O, O2)                     # deterministic
+    B.gs_verify_attn_select(1)                    # the persistent kernel on the same inputs: equal to rounding
+    O3, _ = run_attn(inp)
+    pu.assert_close_rel(O, O3.float(), "cluster vs persistent kernel", rel=2e-2)
+
+
+def test_attention_cluster_kernel_edges_groups_pages(attn_cluster):
+    """The cluster kernel on the awkward shapes: a single key, empty prefixes, more CTAs than visible
+    tiles (parts without work), several position blocks per server, group sizes that do not divide
+    128, bad offsets, and paged caches."""
+    import dataclasses
+    base = wl.shrink(wl.CONFIGS["cfg2"], prefix_scale=0.0, N=4, name="attn_edge")
+    for gamma, prefix in (([0, 1, 16, 3], [1, 1, 1, 700]), ([2, 0, 5, 1], [0, 0, 0, 0]), ([40, 17, 0, 33], [300, 5, 1200, 130])):
+        inp = wl.make_attention_inputs(base, np.array(gamma), np.array(prefix))
+        O, st = run_attn(inp)
+        assert st == 0
+        pu.assert_close_rel(O, orc.ref_attention(inp["Q"], inp["K"], inp["V"], inp["cu_q"], inp["cu_kv"]), f"edge {gamma}")
+    for Hq, Hkv in ((40, 8), (7, 1), (128, 1)):
+        cfg = dataclasses.replace(wl.shrink(wl.CONFIGS["cfg2"], prefix_scale=0.12, N=3, name=f"attn_g{Hq}_{Hkv}"), Hq=Hq, Hkv=Hkv)
+        inp = wl.make_attention_inputs(cfg, np.array([8, 0, 30]), np.array([245, 130, 300]))
+        O, st = run_attn(inp)
+        assert st == 0
+        pu.assert_close_rel(O, orc.ref_attention(inp["Q"], inp["K"], inp["V"], inp["cu_q"], inp["cu_kv"]), f"G={Hq // Hkv}")
+    # a server with fewer keys than new positions: flagged, skipped, the other server is still right
+    cfg = wl.shrink(wl.CONFIGS["cfg2"], prefix_scale=0.05, N=2, name="attn_bad")
+    inp = wl.make_attention_inputs(cfg, np.array([2, 2]), np.array([50, 50]))
+    good = orc.ref_attention(inp["Q"], inp["K"], inp["V"], inp["cu_q"], inp["cu_kv"])
+    inp["cu_kv"] = inp["cu_kv"].clone()
+    inp["cu_kv"][1] = 1
+    O, st = run_attn(inp)
+    assert st == 2
+    assert bool(torch.isnan(O[:3].float()).all())          # server 0's rows were left unwritten
+
+
 @pytest.mark.parametrize("Hq,Hkv", [(40, 8), (6, 2), (4, 4), (7, 1), (128, 1)],
                          ids=["group-5", "group-3", "no-grouping", "group-7", "group-128"])
 def test_attention_group_sizes(Hq, Hkv):
@@ -439,7 +490,7 @@ def test_attention_group_sizes(Hq, Hkv):
     pu.assert_close_rel(O, orc.ref_attention(inp["Q"], inp["K"], inp["V"], inp["cu_q"], inp["cu_kv"]), f"G={Hq // Hkv}")
 
 
-@pytest.mark.parametrize("splits", [0, 2], ids=["auto-splits", "two-tile-splits"])
+@pytest.mark.parametrize("splits", [0, 2, -2, -4], ids=["auto-splits", "two-tile-splits", "clusters-of-2", "clusters-of-4"])
 def test_attention_paged_caches(splits):
     """gs_verify_attn_paged: the caches scattered over a pool of 128-row pages in shuffled order (with
     unused pages in between) give what the contiguous layout gives, i.e. the oracle's attention."""
@@ -469,7 +520,8 @@ def test_attention_paged_caches(splits):
     d = to_dev(inp)
     Tq, Hq, hd = d["Q"].shape
     max_len = int(lens.max())
-    B.gs_verify_attn_configure(splits)
+    B.gs_verify_attn_configure(max(splits, 0))
+    B.gs_verify_attn_select(-splits if splits < 0 else 1)
     try:
         ws = torch.empty(max(256, B.gs_verify_attn_paged_workspace(N, Tq, max_len, Hq, cfg.Hkv, hd, B.GS_BF16)),
                          dtype=torch.uint8, device=DEV)
@@ -481,6 +533,7 @@ def test_attention_paged_caches(splits):
         O2, _ = run_attn(inp)          # the contiguous layout under the same split plan
     finally:
         B.gs_verify_attn_configure(0)
+        B.gs_verify_attn_select(0)
     assert int(st.item()) == 0
     pu.assert_close_rel(O, orc.ref_attention(inp["Q"], inp["K"], inp["V"], inp["cu_q"], inp["cu_kv"]), "paged")
     assert torch.equal(O, O2)          # bit-identical to the contiguous layout (same tiles, same order)
@@ -572,7 +625,7 @@ def test_fused_head_statistics_match_two_pass(T_extra, d, V, tau):
     fused = VerifyRound.for_inputs(dev, C=4 * cfg.N)
     fused.attn(dev["Q"], dev["K"], dev["V"], dev["cu_q"], dev["cu_kv"])
     ran = fused.head_accept_fused(dev["H"], dev["W"], dev["q_probs"], dev["draft_tok"], dev["cu_q"],
-                                  dev["u_accept"], dev["u_sample"], inp["tau"])
+                                  dev["u_accept"], dev["u_sample"], inp["tau"], force=True)
     fused.schedule()
     torch.cuda.synchronize()
     assert ran, "this shape has the fused kernels"
