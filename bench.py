@@ -426,7 +426,31 @@ def measure_config(args, cfg, rank, world, local_rank, steps, warmup, detail):
                         "frac_hbm_on_two_pass_bytes": bytes_acc_two_pass / k_us["spec_accept"] / 1e3 / peak},
         "gs_schedule": {"us": k_us["gs_schedule"]},
     }
-    out = {"cfg": cfg, "inp": inp, "host": host, "rnd": rnd, "first": first, "N": N, "Tq": Tq, "Gamma": Gamma, "C": C,
+    # ---- the same head on a 4-bit weight (codes + per-group scales and zero points), timed alone: the
+    # weight stream is a quarter of the bf16 one
+    w4 = None
+    if detail and world == 1 and cfg.dtype == "bf16" and d % 128 == 0 and V % 16 == 0 and not args.profile_small:
+        layer = wl.make_w4_layer(cfg, 128, dev)
+        lg = torch.empty((min(Tq, 256), V), dtype=torch.float32, device=dev)
+        Hs = inp["H"][:min(Tq, 256)].contiguous()
+        f4 = lambda: B.gs_lm_head_logits_w4(Hs, layer["qweight"], layer["scales"], layer["zeros"], 128, lg, rnd.d_status)
+        for _ in range(3):
+            f4()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(20):                       # 390 MB of packed weights per launch: the inputs are cold
+            f4()
+        b.record()
+        torch.cuda.synchronize()
+        us4 = a.elapsed_time(b) * 1e3 / 20
+        Tw = lg.shape[0]
+        by4 = d * V // 2 + (d // 128) * V * 3 + Tw * V * 4 + Tw * d * 2
+        w4 = {"entry_point": "gs_lm_head_logits_w4", "rows": Tw, "group": 128, "us": us4, "algorithmic_bytes": by4,
+              "gbs": by4 / us4 / 1e3, "frac_hbm": by4 / us4 / 1e3 / peak, "bf16_head_us": k_us["lm_head_logits"],
+              "speedup_over_bf16_head": k_us["lm_head_logits"] / us4}
+        del layer, lg, Hs
+    out = {"cfg": cfg, "inp": inp, "host": host, "rnd": rnd, "first": first, "N": N, "Tq": Tq, "Gamma": Gamma, "C": C, "w4": w4,
            "ms_step": ms_step, "gamma_all": gamma_all, "clocks": clocks, "kernels": kernels, "roofline": roofline,
            "fused": fused, "graph": graph is not None, "launches_per_step": int(launches_per_step), "khash": khash,
            "s_min": s_min, "s_max": s_max, "step": step, "reset_state": reset_state, "total_kv": total_kv,
@@ -543,6 +567,7 @@ def run_ours(args, cfg, rank, world, local_rank):
         "roofline": m["roofline"], "kernels": m["kernels"], "cpu_baseline": m["cpu"], "e2e": m["e2e"],
         "gpu_launches": m["launches_per_step"] * args.steps, "launches_per_step": m["launches_per_step"],
         "clocks": m["clocks"], "parity_vs_oracle": m["parity"], "kernel_source_hash": m["khash"],
+        "lm_head_w4": m["w4"],
         "configs": others,
     }
     print(json.dumps(line), flush=True)

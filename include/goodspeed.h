@@ -161,6 +161,30 @@ gs_status gs_lm_head_logits(const void* H, const void* W, float* logits, int T, 
                             gs_dtype dt, void* ws, size_t ws_bytes, int32_t* d_status, void* stream);
 
 /* --------------------------------------------------------------------------------------------
+ * gs_lm_head_logits_w4 -- Sec. II-A1 with a 4-bit weight: the paper's larger target model is an
+ * AWQ-INT4 checkpoint (Sec. V: Llama3.1-70B-Instruct-AWQ-INT4); it names no storage format, this is
+ * the library's own.  The head weight W [d, V] is given as
+ *
+ *   qweight [d/8, V]     uint32   eight 4-bit codes per word, along d: the code of W[8w + j, v]
+ *                                 (j = 0..7) sits in bits [4n, 4n+4) of qweight[w, v] with
+ *                                 n = (j >> 1) + 4 (j & 1)  (nibbles 0..3 hold j = 0, 2, 4, 6 and
+ *                                 nibbles 4..7 hold j = 1, 3, 5, 7: a shift and one mask then yield
+ *                                 two neighbouring k in the two halves of a register)
+ *   scales  [d/group, V] bf16     one scale per group of `group` consecutive k and column
+ *   zeros   [d/group, V] uint8    the group's zero point, 0..15
+ *   W[k, v] = scales[k / group, v] * (code[k, v] - zeros[k / group, v])
+ *
+ *   H [T, d] bf16, logits [T, V] fp32 as gs_lm_head_logits:
+ *   logits[t, v] = sum_k H[t, k] * bf16(W[k, v])   -- every weight is rounded to bf16 once (the one
+ *   multiplication by the scale), products exact, accumulation fp32 on the tensor cores.
+ * Needs group % 64 == 0, d % group == 0, V % 16 == 0 and 16-byte aligned pointers (UNSUPPORTED
+ * otherwise).  No workspace.  More than 256 rows stream the weights once per 256 rows.
+ * Errors: INVALID_ARG, UNSUPPORTED, CUDA.  Device status: GS_ERR_TIMEOUT only.
+ */
+gs_status gs_lm_head_logits_w4(const void* H, const uint32_t* qweight, const void* scales, const uint8_t* zeros,
+                               int group, float* logits, int T, int d, int V, int32_t* d_status, void* stream);
+
+/* --------------------------------------------------------------------------------------------
  * gs_spec_accept -- Sec. II-A2 (acceptance rule, accepted count m, correction / bonus token),
  * with the estimator updates of Sec. III-C fused at its tail (Eq. updatealpha, Eq. updateX).
  *

@@ -13,6 +13,8 @@ before use.  Each function names the passage of the paper it restates:
                         attention formula, the textbook scaled-dot-product
                         definition with grouped KV heads is written out.
 * ref_lm_head        -- Sec. II-A1, P_M = softmax(W h): the W h product.
+* ref_dequant_w4     -- Sec. V names an AWQ-INT4 target: the 4-bit head weight, dequantised by
+                        its definition (scale * (code - zero)), then ref_lm_head as before.
 * ref_softmax_T      -- Sec. II-A1 softmax; temperature 0 is the "greedy
                         sampling ... argmax" case of the same paragraph.
 * ref_spec_accept    -- Sec. II-A2: accept s_j iff r_j <= p_j(s_j)/q_j(s_j);
@@ -102,6 +104,28 @@ def ref_lm_head(H, W, cols=None):
         else:
             W = np.asarray(W)[:, cols]
     return H @ _f64(W)
+
+
+def ref_dequant_w4(qweight, scales, zeros, group):
+    """The head weight of a 4-bit checkpoint, W[k, v] = scale[k // group, v] * (code[k, v] - zero[k // group, v]).
+
+    The paper's larger target is an AWQ-INT4 model (Sec. V) and gives no storage format; the format is
+    the library's, restated here from its definition: qweight [d/8, V] holds eight 4-bit codes per
+    32-bit word along d, the code of row 8w + j in bits [4n, 4n+4) of word [w, v] with
+    n = (j >> 1) + 4 (j & 1); scales [d/group, V]; zeros [d/group, V] in 0..15.  Returns W [d, V] float64
+    (exact: no rounding of the product).
+    """
+    qw = _i64(qweight) & 0xFFFFFFFF
+    scales, zeros = _f64(scales), _f64(zeros)
+    d8, V = qw.shape
+    W = np.empty((8 * d8, V))
+    for w in range(d8):
+        for j in range(8):
+            n = (j >> 1) + 4 * (j & 1)
+            k = 8 * w + j
+            code = (qw[w] >> (4 * n)) & 15
+            W[k] = scales[k // group] * (code.astype(F64) - zeros[k // group])
+    return W
 
 
 # --------------------------------------------------------------------------- #

@@ -41,6 +41,7 @@ SIGNATURES = {
     "gs_schedule_select": (_i, [_i]),
     "gs_set_dependent_launch": (_i, [_i]),
     "gs_lm_head_logits": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _vp, _sz, _vp, _vp]),
+    "gs_lm_head_logits_w4": (_i, [_vp, _vp, _vp, _vp, _i, _vp, _i, _i, _i, _vp, _vp]),
     "gs_spec_accept_workspace": (_sz, [_i, _i, _i]),
     "gs_spec_accept": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _f, _i, _i, _i,
                             _vp, _vp, _vp, _vp, _vp, _vp,
@@ -211,6 +212,20 @@ def gs_lm_head_logits(H, W, logits, ws, d_status=None):
 
 
 GS_ERR_UNSUPPORTED = 3
+
+
+def gs_lm_head_logits_w4(H, qweight, scales, zeros, group, logits, d_status=None):
+    """LM head on a 4-bit weight: qweight [d/8, V] int32 (eight codes per word along d), scales
+    [d/group, V] bf16, zeros [d/group, V] uint8 (see the header for the nibble order)."""
+    T, d = H.shape
+    V = qweight.shape[1]
+    if qweight.shape[0] * 8 != d or tuple(logits.shape) != (T, V) or tuple(scales.shape) != (d // group, V) \
+            or tuple(zeros.shape) != (d // group, V):
+        raise ValueError("shape mismatch")
+    code = lib().gs_lm_head_logits_w4(_ptr(H, torch.bfloat16), _ptr(qweight, torch.int32), _ptr(scales, torch.bfloat16),
+                                      _ptr(zeros, torch.uint8), int(group), _ptr(logits, torch.float32), T, d, V,
+                                      _ptr(d_status, torch.int32), _stream())
+    _check("gs_lm_head_logits_w4", code)
 
 
 def gs_lm_head_stats_bytes(T) -> int:

@@ -21,6 +21,7 @@
 #include "common.cuh"
 #include "attn_generic.cuh"
 #include "sm100_ptx.cuh"
+#include "lm_head_w4.cuh"
 
 namespace gs {
 
@@ -491,4 +492,20 @@ extern "C" gs_status gs_lm_head_logits_stats(const void* H, const void* W, float
   const float k2 = temperature > 0.f ? 1.4426950408889634f / temperature : 0.f;
   return launch_lm_head_pair(H, W, logits, T, d, V, d_status, g_head_mt, g_head_stages,
                              static_cast<cudaStream_t>(stream), static_cast<ChunkStat*>(stats), k2, sm_count(), n_chunk);
+}
+
+// ------------------------------------------------------------------------------------------------
+// gs_lm_head_logits_w4: the LM head on 4-bit weights (codes, per-group scales and zero points).
+extern "C" gs_status gs_lm_head_logits_w4(const void* H, const uint32_t* qweight, const void* scales,
+                                          const uint8_t* zeros, int group, float* logits, int T, int d, int V,
+                                          int32_t* d_status, void* stream) {
+  using namespace gs;
+  if (T < 0 || d < 0 || V < 0 || group <= 0) return GS_ERR_INVALID_ARG;
+  if (T == 0 || V == 0) return GS_OK;
+  if (!H || !qweight || !scales || !zeros || !logits) return GS_ERR_INVALID_ARG;
+  if (d == 0 || group % (int)kW4BlockK != 0 || d % group != 0 || V % 16 != 0) return GS_ERR_UNSUPPORTED;
+  if ((reinterpret_cast<uintptr_t>(H) | reinterpret_cast<uintptr_t>(qweight) | reinterpret_cast<uintptr_t>(scales) |
+       reinterpret_cast<uintptr_t>(zeros)) % 16 != 0)
+    return GS_ERR_UNSUPPORTED;
+  return launch_lm_head_w4(H, qweight, scales, zeros, group, logits, T, d, V, d_status, static_cast<cudaStream_t>(stream));
 }

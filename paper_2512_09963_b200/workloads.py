@@ -187,6 +187,19 @@ def make_layer(cfg: VerifyConfig, device="cpu"):
     return {"W": _normal(cfg, "W", 0, (cfg.d, cfg.V), cfg.d ** -0.5, torch_dtype(cfg), device)}
 
 
+def make_w4_layer(cfg: VerifyConfig, group: int = 128, device="cpu"):
+    """A synthetic 4-bit head weight in the library's storage format (include/goodspeed.h): random
+    codes (every bit of every word drawn uniformly), per-group scales around 1 / (4.6 sqrt(d)) (so
+    that the dequantised weight has about the variance 1/d of the bf16 layer) and zero points in
+    6..9.  Returns qweight [d/8, V] int32, scales [d/group, V] bf16, zeros [d/group, V] uint8."""
+    g = _tgen(cfg, "w4", 0, device)
+    qweight = torch.randint(-(1 << 31), (1 << 31), (cfg.d // 8, cfg.V), generator=g, device=device, dtype=torch.int64).to(torch.int32)
+    u = torch.rand((cfg.d // group, cfg.V), generator=g, device=device, dtype=torch.float32)
+    scales = ((0.75 + 0.5 * u) / (4.6 * cfg.d ** 0.5)).to(torch.bfloat16)
+    zeros = torch.randint(6, 10, (cfg.d // group, cfg.V), generator=g, device=device, dtype=torch.int64).to(torch.uint8)
+    return {"qweight": qweight.contiguous(), "scales": scales.contiguous(), "zeros": zeros.contiguous(), "group": group}
+
+
 def make_attention_inputs(cfg: VerifyConfig, gamma, prefix, round_idx=0, device="cpu"):
     """Q [T_q,H_q,hd], K/V [sum L_kv,H_kv,hd] ~ N(0,1) and the ragged offsets.
     L_kv,i = prefix_i + gamma_i + 1: the new positions' K/V are already appended."""

@@ -719,6 +719,67 @@ def test_lm_head_small(T, d, V, variant):
     pu.assert_close_rel(logits, ref, "logits (accumulation bar)", rel=2e-4)
 
 
+# ------------------------------------------------------------------ LM head on 4-bit weights
+@pytest.mark.parametrize("T,d,V,group", [(46, 512, 9008, 128), (96, 1024, 4112, 128), (1, 64, 16, 64), (130, 192, 1008, 64),
+                                         (256, 256, 2048, 128), (300, 128, 528, 128), (16, 5120, 4096, 128),
+                                         (144, 384, 20000, 128)])
+def test_lm_head_w4_small(T, d, V, group):
+    """gs_lm_head_logits_w4 against the oracle's dequantised weight and plain product: ragged vocabulary
+    tails, tiles of one to four units, one and two accumulator buffers, more than 256 rows (two
+    launches), the real model width."""
+    cfg = wl.shrink(wl.CONFIGS["cfg2"], d=d, V=V, name=f"w4_{T}_{d}_{V}")
+    layer = wl.make_w4_layer(cfg, group)
+    H = wl.make_hidden(cfg, T)
+    logits = torch.full((T, V), float("nan"), dtype=torch.float32, device=DEV)
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    B.gs_lm_head_logits_w4(H.to(DEV), layer["qweight"].to(DEV), layer["scales"].to(DEV), layer["zeros"].to(DEV), group,
+                           logits, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    W = orc.ref_dequant_w4(layer["qweight"], layer["scales"], layer["zeros"], group)
+    ref = orc.ref_lm_head(H, W)
+    pu.assert_close_rel(logits, ref, "logits on 4-bit weights")
+    # every weight is rounded to bf16 once (relative error up to 2^-9, mean square a third of that), the
+    # products are exact and the errors add up like a random walk: about 1.1e-3 of the row's rms per
+    # logit on average; the worst of a few hundred thousand elements reaches about ten times that
+    pu.assert_close_rel(logits, ref, "logits on 4-bit weights (rounding bar)", rel=1.5e-2)
+    logits2 = torch.empty_like(logits)
+    B.gs_lm_head_logits_w4(H.to(DEV), layer["qweight"].to(DEV), layer["scales"].to(DEV), layer["zeros"].to(DEV), group,
+                           logits2, st)
+    torch.cuda.synchronize()
+    assert torch.equal(logits, logits2)
+
+
+def test_lm_head_w4_feeds_the_acceptance_step():
+    """A round whose head weight is 4-bit: gs_lm_head_logits_w4 then gs_spec_accept, against the oracle on
+    its own dequantised product for the logits, and on the library's logits for the acceptance step."""
+    cfg = wl.shrink(wl.CONFIGS["cfg2"], d=512, V=8192, prefix_scale=0.02, name="w4_round")
+    inp = wl.make_step(cfg, gamma=[3, 1, 8, 2, 5, 4, 7, 6])
+    layer = wl.make_w4_layer(cfg, 128)
+    W = orc.ref_dequant_w4(layer["qweight"], layer["scales"], layer["zeros"], 128)
+    # drafts simulated from the 4-bit target's own logits
+    logits_sim = torch.from_numpy(orc.ref_lm_head(inp["H"], W)).float()
+    q, tok = wl.simulate_drafts(cfg, logits_sim, inp["cu_q"], inp["sigma"], inp["tau"])
+    inp["q_probs"], inp["draft_tok"] = q, tok
+    d = to_dev(inp)
+    rnd = VerifyRound.for_inputs(d, C=64)
+    B.gs_lm_head_logits_w4(d["H"], layer["qweight"].to(DEV), layer["scales"].to(DEV), layer["zeros"].to(DEV), 128,
+                           rnd.logits, rnd.d_status)
+    rnd.accept(d["q_probs"], d["draft_tok"], d["cu_q"], d["u_accept"], d["u_sample"], inp["tau"])
+    torch.cuda.synchronize()
+    assert int(rnd.d_status.item()) == 0
+    tau = tau32(inp["tau"])
+    pu.assert_close_rel(rnd.logits, orc.ref_lm_head(inp["H"], W), "logits on 4-bit weights")
+    # the acceptance step on the logits the library produced, widened to fp64: identical logits on both
+    # sides, so the strict band applies (the weights' bf16 rounding moves a logit by up to 1e-2, which as
+    # slack would swallow every decision)
+    got_logits = rnd.logits.cpu()
+    ref = orc.ref_spec_accept(got_logits, inp["q_probs"], inp["draft_tok"], inp["cu_q"], inp["u_accept"], inp["u_sample"], tau)
+    log = pu.compare_accept(pu.gpu_accept_dict(rnd), ref, got_logits, inp["q_probs"], inp["cu_q"].numpy(), inp["u_sample"],
+                            tau, cfg.V)
+    assert len(log["accept_near_ties"]) <= 1
+
+
 # ------------------------------------------------------------------ full-size configurations
 def _full_round(cfg_name, C, max_head_bytes=40e9):
     cfg = wl.CONFIGS[cfg_name]

@@ -122,6 +122,25 @@ def test_lm_head_selection_matrix_and_python_loops():
     np.testing.assert_allclose(orc.ref_lm_head(H, W, cols=[6, 1]), np.asarray(want)[:, [6, 1]], rtol=1e-14)
 
 
+def test_dequant_w4_hand_written_words():
+    """The 4-bit weight format on words written out by hand: nibble n of a word holds the code of row
+    offset j with n = (j >> 1) + 4 (j & 1), so 0x76543210 (nibble n holds n) reads, in row order,
+    0 4 1 5 2 6 3 7.  Two groups of 8 rows with different scales and zero points, two columns."""
+    qweight = np.array([[0x76543210, 0xFFFF0000],
+                        [0x89ABCDEF, 0x00000001]], dtype=np.uint32).view(np.int32)
+    scales = np.array([[0.5, 2.0], [0.25, 1.0]])
+    zeros = np.array([[3, 8], [8, 0]], dtype=np.uint8)
+    W = orc.ref_dequant_w4(qweight, scales, zeros, group=8)
+    assert W.shape == (16, 2)
+    np.testing.assert_array_equal(W[:8, 0], [-1.5, 0.5, -1.0, 1.0, -0.5, 1.5, 0.0, 2.0])       # 0.5 (code - 3)
+    np.testing.assert_array_equal(W[8:, 0], [1.75, 0.75, 1.5, 0.5, 1.25, 0.25, 1.0, 0.0])      # 0.25 ((15 11 14 10 13 9 12 8) - 8)
+    np.testing.assert_array_equal(W[:8, 1], [-16.0, 14.0] * 4)                                 # 2 ((0 15 0 15 ...) - 8)
+    np.testing.assert_array_equal(W[8:, 1], [1.0, 0, 0, 0, 0, 0, 0, 0])
+    # the head on it is the plain product with the dequantised weight
+    H = rng(21).standard_normal((3, 16))
+    np.testing.assert_allclose(orc.ref_lm_head(H, W), H @ W, rtol=1e-14)
+
+
 # -------------------------------------------------------------------- softmax
 def test_softmax_closed_forms():
     p = orc.ref_softmax_T(np.array([1.5, -0.5]), 0.5)
