@@ -39,9 +39,9 @@ ETA, BETA = 0.1, 0.5
 # per launch), keyed by the sha256 of the kernel source it was taken on; a changed kernel reports null.
 # cfg2's full launch is within ncu's single-pass size rule only for the launch list, so the counters
 # were taken on a smaller vocabulary and scale with the units processed (see profiles/).
-# small case (V = 32768), the kernel with the statistics epilogue: 336.085 MB read + 6.565 MB written
-# per launch, times 151936/32768
-NCU_TRAFFIC = {"26b8c6888d7758e0": {"cfg2": 1588769825}}
+# small case (V = 32768), the kernel with the statistics epilogue: 336.082 MB read + 3.849 MB written
+# per launch (part of the logits was still in L2 when the capture ended), times 151936/32768
+NCU_TRAFFIC = {"4722f17fd07b2b8e": {"cfg2": 1576166258}}
 
 
 def _kernel_hash():
@@ -637,6 +637,7 @@ def run_head_sweep(args, cfg, local_rank):
     W = wl.make_layer(cfg, dev)["W"]
     d, V = cfg.d, cfg.V
     rows_out = []
+    w4_layer = None
     for T in (16, 46, 96, 144, 256, 288, 512, 1024, 2048):
         H = wl.make_hidden(cfg, T, 0, dev)
         logits = torch.empty((T, V), dtype=torch.float32, device=dev)
@@ -655,12 +656,100 @@ def run_head_sweep(args, cfg, local_rank):
         by = d * V * 2 + T * V * 4 + T * d * 2
         fl = 2.0 * T * d * V
         gbs, tfs = by / us / 1e3, fl / us / 1e6
-        rows_out.append({"rows": T, "us": us, "GBps": gbs, "frac_hbm": gbs / peak_hbm, "TFLOPs": tfs,
-                         "frac_bf16_burst": tfs / tf_burst, "frac_bf16_sustained": tfs / tf_sust,
-                         "bound": "hbm" if by / peak_hbm / 1e3 > fl / tf_burst / 1e6 else "tensor"})
+        row = {"rows": T, "us": us, "GBps": gbs, "frac_hbm": gbs / peak_hbm, "TFLOPs": tfs,
+               "frac_bf16_burst": tfs / tf_burst, "frac_bf16_sustained": tfs / tf_sust,
+               "bound": "hbm" if by / peak_hbm / 1e3 > fl / tf_burst / 1e6 else "tensor"}
+        if T <= 256 and d % 128 == 0 and V % 16 == 0:      # the same rows on a 4-bit weight
+            if w4_layer is None:
+                w4_layer = wl.make_w4_layer(cfg, 128, dev)
+            f4 = lambda: B.gs_lm_head_logits_w4(H, w4_layer["qweight"], w4_layer["scales"], w4_layer["zeros"], 128, logits)
+            for _ in range(3):
+                f4()
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(n):
+                f4()
+            e1.record()
+            torch.cuda.synchronize()
+            us4 = e0.elapsed_time(e1) * 1e3 / n
+            by4 = d * V // 2 + (d // 128) * V * 3 + T * V * 4 + T * d * 2
+            row.update(w4_us=us4, w4_GBps=by4 / us4 / 1e3, w4_frac_hbm=by4 / us4 / 1e3 / peak_hbm)
+        rows_out.append(row)
         del H, logits, ws
     print(json.dumps({"head_sweep": rows_out, "d": d, "V": V, "peaks": {"hbm_gbs": peak_hbm, "bf16_tflops": tf_burst,
                                                                       "bf16_tflops_sustained": tf_sust, "source": kind}}), flush=True)
+
+
+def run_attn_sweep(args, local_rank):
+    """gs_verify_attn alone on every workload's attention inputs, per kernel choice: automatic, the
+    persistent kernel, clusters of 2 / 4 / 8.  Timed as CUDA-graph replays of [read 256 MB; call] minus
+    replays of [read 256 MB] alone (cold L2, no host launch cost), best of three."""
+    from paper_2512_09963_b200 import binding as B
+    from paper_2512_09963_b200 import build as gs_build
+    gs_build.build()
+    B.lib()
+    dev = torch.device("cuda", local_rank)
+    peak, kind, _ = _peaks()
+    flush_buf = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
+    sink = torch.zeros((), dtype=torch.int64, device=dev)
+
+    def graph_of(fn):
+        def body():
+            sink.copy_(flush_buf.view(torch.int64).sum())
+            if fn is not None:
+                fn()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            body()
+        torch.cuda.current_stream().wait_stream(side)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            body()
+        return g
+
+    def replay_us(g, n=30):
+        g.replay()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(n):
+            g.replay()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) * 1e3 / n
+
+    base = replay_us(graph_of(None))
+    rows = []
+    for name in ("cfg2", "cfg6", "cfg5", "cfg3", "cfg4"):
+        cfg = wl.CONFIGS[name]
+        if name == "cfg5":                      # one round of the closed loop at its first allocation, C / N drafts each
+            cfg = dataclasses.replace(cfg, gamma_mode="uniform", gamma_lo=cfg.C // cfg.N, gamma_hi=cfg.C // cfg.N)
+        alloc = library_allocator(dev) if cfg.gamma_mode == "alloc" else None
+        inp = wl.make_attention_inputs(cfg, wl.draw_gamma(cfg, allocator=alloc), wl.draw_prefix(cfg), device=dev)
+        Tq, Hq, hd = inp["Q"].shape
+        total_kv, Hkv, _ = inp["K"].shape
+        cu = inp["cu_kv"].cpu()
+        max_len, N = int((cu[1:] - cu[:-1]).max()), cu.numel() - 1
+        by = 2 * total_kv * Hkv * hd * 2 + 2 * Tq * Hq * hd * 2
+        O = torch.empty_like(inp["Q"])
+        st = torch.zeros(1, dtype=torch.int32, device=dev)
+        for variant in (0, 1, 2, 4, 8):
+            B.gs_verify_attn_select(variant)
+            ws = torch.empty(max(256, B.gs_verify_attn_workspace(N, Tq, total_kv, max_len, Hq, Hkv, hd, B.GS_BF16)),
+                             dtype=torch.uint8, device=dev)
+            call = lambda: B.gs_verify_attn(inp["Q"], inp["K"], inp["V"], O, inp["cu_q"], inp["cu_kv"], max_len, hd ** -0.5, ws, st)
+            c0 = B.gs_launch_count()
+            call()
+            torch.cuda.synchronize()
+            launches = B.gs_launch_count() - c0
+            assert int(st.item()) == 0
+            us = min(replay_us(graph_of(call)) - base for _ in range(3))
+            rows.append({"workload": name, "kernel": {0: "automatic", 1: "persistent", 2: "clusters of 2", 4: "clusters of 4",
+                                                      8: "clusters of 8"}[variant], "launches": int(launches), "us": us,
+                         "algorithmic_bytes": by, "GBps": by / us / 1e3, "frac_hbm": by / us / 1e3 / peak})
+        B.gs_verify_attn_select(0)
+    print(json.dumps({"attn_sweep": rows, "peak_hbm_gbs": peak, "peak_source": kind}), flush=True)
 
 
 def main():
@@ -678,6 +767,8 @@ def main():
                     help="plain gs_lm_head_logits + gs_spec_accept even where the LM head could write the softmax statistics")
     ap.add_argument("--head-sweep", action="store_true",
                     help="time gs_lm_head_logits alone for 16..2048 rows at the workload's d and V")
+    ap.add_argument("--attn-sweep", action="store_true",
+                    help="time gs_verify_attn alone on every workload's attention inputs, per kernel choice")
     ap.add_argument("--no-dependent-launch", action="store_true",
                     help="launch the kernels without the programmatic-dependent-launch attribute")
     ap.add_argument("--only-headline", action="store_true",
@@ -713,6 +804,10 @@ def main():
     if args.head_sweep:
         if rank == 0:
             run_head_sweep(args, cfg, local_rank)
+        return
+    if args.attn_sweep:
+        if rank == 0:
+            run_attn_sweep(args, local_rank)
         return
     if args.config == "cfg5":
         # closed-loop scheduling: Algorithm 1 for --rounds rounds with gs_schedule in the loop
