@@ -346,7 +346,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
   auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
   constexpr int kSFull = 2, kPFull = 4, kOFull = 6, kPvDone = 7, kKvFull = 8, kKvEmpty = 8 + kAtStages;
   constexpr int kEpiA = 8 + 2 * kAtStages, kEpiB = kEpiA + 1, kStatsFull = kEpiA + 2, kODrained = kEpiA + 3;
-  uint8_t* tail = smem_raw + (bars - base) + 8 * (12 + 2 * kAtStages);
+  // kv_full[s] counts the K half of a stage only; V has barriers of its own (v_full[S]), so that a tile's
+  // scores can start as soon as its keys are there (the values are needed a softmax later)
+  constexpr int kVFull = kODrained + 1;
+  uint8_t* tail = smem_raw + (bars - base) + 8 * (12 + 3 * kAtStages);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 4);
   volatile int* s_last = reinterpret_cast<volatile int*>(tail + 8);
@@ -390,7 +393,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
     mbar_init(bar(kSFull), 1); mbar_init(bar(kSFull + 1), 1);
     mbar_init(bar(kPFull), 4); mbar_init(bar(kPFull + 1), 4);
     mbar_init(bar(kOFull), 1); mbar_init(bar(kPvDone), 1);
-    for (int s = 0; s < kAtStages; ++s) { mbar_init(bar(kKvFull + s), 1); mbar_init(bar(kKvEmpty + s), 1); }
+    for (int s = 0; s < kAtStages; ++s) { mbar_init(bar(kKvFull + s), 1); mbar_init(bar(kKvEmpty + s), 1); mbar_init(bar(kVFull + s), 1); }
     mbar_init(bar(kEpiA), 128); mbar_init(bar(kEpiB), 128);
     mbar_init(bar(kStatsFull), 4); mbar_init(bar(kODrained), 4);
     *abort_flag = 0;
@@ -408,7 +411,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
   AttnItem* s_items = reinterpret_cast<AttnItem*>(s_gbase_w + (kAtMaxCached + 1));
   // K and V of tile j of an item into ring stage st (one elected lane of the producer warp).
   auto issue_tile = [&](const AttnItem& it, int j, uint32_t st) {
-    mbar_arrive_expect_tx(bar(kKvFull + st), kAtKvBytes);
+    mbar_arrive_expect_tx(bar(kKvFull + st), kAtKvBytes / 2);
+    mbar_arrive_expect_tx(bar(kVFull + st), kAtKvBytes / 2);
     const uint32_t dst = kv_base + st * kAtKvBytes;
     // contiguous caches: the server's rows follow one another; paged caches: tile = page
     const int key = (P.block_table == nullptr)
@@ -417,8 +421,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
     const int col = it.g * kAtHd;
     tma_load_2d(dst, &tmapK, col, key, bar(kKvFull + st));
     tma_load_2d(dst + kAtHalfBytes, &tmapK, col + 64, key, bar(kKvFull + st));
-    tma_load_2d(dst + 2 * kAtHalfBytes, &tmapV, col, key, bar(kKvFull + st));
-    tma_load_2d(dst + 3 * kAtHalfBytes, &tmapV, col + 64, key, bar(kKvFull + st));
+    tma_load_2d(dst + 2 * kAtHalfBytes, &tmapV, col, key, bar(kVFull + st));
+    tma_load_2d(dst + 3 * kAtHalfBytes, &tmapV, col + 64, key, bar(kVFull + st));
   };
   int pre_issued = 0;          // CLUSTER: 1 once the producer warp has started the first tile's loads, before the CTA's first barrier
   if (CLUSTER && warp == 0) {
@@ -452,6 +456,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  if (CLUSTER && !misaligned && !s_items[0].valid) {
+    // A group beyond the batch's real number (the grid is sized for a bound): the same holds for every
+    // CTA of this cluster, so all of them leave here, before any cluster barrier.  Such clusters are the
+    // last in launch order; the sooner they are gone, the sooner the grid is.
+    if (warp == 1) tmem_dealloc(*tmem_slot, kAtTmemCols);
+    return;
+  }
   if (sorted) {
     // Longest cache first: the CTAs' first items are then the largest ones and the short ones fill
     // in behind them, which evens out a ragged batch (cfg3: 79 -> 64 us).  Rank = servers with a
@@ -554,7 +565,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
     const uint64_t dv0 = smem_desc_sw128(kv_base + 2 * kAtHalfBytes, kAtHalfBytes, 1024u); // 64-column blocks one half apart
     // Two cursors walk the K/V ring: S = Q K^T runs one tile ahead of O += P V, so the tensor core
     // computes the next tile's scores while the softmax warps work on the current tile.
-    uint32_t st_s = 0, ph_s = 0, st_v = 0;
+    uint32_t st_s = 0, ph_s = 0, st_v = 0, ph_v = 0;
     int n_item = 0, n_tile_total = 0;
     bool ok = true;
     auto issue_S = [&](uint32_t stage, int n) {
@@ -595,6 +606,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
         if (j == 0 && n_item > 0) {      // the first product overwrites O: the previous item's O must have been read out
           if (!mbar_wait_warp(bar(kODrained), (uint32_t)(n_item - 1) & 1u, abort_flag)) { ok = false; break; }
         }
+        if (!mbar_wait_warp(bar(kVFull + st_v), ph_v, abort_flag)) { ok = false; break; }     // the tile's values have landed
         tc_fence_after();
         if (elect_one()) {
           const uint64_t dv = dv0 + (uint64_t)(st_v * (kAtKvBytes >> 4));
@@ -609,7 +621,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
           if (j + 1 == it.n_tiles) umma_commit(bar(kOFull));                 // O complete
         }
         __syncwarp();
-        if (++st_v == kAtStages) st_v = 0;
+        if (++st_v == kAtStages) { st_v = 0; ph_v ^= 1u; }
       }
       ++n_item;
     }
