@@ -35,7 +35,7 @@
 
 namespace gs {
 
-constexpr int kAtThreads = 320;          // warp 0 TMA, warp 1 MMA, warps 2-5 softmax, warps 6-9 epilogue
+constexpr int kAtThreads = 352;          // warp 0 TMA (keys), warp 1 MMA, warps 2-5 softmax, warps 6-9 epilogue, warp 10 TMA (values)
 constexpr int kAtTile = 128;             // keys per tile
 constexpr int kAtHd = 128;
 constexpr int kAtRows = 128;
@@ -346,10 +346,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
   auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
   constexpr int kSFull = 2, kPFull = 4, kOFull = 6, kPvDone = 7, kKvFull = 8, kKvEmpty = 8 + kAtStages;
   constexpr int kEpiA = 8 + 2 * kAtStages, kEpiB = kEpiA + 1, kStatsFull = kEpiA + 2, kODrained = kEpiA + 3;
-  // kv_full[s] counts the K half of a stage only; V has barriers of its own (v_full[S]), so that a tile's
-  // scores can start as soon as its keys are there (the values are needed a softmax later)
-  constexpr int kVFull = kODrained + 1;
-  uint8_t* tail = smem_raw + (bars - base) + 8 * (12 + 3 * kAtStages);
+  // kv_full[s] / kv_empty[s] belong to the K half of a stage only; the V half has barriers of its own
+  // (v_full[S], v_empty[S]) and a producer warp of its own.  A tile's keys are needed one softmax before
+  // its values and are done with as soon as its scores exist, so the K halves turn over faster than the V
+  // halves: more bytes in flight per SM than with whole stages that wait for the tile's second product.
+  constexpr int kVFull = kODrained + 1, kVEmpty = kVFull + kAtStages;
+  uint8_t* tail = smem_raw + (bars - base) + 8 * (12 + 4 * kAtStages);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 4);
   volatile int* s_last = reinterpret_cast<volatile int*>(tail + 8);
@@ -393,7 +395,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
     mbar_init(bar(kSFull), 1); mbar_init(bar(kSFull + 1), 1);
     mbar_init(bar(kPFull), 4); mbar_init(bar(kPFull + 1), 4);
     mbar_init(bar(kOFull), 1); mbar_init(bar(kPvDone), 1);
-    for (int s = 0; s < kAtStages; ++s) { mbar_init(bar(kKvFull + s), 1); mbar_init(bar(kKvEmpty + s), 1); mbar_init(bar(kVFull + s), 1); }
+    for (int s = 0; s < kAtStages; ++s) {
+      mbar_init(bar(kKvFull + s), 1); mbar_init(bar(kKvEmpty + s), 1);
+      mbar_init(bar(kVFull + s), 1); mbar_init(bar(kVEmpty + s), 1);
+    }
     mbar_init(bar(kEpiA), 128); mbar_init(bar(kEpiB), 128);
     mbar_init(bar(kStatsFull), 4); mbar_init(bar(kODrained), 4);
     *abort_flag = 0;
@@ -409,27 +414,32 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
   // on the stream; global memory is touched only after that work has finished.
   pdl_wait();
   AttnItem* s_items = reinterpret_cast<AttnItem*>(s_gbase_w + (kAtMaxCached + 1));
-  // K and V of tile j of an item into ring stage st (one elected lane of the producer warp).
-  auto issue_tile = [&](const AttnItem& it, int j, uint32_t st) {
-    mbar_arrive_expect_tx(bar(kKvFull + st), kAtKvBytes / 2);
-    mbar_arrive_expect_tx(bar(kVFull + st), kAtKvBytes / 2);
-    const uint32_t dst = kv_base + st * kAtKvBytes;
+  // K (or V) of tile j of an item into ring stage st (one elected lane of the producer warp).
+  auto tile_row = [&](const AttnItem& it, int j) -> int {
     // contiguous caches: the server's rows follow one another; paged caches: tile = page
-    const int key = (P.block_table == nullptr)
-                        ? it.kv0 + (it.tile0 + j) * kAtTile
-                        : P.block_table[(size_t)it.server * P.max_pages + it.tile0 + j] * kAtTile;
-    const int col = it.g * kAtHd;
+    return (P.block_table == nullptr) ? it.kv0 + (it.tile0 + j) * kAtTile
+                                      : P.block_table[(size_t)it.server * P.max_pages + it.tile0 + j] * kAtTile;
+  };
+  auto issue_k = [&](const AttnItem& it, int j, uint32_t st) {
+    mbar_arrive_expect_tx(bar(kKvFull + st), kAtKvBytes / 2);
+    const uint32_t dst = kv_base + st * kAtKvBytes;
+    const int key = tile_row(it, j), col = it.g * kAtHd;
     tma_load_2d(dst, &tmapK, col, key, bar(kKvFull + st));
     tma_load_2d(dst + kAtHalfBytes, &tmapK, col + 64, key, bar(kKvFull + st));
-    tma_load_2d(dst + 2 * kAtHalfBytes, &tmapV, col, key, bar(kVFull + st));
-    tma_load_2d(dst + 3 * kAtHalfBytes, &tmapV, col + 64, key, bar(kVFull + st));
+  };
+  auto issue_v = [&](const AttnItem& it, int j, uint32_t st) {
+    mbar_arrive_expect_tx(bar(kVFull + st), kAtKvBytes / 2);
+    const uint32_t dst = kv_base + st * kAtKvBytes + 2 * kAtHalfBytes;
+    const int key = tile_row(it, j), col = it.g * kAtHd;
+    tma_load_2d(dst, &tmapV, col, key, bar(kVFull + st));
+    tma_load_2d(dst + kAtHalfBytes, &tmapV, col + 64, key, bar(kVFull + st));
   };
   int pre_issued = 0;          // CLUSTER: 1 once the producer warp has started the first tile's loads, before the CTA's first barrier
   if (CLUSTER && warp == 0) {
     // Exactly one item per CTA: part (blockIdx.x % cluster) of group (blockIdx.x / cluster), found with
     // one round of loads.  The same warp initialised the barriers (its lane 0, above), so it starts the
-    // loads of the first tile at once, without waiting for the other warps (only the first: measured,
-    // asking for three tiles at once delays the one the first scores wait for).
+    // loads of the first tile's keys at once, without waiting for the other warps (only the first:
+    // measured, asking for three tiles at once delays the one the first scores wait for).
     __syncwarp();
     if (misaligned) { if (lane == 0) s_items[0].valid = 0; }
     else attn_cluster_find_item(P, (int)blockIdx.x / P.cluster, (int)blockIdx.x % P.cluster, lane, &s_items[0]);
@@ -438,7 +448,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
     if (it.valid) {
       pre_issued = min(it.n_tiles, 1);
       if (elect_one())
-        for (int j = 0; j < pre_issued; ++j) issue_tile(it, j, (uint32_t)j);
+        for (int j = 0; j < pre_issued; ++j) issue_k(it, j, (uint32_t)j);
       __syncwarp();
     }
   }
@@ -536,19 +546,24 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
     }
     __syncwarp();
   }
-  if (warp == 0) {
-    // ------------------------------------------------ TMA producer (whole warp in the loops, one elected lane issues)
+  if (warp == 0 || warp == 10) {
+    // ------------------------------------------------ TMA producers: warp 0 the keys, warp 10 the values
+    // (whole warp in the loops, one elected lane issues)
     {
-      // CLUSTER: the first tiles are already on their way (stages 0 .. pre_issued-1)
-      uint32_t st = (uint32_t)pre_issued % kAtStages, ph = (pre_issued == kAtStages) ? 1u : 0u;
+      const bool keys = (warp == 0);
+      const int first = keys ? pre_issued : 0;      // CLUSTER: the first tile's keys are already on their way (stage 0)
+      const int b_empty = keys ? kKvEmpty : kVEmpty;
+      uint32_t st = (uint32_t)first % kAtStages, ph = (first == kAtStages) ? 1u : 0u;
       bool ok = true;
       for (long long k_item = 0, id = item_id(0); id < P.max_items && ok && (!CLUSTER || k_item == 0); ++k_item, id = item_id((int)k_item)) {
         const AttnItem it = item_at((int)k_item, (int)id);
         if (!it.valid) break;
         if (it.n_tiles == 0) continue;
-        for (int j = pre_issued; j < it.n_tiles; ++j) {
-          if (!mbar_wait_warp(bar(kKvEmpty + st), ph ^ 1u, abort_flag)) { ok = false; break; }
-          if (elect_one()) issue_tile(it, j, st);
+        for (int j = first; j < it.n_tiles; ++j) {
+          if (!mbar_wait_warp(bar(b_empty + st), ph ^ 1u, abort_flag)) { ok = false; break; }
+          if (elect_one()) {
+            if (keys) issue_k(it, j, st); else issue_v(it, j, st);
+          }
           __syncwarp();
           if (++st == kAtStages) { st = 0; ph ^= 1u; }
         }
@@ -578,6 +593,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
           umma_bf16_ts(d, tmem_Q + (uint32_t)(kk * 8), b, idesc_s, kk > 0 ? 1u : 0u);
         }
         umma_commit(bar(kSFull + (n & 1)));                                  // S of tile n ready
+        umma_commit(bar(kKvEmpty + stage));                                  // and the tile's keys are done with
       }
       __syncwarp();
     };
@@ -616,7 +632,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
             const uint64_t b = dv + (uint64_t)(kk * (2048 >> 4));
             umma_bf16_ts(tmem_O, pn + (uint32_t)(kk * 8), b, idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
           }
-          umma_commit(bar(kKvEmpty + st_v));                                 // K/V stage free
+          umma_commit(bar(kVEmpty + st_v));                                  // the tile's values are done with
           umma_commit(bar(kPvDone));                                         // O holds tiles <= n
           if (j + 1 == it.n_tiles) umma_commit(bar(kOFull));                 // O complete
         }
@@ -767,7 +783,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
       if (lane == 0) mbar_arrive(bar(kStatsFull));
       ++n_item;
     }
-  } else {
+  } else if (warp < 10) {
     // ------------------------------------------------ epilogue: thread = row; runs one item behind
     // the softmax warps, so partial stores, tickets and merges overlap the next item's tiles
     const int q = warp & 3;
