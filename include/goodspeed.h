@@ -100,8 +100,9 @@ gs_status gs_verify_attn_configure(int tiles_per_split);
  * group (each CTA takes a part of the group's keys, the parts are merged through distributed shared
  * memory; the workspace is not touched), every other batch -- and any batch while a split size is
  * forced by gs_verify_attn_configure -- runs persistent CTAs that walk the batch's items and merge
- * KV splits through the workspace.  1 = always the persistent kernel; 2, 4, 8 = always clusters of that
- * size.  Results agree to rounding.  Errors: INVALID_ARG. */
+ * KV splits through the workspace.  A batch with no more groups than SMs, but too many for clusters,
+ * runs the cluster kernel with one CTA per group.  1 = always the persistent kernel; 2, 4, 8 = always
+ * clusters of that size; 3 = always one CTA per group.  Results agree to rounding.  Errors: INVALID_ARG. */
 gs_status gs_verify_attn_select(int variant);
 gs_status gs_verify_attn(const void* Q, const void* K, const void* V, void* O,
                          const int32_t* cu_q, const int32_t* cu_kv,

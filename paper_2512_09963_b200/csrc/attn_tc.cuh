@@ -973,7 +973,7 @@ inline int& attn_tiles_per_split_override() {
 }
 
 // Kernel choice forced by gs_verify_attn_select: 0 = automatic, 1 = the persistent kernel, 2 / 4 / 8 =
-// the CLUSTER kernel with that many CTAs per group.
+// the CLUSTER kernel with that many CTAs per group, 3 = the CLUSTER kernel with one CTA per group.
 inline int& attn_variant_override() {
   static int v = 0;
   return v;
@@ -1058,11 +1058,16 @@ inline AttnTcPlan attn_tc_plan(int N, int Tq, int total_kv, int max_kv_len, int 
   const int forced = attn_variant_override();
   if (forced == 2 || forced == 4 || forced == 8) {
     pl.cluster = forced;
+  } else if (forced == 3) {
+    pl.cluster = 1;
   } else if (forced == 0 && attn_tiles_per_split_override() == 0) {
     const int avg_new = (Tq + max(1, N) - 1) / max(1, N);
     const long long groups_est = (long long)N * Hkv * ((avg_new + pl.TB - 1) / pl.TB);
     for (int cs = 8; cs >= 2 && pl.cluster == 0; cs >>= 1)
       if (tiles_avg >= 2 * cs && groups_est * cs <= (long long)attn_max_clusters(cs) * cs) pl.cluster = cs;
+    // no more groups than SMs: still one item per CTA, so the same kernel with "clusters" of one CTA
+    // (its short set-up, no ticket-clearing launch) instead of the persistent one
+    if (pl.cluster == 0 && groups_est <= slots) pl.cluster = 1;
   }
   return pl;
 }

@@ -11,7 +11,7 @@ extern "C" gs_status gs_verify_attn_configure(int tiles_per_split) {
 }
 
 extern "C" gs_status gs_verify_attn_select(int variant) {
-  if (variant != 0 && variant != 1 && variant != 2 && variant != 4 && variant != 8) return GS_ERR_INVALID_ARG;
+  if (variant != 0 && variant != 1 && variant != 2 && variant != 3 && variant != 4 && variant != 8) return GS_ERR_INVALID_ARG;
   gs::attn_variant_override() = variant;
   return GS_OK;
 }

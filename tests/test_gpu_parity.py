@@ -425,7 +425,7 @@ def test_attention_small(name, cfg, attn_splits):
     assert torch.equal(O, O2)                     # deterministic
 
 
-@pytest.fixture(params=[2, 4, 8], ids=["clusters-of-2", "clusters-of-4", "clusters-of-8"])
+@pytest.fixture(params=[2, 4, 8, 3], ids=["clusters-of-2", "clusters-of-4", "clusters-of-8", "one-cta-per-group"])
 def attn_cluster(request):
     """The cluster kernel forced for any batch: one cluster of that many CTAs per (server, position
     block, KV head) group, parts merged through distributed shared memory."""
@@ -440,7 +440,7 @@ def test_attention_cluster_kernel(name, cfg, attn_cluster):
     O, st = run_attn(inp)
     assert st == 0
     ref = orc.ref_attention(inp["Q"], inp["K"], inp["V"], inp["cu_q"], inp["cu_kv"])
-    pu.assert_close_rel(O, ref, f"attention {name}, clusters of {attn_cluster}")
+    pu.assert_close_rel(O, ref, f"attention {name}, cluster kernel variant {attn_cluster}")
     O2, _ = run_attn(inp)
     assert torch.equal(O, O2)                     # deterministic
     B.gs_verify_attn_select(1)                    # the persistent kernel on the same inputs: equal to rounding
