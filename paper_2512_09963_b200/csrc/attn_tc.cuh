@@ -16,9 +16,12 @@
 // stores its rows directly; otherwise it writes an unnormalised partial (m, l, O) to the workspace
 // and takes a ticket, and the last split of a (server, position block, KV head) to finish merges
 // them (nobody waits).  Four more warps do that epilogue, one item behind the softmax warps, so
-// stores, tickets and merges overlap the next item's tiles.  CTAs are persistent and stride over the
-// items, which are enumerated longest cache first.  The caches may be contiguous or pages of a pool
-// named by a block table (a page is one tile).
+// stores, tickets and merges overlap the next item's tiles.  CTAs are persistent.  The items are
+// enumerated longest cache first; a CTA's first item is the one with its own index, every further one
+// is claimed from a global counter when the key producer has asked for the last tile of the one before it (longest
+// processing time first, handed out on demand), by a scheduler warp that works out the descriptor once
+// and passes it to the other warps through a small queue in shared memory.  The caches may be
+// contiguous or pages of a pool named by a block table (a page is one tile).
 //
 // Small batches (fewer (server, position block, KV head) groups than half the SMs) run the CLUSTER
 // instantiation instead: one thread-block cluster of 2, 4 or 8 CTAs per group, CTA k taking the k-th
@@ -35,7 +38,7 @@
 
 namespace gs {
 
-constexpr int kAtThreads = 352;          // warp 0 TMA (keys), warp 1 MMA, warps 2-5 softmax, warps 6-9 epilogue, warp 10 TMA (values)
+constexpr int kAtThreads = 384;          // warp 0 TMA (keys), warp 1 MMA, warps 2-5 softmax, warps 6-9 epilogue, warp 10 TMA (values), warp 11 item scheduler
 constexpr int kAtTile = 128;             // keys per tile
 constexpr int kAtHd = 128;
 constexpr int kAtRows = 128;
@@ -43,11 +46,13 @@ constexpr int kAtStages = 3;
 constexpr uint32_t kAtKvBytes = 2 * kAtTile * kAtHd * 2;       // K + V of one tile: 64 KB
 constexpr int kAtMinSplitTiles = 12;     // smallest split the automatic plan makes (tiles of 128 keys)
 constexpr int kAtMaxCached = 1023;       // servers whose offsets are cached in shared memory
-constexpr int kAtItemCache = 32;         // items of a CTA whose descriptors are worked out once, in parallel
-constexpr uint32_t kAtItemCacheBytes = 2304; // >= kAtItemCache * sizeof(AttnItem)
+constexpr int kAtQueue = 8;              // item descriptors in flight between the scheduler warp and the slowest role
+constexpr int kAtQueueReaders = 11;      // warps that read every descriptor (all but the scheduler)
+constexpr uint32_t kAtItemCacheBytes = 640;  // >= kAtQueue * sizeof(AttnItem)
+constexpr uint32_t kAtBarBytes = 512;    // mbarriers and three words behind them
 constexpr int kAtSortMax = 256;          // batches of at most this many servers are walked longest cache first
 constexpr uint32_t kAtSortBytes = 3 * kAtSortMax * 4;
-constexpr uint32_t kAtSmem = kAtStages * kAtKvBytes + 256 + 1024 + 4 * (kAtMaxCached + 1) * 4 + kAtItemCacheBytes +
+constexpr uint32_t kAtSmem = kAtStages * kAtKvBytes + kAtBarBytes + 1024 + 4 * (kAtMaxCached + 1) * 4 + kAtItemCacheBytes +
                              kAtSortBytes;     // 214.5 KB: one CTA per SM
 // Tensor memory (512 columns): S two buffers 0..127 / 128..255 (P, as bf16 pairs, overwrites the first
 // 64 columns of its S buffer once the thread has read its scores), O 256..383, Q (bf16 pairs) 384..447.
@@ -65,6 +70,7 @@ struct AttnTcParams {
   int max_pages, n_pages;
   float* part;              // [items][128][132]
   int* tickets;             // [groups] splits of a (server, position block, KV head) that are done
+  int* next_item;           // items claimed beyond every CTA's first (persistent kernel)
   __nv_bfloat16* O;
   const __nv_bfloat16* Q;
   int32_t* d_status;
@@ -84,6 +90,7 @@ struct AttnItem {
   int tile0, n_tiles;              // tiles [tile0, tile0 + n_tiles) of the server
   int item_base, nsplit, n_used;   // first item of the server, its splits, splits that see any key
   int group;                       // index of (server, position block, KV head) over the whole batch
+  int id;                          // index in the enumeration (persistent kernel: names the partial rows' place)
   int valid;
 };
 
@@ -120,7 +127,7 @@ GS_DEVINL AttnItem attn_item_of_server(const AttnTcParams& P, int i, int q0, int
   int rem = id - base;
   it.g = rem % P.Hkv; rem /= P.Hkv;
   it.split = rem % nsplit; it.tg = rem / nsplit;
-  it.server = i;
+  it.server = i; it.id = id;
   it.item_base = base; it.nsplit = nsplit;
   it.group = gbase + it.tg * P.Hkv + it.g;
   it.q_row0 = q0 + it.tg * P.TB;
@@ -173,7 +180,7 @@ GS_DEVINL AttnItem attn_find_item(const AttnTcParams& P, const int32_t* cu_q, co
   return it;
 }
 
-static_assert(sizeof(AttnItem) * kAtItemCache <= kAtItemCacheBytes, "item cache too small");
+static_assert(sizeof(AttnItem) * kAtQueue <= kAtItemCacheBytes, "item queue too small");
 
 // CLUSTER kernel: part `split` of group `grp` of server i, whose first group is `gbase` (groups are
 // numbered server -> position block -> KV head).  Only the tiles that hold a key the block can see are
@@ -183,7 +190,7 @@ GS_DEVINL AttnItem attn_cluster_item(const AttnTcParams& P, int i, int q0, int n
   AttnItem it;
   const int rem = grp - gbase;
   it.g = rem % P.Hkv; it.tg = rem / P.Hkv; it.split = split; it.server = i;
-  it.item_base = 0; it.nsplit = P.cluster; it.group = grp;
+  it.item_base = 0; it.nsplit = P.cluster; it.group = grp; it.id = 0;
   it.q_row0 = q0 + it.tg * P.TB;
   it.n_t = min(P.TB, n_new - it.tg * P.TB);
   it.kv0 = k0; it.Lkv = Lkv; it.L = Lkv - n_new;
@@ -322,7 +329,7 @@ GS_DEVINL uint32_t pack_bf16_pos(float lo, float hi) {
   return __byte_perm(__float_as_uint(lo) + 0x8000u, __float_as_uint(hi) + 0x8000u, 0x7632);
 }
 
-// Clears the tickets.  The attention kernel is launched behind it as its programmatic dependent: it
+// Clears the tickets and the item counter.  The attention kernel is launched behind it as its programmatic dependent: it
 // starts at once (this kernel only began after everything earlier on the stream had finished, so the
 // inputs are complete) and waits for this grid only where it first touches a ticket.
 __global__ void attn_zero_kernel(int* p, int n) {
@@ -351,13 +358,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
   // its values and are done with as soon as its scores exist, so the K halves turn over faster than the V
   // halves: more bytes in flight per SM than with whole stages that wait for the tile's second product.
   constexpr int kVFull = kODrained + 1, kVEmpty = kVFull + kAtStages;
-  uint8_t* tail = smem_raw + (bars - base) + 8 * (12 + 4 * kAtStages);
+  // q_full[Q] / q_empty[Q]: the item queue's slots (written by the scheduler warp, read by every other
+  // warp); q_taken: the key producer has started on an item, the scheduler may claim the next
+  constexpr int kQFull = kVEmpty + kAtStages, kQEmpty = kQFull + kAtQueue, kQTaken = kQEmpty + kAtQueue;
+  static_assert(8 * (kQTaken + 1) + 12 <= (int)kAtBarBytes, "barrier area too small");
+  uint8_t* tail = smem_raw + (bars - base) + 8 * (kQTaken + 1);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 4);
   volatile int* s_last = reinterpret_cast<volatile int*>(tail + 8);
   // The offsets are read by every role for every item: keep them in shared memory when they fit.
-  float* s_ml = reinterpret_cast<float*>(smem_raw + kAtStages * kAtKvBytes + 256);     // [128][2] row maximum, row sum
-  int32_t* s_cu = reinterpret_cast<int32_t*>(smem_raw + kAtStages * kAtKvBytes + 256 + 1024);
+  float* s_ml = reinterpret_cast<float*>(smem_raw + kAtStages * kAtKvBytes + kAtBarBytes);     // [128][2] row maximum, row sum
+  int32_t* s_cu = reinterpret_cast<int32_t*>(smem_raw + kAtStages * kAtKvBytes + kAtBarBytes + 1024);
   const bool cached = !CLUSTER && P.N <= kAtMaxCached;
   const int32_t* cu_q = cached ? s_cu : P.cu_q;
   const int32_t* cu_kv = cached ? s_cu + (P.N + 1) : P.cu_kv;
@@ -374,14 +385,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
   const int32_t* s_order = sorted ? s_order_w : nullptr;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // The k-th item of this CTA.  The items are enumerated longest cache first and dealt out in rounds of
-  // gridDim.x; every other round runs backwards, so that the CTA that got the longest item of one round
-  // gets the shortest of the next (a plain stride would hand CTA 0 the longest item of every round).
-  // Ids past the end of the enumeration only occur in the last round, so the first one ends a CTA's walk.
-  auto item_id = [&](int k) -> long long {
-    const long long b = (k & 1) ? (long long)gridDim.x - 1 - blockIdx.x : (long long)blockIdx.x;
-    return (long long)k * gridDim.x + b;
-  };
   // The next kernel on the stream may set itself up on idle SMs right away (it still waits for this
   // grid to finish before it touches global memory).
   pdl_launch_dependents();
@@ -401,6 +404,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
     }
     mbar_init(bar(kEpiA), 128); mbar_init(bar(kEpiB), 128);
     mbar_init(bar(kStatsFull), 4); mbar_init(bar(kODrained), 4);
+    for (int s = 0; s < kAtQueue; ++s) { mbar_init(bar(kQFull + s), 1); mbar_init(bar(kQEmpty + s), kAtQueueReaders); }
+    mbar_init(bar(kQTaken), 1);
     *abort_flag = 0;
     fence_barrier_init();
     fence_proxy_async();
@@ -489,8 +494,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
     }
     __syncthreads();
   }
-  if (cached && warp == 2) {
-    // counts -> exclusive prefix sums, 32 servers per step
+  if (cached && warp == 11) {
+    // counts -> exclusive prefix sums, 32 servers per step (the scheduler warp: it goes straight on to
+    // the CTA's first item)
     int carry = 0, gcarry = 0;
     for (int c = 0; c <= P.N; c += 32) {
       const int i = c + lane;
@@ -506,21 +512,46 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
       gcarry += __shfl_sync(0xffffffffu, ginc, 31);
     }
   }
-  if (!CLUSTER) {
-    __syncthreads();
-    // The descriptors of this CTA's first items, one thread each: a descriptor costs a dozen integer
-    // divisions, which every role would otherwise repeat, one after the other, at every item.
-    if (warp == 3) {
-      const long long id = item_id(lane);
+  // One item descriptor, worked out by one lane and published in slot k mod kAtQueue (scheduler warp).
+  auto publish_item = [&](int k, long long id) -> int {
+    int valid = 0;
+    if (lane == 0) {
       AttnItem it;
       it.valid = 0;
       if (id < P.max_items) it = attn_find_item(P, cu_q, cu_kv, s_base, s_gbase, s_order, (int)id);
-      s_items[lane] = it;
+      s_items[k % kAtQueue] = it;
+      valid = it.valid;
+      mbar_arrive(bar(kQFull + k % kAtQueue));
+    }
+    return __shfl_sync(0xffffffffu, valid, 0);
+  };
+  int sched_live = 0;
+  if (!CLUSTER) {
+    // The CTA's first item is the one with its own index.  It is published before the barrier the other
+    // warps sleep at: warps that polled the queue instead would take issue slots from the lane that works
+    // the descriptor out (measured: 2 us later first loads).
+    if (warp == 11) {
+      __syncwarp();
+      sched_live = publish_item(0, (long long)blockIdx.x);
     }
     __syncthreads();
   }
-  auto item_at = [&](int k, int id) -> AttnItem {
-    return k < kAtItemCache ? s_items[k] : attn_find_item(P, cu_q, cu_kv, s_base, s_gbase, s_order, id);
+  // The k-th item of this CTA (whole warp; false: there is none, or a wait ran out).  CLUSTER: the one
+  // item found above.  Otherwise the scheduler warp's k-th descriptor, from slot k mod kAtQueue of the
+  // queue; the slot goes back to the scheduler once every warp has read it.  The descriptor that ends
+  // the sequence (valid = 0) is read by everybody as well.
+  auto take_item = [&](int k, AttnItem& it) -> bool {
+    if (CLUSTER) {
+      if (k > 0) return false;
+      it = s_items[0];
+      return it.valid != 0;
+    }
+    const int slot = k % kAtQueue;
+    if (!mbar_wait_warp(bar(kQFull + slot), (uint32_t)(k / kAtQueue) & 1u, abort_flag)) return false;
+    it = s_items[slot];
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar(kQEmpty + slot));
+    return it.valid != 0;
   };
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t tmem_S = tmem_base + kAtColS, tmem_O = tmem_base + kAtColO;     // S buffer b at tmem_S + 128 b
@@ -555,10 +586,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
       const int b_empty = keys ? kKvEmpty : kVEmpty;
       uint32_t st = (uint32_t)first % kAtStages, ph = (first == kAtStages) ? 1u : 0u;
       bool ok = true;
-      for (long long k_item = 0, id = item_id(0); id < P.max_items && ok && (!CLUSTER || k_item == 0); ++k_item, id = item_id((int)k_item)) {
-        const AttnItem it = item_at((int)k_item, (int)id);
-        if (!it.valid) break;
-        if (it.n_tiles == 0) continue;
+      AttnItem it;
+      for (int k_item = 0; ok && take_item(k_item, it); ++k_item) {
         for (int j = first; j < it.n_tiles; ++j) {
           if (!mbar_wait_warp(bar(b_empty + st), ph ^ 1u, abort_flag)) { ok = false; break; }
           if (elect_one()) {
@@ -567,8 +596,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
           __syncwarp();
           if (++st == kAtStages) { st = 0; ph ^= 1u; }
         }
+        // every key tile of the item is on its way: time to claim the next item
+        if (!CLUSTER && keys && lane == 0) mbar_arrive(bar(kQTaken));
       }
-      if (!ok) { const uint64_t t0 = global_timer_ns(); while (global_timer_ns() - t0 < 200000ull) { } }
+      if (!ok || *abort_flag) { const uint64_t t0 = global_timer_ns(); while (global_timer_ns() - t0 < 200000ull) { } }
     }
     __syncwarp();
   } else if (warp == 1) {
@@ -597,9 +628,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
       }
       __syncwarp();
     };
-    for (long long k_item = 0, id = item_id(0); id < P.max_items && ok && (!CLUSTER || k_item == 0); ++k_item, id = item_id((int)k_item)) {
-      const AttnItem it = item_at((int)k_item, (int)id);
-      if (!it.valid) break;
+    AttnItem it;
+    for (int k_item = 0; ok && take_item(k_item, it); ++k_item) {
       if (it.n_tiles == 0) continue;
       // Q of this item sits in tensor memory (written by the softmax warps after they have
       // drained O of the previous item)
@@ -641,7 +671,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
       }
       ++n_item;
     }
-    if (!ok) { const uint64_t t0 = global_timer_ns(); while (global_timer_ns() - t0 < 200000ull) { } }
+    if (!ok || *abort_flag) { const uint64_t t0 = global_timer_ns(); while (global_timer_ns() - t0 < 200000ull) { } }
     __syncwarp();
   } else if (warp < 6) {
     // ------------------------------------------------ softmax: thread = row
@@ -650,9 +680,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
     int n_item = 0, n_tile_total = 0;
     bool ok = true;
-    for (long long k_item = 0, id = item_id(0); id < P.max_items && ok && (!CLUSTER || k_item == 0); ++k_item, id = item_id((int)k_item)) {
-      const AttnItem it = item_at((int)k_item, (int)id);
-      if (!it.valid) break;
+    AttnItem it;
+    for (int k_item = 0; ok && take_item(k_item, it); ++k_item) {
       if (it.n_tiles == 0) continue;
       const int R = it.n_t * P.G;
       const bool row_ok = r < R;
@@ -791,9 +820,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
     int n_item = 0, n_ticket = 0;
     bool ok = true;
-    for (long long k_item = 0, id = item_id(0); id < P.max_items && ok && (!CLUSTER || k_item == 0); ++k_item, id = item_id((int)k_item)) {
-      const AttnItem it = item_at((int)k_item, (int)id);
-      if (!it.valid) break;
+    AttnItem it;
+    for (int k_item = 0; ok && take_item(k_item, it); ++k_item) {
       if (it.n_tiles == 0) continue;
       const int R = it.n_t * P.G;
       const bool row_ok = r < R;
@@ -805,7 +833,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
       // partial rows go to the workspace, or (CLUSTER) to this CTA's own shared memory: every tile of
       // the item has been consumed by now, so the K/V ring is free
       float* out = CLUSTER ? reinterpret_cast<float*>(smem_raw) + (size_t)r * kAtPartStride
-                           : P.part + ((size_t)id * kAtRows + r) * kAtPartStride;
+                           : P.part + ((size_t)it.id * kAtRows + r) * kAtPartStride;
       const bool single = (it.n_used == 1);            // the only split of its group: normalise and store
       const float inv1 = single ? 1.f / l_run : 1.f;
 #pragma unroll
@@ -935,6 +963,21 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant_
       }
       ++n_item;
     }
+  } else if (warp == 11 && !CLUSTER) {
+    // ------------------------------------------------ item scheduler: descriptor k goes to slot k mod
+    // kAtQueue once every warp has read the descriptor that was there.  The first item (the CTA's own
+    // index) was published during the set-up; item k >= 1 is claimed from the global counter when the key producer has asked for the
+    // last tile of item k - 1, not earlier: the items come longest first, and a CTA that reserved
+    // several ahead would sit on work that an idle CTA could do.  The ring still holds that item's last
+    // tiles then, which covers the time the descriptor takes (a bisection and a dozen integer divisions).
+    for (int k = 1; sched_live; ++k) {
+      const int slot = k % kAtQueue;
+      if (k >= kAtQueue && !mbar_wait_warp(bar(kQEmpty + slot), (uint32_t)(k / kAtQueue - 1) & 1u, abort_flag)) break;
+      if (!mbar_wait_warp(bar(kQTaken), (uint32_t)(k - 1) & 1u, abort_flag)) break;
+      long long id = 0;
+      if (lane == 0) id = (long long)gridDim.x + atomicAdd(P.next_item, 1);
+      sched_live = publish_item(k, id);
+    }
   }
   tc_fence_before();
   __syncthreads();
@@ -1050,7 +1093,7 @@ inline AttnTcPlan attn_tc_plan(int N, int Tq, int total_kv, int max_kv_len, int 
   pl.max_items = (int)min(items, (long long)INT_MAX / 2);
   pl.grid = min(pl.max_items, slots);
   pl.max_groups = (int)min((long long)Hkv * blocks, (long long)INT_MAX / 2);
-  pl.ticket_bytes = align_up((size_t)pl.max_groups * sizeof(int), 256);
+  pl.ticket_bytes = align_up(((size_t)pl.max_groups + 1) * sizeof(int), 256);      // and the item counter behind them
   pl.ws_bytes = pl.ticket_bytes + (size_t)pl.max_items * kAtRows * kAtPartStride * sizeof(float);
   // Few groups (a small batch): one cluster per group, as wide as still lets every cluster of the
   // expected number of groups be resident at once, and no wider than leaves a part two tiles.
@@ -1085,6 +1128,7 @@ inline gs_status launch_attn_tc(const void* Q, const void* K, const void* V, voi
   P.cu_q = cu_q; P.cu_kv = cu_kv; P.d_status = d_status;
   P.block_table = block_table; P.max_pages = max_pages; P.n_pages = n_pages;
   P.tickets = static_cast<int*>(ws);
+  P.next_item = P.tickets + pl.max_groups;
   P.part = reinterpret_cast<float*>(static_cast<char*>(ws) + pl.ticket_bytes);
   P.O = static_cast<__nv_bfloat16*>(O);
   P.Q = static_cast<const __nv_bfloat16*>(Q);
