@@ -682,7 +682,7 @@ def run_head_sweep(args, cfg, local_rank):
 
 def run_attn_sweep(args, local_rank):
     """gs_verify_attn alone on every workload's attention inputs, per kernel choice: automatic, the
-    persistent kernel, clusters of 2 / 4 / 8.  Timed as CUDA-graph replays of [read 256 MB; call] minus
+    persistent kernel, one CTA per group, clusters of 2 / 4 / 8.  Timed as CUDA-graph replays of [read 256 MB; call] minus
     replays of [read 256 MB] alone (cold L2, no host launch cost), best of three."""
     from paper_2512_09963_b200 import binding as B
     from paper_2512_09963_b200 import build as gs_build
@@ -734,7 +734,7 @@ def run_attn_sweep(args, local_rank):
         by = 2 * total_kv * Hkv * hd * 2 + 2 * Tq * Hq * hd * 2
         O = torch.empty_like(inp["Q"])
         st = torch.zeros(1, dtype=torch.int32, device=dev)
-        for variant in (0, 1, 2, 4, 8):
+        for variant in (0, 1, 3, 2, 4, 8):
             B.gs_verify_attn_select(variant)
             ws = torch.empty(max(256, B.gs_verify_attn_workspace(N, Tq, total_kv, max_len, Hq, Hkv, hd, B.GS_BF16)),
                              dtype=torch.uint8, device=dev)
@@ -745,8 +745,8 @@ def run_attn_sweep(args, local_rank):
             launches = B.gs_launch_count() - c0
             assert int(st.item()) == 0
             us = min(replay_us(graph_of(call)) - base for _ in range(3))
-            rows.append({"workload": name, "kernel": {0: "automatic", 1: "persistent", 2: "clusters of 2", 4: "clusters of 4",
-                                                      8: "clusters of 8"}[variant], "launches": int(launches), "us": us,
+            rows.append({"workload": name, "kernel": {0: "automatic", 1: "persistent", 3: "one CTA per group", 2: "clusters of 2",
+                                                      4: "clusters of 4", 8: "clusters of 8"}[variant], "launches": int(launches), "us": us,
                          "algorithmic_bytes": by, "GBps": by / us / 1e3, "frac_hbm": by / us / 1e3 / peak})
         B.gs_verify_attn_select(0)
     print(json.dumps({"attn_sweep": rows, "peak_hbm_gbs": peak, "peak_source": kind}), flush=True)

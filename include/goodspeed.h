@@ -178,7 +178,7 @@ gs_status gs_lm_head_logits(const void* H, const void* W, float* logits, int T, 
  *   H [T, d] bf16, logits [T, V] fp32 as gs_lm_head_logits:
  *   logits[t, v] = sum_k H[t, k] * bf16(W[k, v])   -- every weight is rounded to bf16 once (the one
  *   multiplication by the scale), products exact, accumulation fp32 on the tensor cores.
- * Needs group % 64 == 0, d % group == 0, V % 16 == 0 and 16-byte aligned pointers (UNSUPPORTED
+ * Needs group == 64 or group % 128 == 0, d % 128 == 0, d % group == 0, V % 16 == 0 and 16-byte aligned pointers (UNSUPPORTED
  * otherwise).  No workspace.  More than 256 rows stream the weights once per 256 rows.
  * Errors: INVALID_ARG, UNSUPPORTED, CUDA.  Device status: GS_ERR_TIMEOUT only.
  */

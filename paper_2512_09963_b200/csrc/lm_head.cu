@@ -503,7 +503,8 @@ extern "C" gs_status gs_lm_head_logits_w4(const void* H, const uint32_t* qweight
   if (T < 0 || d < 0 || V < 0 || group <= 0) return GS_ERR_INVALID_ARG;
   if (T == 0 || V == 0) return GS_OK;
   if (!H || !qweight || !scales || !zeros || !logits) return GS_ERR_INVALID_ARG;
-  if (d == 0 || group % (int)kW4BlockK != 0 || d % group != 0 || V % 16 != 0) return GS_ERR_UNSUPPORTED;
+  if (d == 0 || d % (int)kW4StageK != 0 || (group != (int)kW4EntryK && group % (int)kW4StageK != 0) || d % group != 0 || V % 16 != 0)
+    return GS_ERR_UNSUPPORTED;
   if ((reinterpret_cast<uintptr_t>(H) | reinterpret_cast<uintptr_t>(qweight) | reinterpret_cast<uintptr_t>(scales) |
        reinterpret_cast<uintptr_t>(zeros)) % 16 != 0)
     return GS_ERR_UNSUPPORTED;

@@ -720,7 +720,7 @@ def test_lm_head_small(T, d, V, variant):
 
 
 # ------------------------------------------------------------------ LM head on 4-bit weights
-@pytest.mark.parametrize("T,d,V,group", [(46, 512, 9008, 128), (96, 1024, 4112, 128), (1, 64, 16, 64), (130, 192, 1008, 64),
+@pytest.mark.parametrize("T,d,V,group", [(46, 512, 9008, 128), (96, 1024, 4112, 128), (1, 128, 16, 64), (130, 384, 1008, 64),
                                          (256, 256, 2048, 128), (300, 128, 528, 128), (16, 5120, 4096, 128),
                                          (144, 384, 20000, 128)])
 def test_lm_head_w4_small(T, d, V, group):
