@@ -109,6 +109,39 @@ GS_DEVINL void head_w4_issue_unit(uint32_t d_acc, uint32_t a0, uint32_t b_hi, ui
   }
 }
 
+// One warp's share of an entry: for each of the tile's WIDTH units the four packed words of its 32 k,
+// expanded and stored to the entry's columns.  WIDTH is a compile-time constant so that all the loads
+// are issued up front and the units' instruction streams interleave.  The entry's previous contents
+// must have been consumed by the MMAs that read them before the first store: that wait comes after the
+// first unit's expansion, which does not need the entry yet.
+template <int WIDTH>
+GS_DEVINL bool head_w4_expand_entry(const uint32_t* qw0, const __nv_bfloat16* sc0, const uint8_t* zp0, uint32_t dst0,
+                                    uint32_t aempty, uint32_t aempty_parity, volatile int* abort_flag) {
+  uint32_t words[WIDTH][4];
+  __nv_bfloat162 zz[WIDTH], ss[WIDTH];
+#pragma unroll
+  for (int u = 0; u < WIDTH; ++u) {
+#pragma unroll
+    for (int w = 0; w < 4; ++w) words[u][w] = qw0[u * (int)(kW4QBytes / 4u) + w * (int)kW4Unit];
+    const __nv_bfloat16 sc = sc0[u * (int)(kW4SBytes / 2u)];
+    const uint32_t zbits = 0x4300u | ((uint32_t)zp0[u * (int)kW4ZBytes] & 15u);
+    const uint32_t zz_u = zbits | (zbits << 16);
+    zz[u] = *reinterpret_cast<const __nv_bfloat162*>(&zz_u);
+    ss[u] = __halves2bfloat162(sc, sc);
+  }
+#pragma unroll
+  for (int u = 0; u < WIDTH; ++u) {
+    uint32_t x[16];
+    w4_expand4(words[u], zz[u], ss[u], x);
+    if (u == 0) {
+      if (!mbar_wait(aempty, aempty_parity, abort_flag)) return false;
+      tc_fence_after();
+    }
+    tmem_st16(dst0 + (uint32_t)u * kW4SlotCols, x);
+  }
+  return true;
+}
+
 __global__ void __launch_bounds__(kW4Threads, 1)
 lm_head_w4_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant__ CUtensorMap tmapS,
                   const __grid_constant__ CUtensorMap tmapZ, const __grid_constant__ CUtensorMap tmapH,
@@ -272,25 +305,15 @@ lm_head_w4_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_consta
         if (!mbar_wait(full_bar(st), ph, abort_flag)) { ok = false; break; }
         const int wrow = (int)set * 8 + half * 4;               // first of this warp's four rows of packed words
         const int grow = two_groups ? (int)set : 0;             // the entry's group within the stage
-        for (int u = 0; u < width; ++u) {
-          const uint32_t* qw = reinterpret_cast<const uint32_t*>(stage + q_off + (uint32_t)u * kW4QBytes) + wrow * (int)kW4Unit + col;
-          const __nv_bfloat16 sc = *(reinterpret_cast<const __nv_bfloat16*>(stage + s_off + (uint32_t)u * kW4SBytes) + grow * (int)kW4Unit + col);
-          const uint32_t zp = *(stage + z_off + (uint32_t)u * kW4ZBytes + grow * (int)kW4Unit + col);
-          const uint32_t zbits = 0x4300u | (zp & 15u);
-          const uint32_t zz_u = zbits | (zbits << 16);
-          const __nv_bfloat162 zz = *reinterpret_cast<const __nv_bfloat162*>(&zz_u);
-          const __nv_bfloat162 ss = __halves2bfloat162(sc, sc);
-          uint32_t words[4];
-#pragma unroll
-          for (int w = 0; w < 4; ++w) words[w] = qw[w * (int)kW4Unit];
-          uint32_t x[16];
-          w4_expand4(words, zz, ss, x);
-          if (u == 0) {
-            // the entry's previous contents have been consumed by the MMAs that read them
-            if (!mbar_wait(aempty_bar(buf), bph ^ 1u, abort_flag)) { ok = false; break; }
-            tc_fence_after();
-          }
-          tmem_st16(tmem_A + lane_addr + buf * buf_cols + (uint32_t)u * kW4SlotCols + (uint32_t)half * 16u, x);
+        const uint32_t* qw0 = reinterpret_cast<const uint32_t*>(stage + q_off) + wrow * (int)kW4Unit + col;
+        const __nv_bfloat16* sc0 = reinterpret_cast<const __nv_bfloat16*>(stage + s_off) + grow * (int)kW4Unit + col;
+        const uint8_t* zp0 = stage + z_off + grow * (int)kW4Unit + col;
+        const uint32_t dst0 = tmem_A + lane_addr + buf * buf_cols + (uint32_t)half * 16u;
+        switch (width) {
+          case 1: ok = head_w4_expand_entry<1>(qw0, sc0, zp0, dst0, aempty_bar(buf), bph ^ 1u, abort_flag); break;
+          case 2: ok = head_w4_expand_entry<2>(qw0, sc0, zp0, dst0, aempty_bar(buf), bph ^ 1u, abort_flag); break;
+          case 3: ok = head_w4_expand_entry<3>(qw0, sc0, zp0, dst0, aempty_bar(buf), bph ^ 1u, abort_flag); break;
+          default: ok = head_w4_expand_entry<4>(qw0, sc0, zp0, dst0, aempty_bar(buf), bph ^ 1u, abort_flag); break;
         }
         if (!ok) break;
         tmem_st_wait();
