@@ -90,7 +90,9 @@ GS_DEVINL void w4_expand4(const uint32_t (&words)[4], __nv_bfloat162 zz, __nv_bf
   for (int w = 0; w < 4; ++w) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      const uint32_t t = ((words[w] >> (4 * i)) & 0x000F000Fu) | 0x43004300u;
+      // (x >> 4i) & 0x000F000F | 0x43004300 as one shift and ONE three-input logic instruction
+      uint32_t t;
+      asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(t) : "r"(words[w] >> (4 * i)), "r"(0x000F000Fu), "r"(0x43004300u));
       const __nv_bfloat162 c = *reinterpret_cast<const __nv_bfloat162*>(&t);
       const __nv_bfloat162 x = __hmul2(__hsub2(c, zz), ss);
       out[4 * w + i] = *reinterpret_cast<const uint32_t*>(&x);
