@@ -449,6 +449,42 @@ def measure_config(args, cfg, rank, world, local_rank, steps, warmup, detail):
         w4 = {"entry_point": "gs_lm_head_logits_w4", "rows": Tw, "group": 128, "us": us4, "algorithmic_bytes": by4,
               "gbs": by4 / us4 / 1e3, "frac_hbm": by4 / us4 / 1e3 / peak, "bf16_head_us": k_us["lm_head_logits"],
               "speedup_over_bf16_head": k_us["lm_head_logits"] / us4}
+        # ... and the whole step with that head: attention, 4-bit head, acceptance (statistics pass + finish on
+        # its logits), scheduler, as a CUDA-graph replay like the headline.  The synthetic codes are unrelated
+        # to the drafts, so nearly every first draft is rejected; the metric counts verified drafts per second.
+        if not args.no_graph:
+            lg_full = torch.empty((Tq, V), dtype=torch.float32, device=dev)
+
+            def step4():
+                rnd.attn(inp["Q"], inp["K"], inp["V"], inp["cu_q"], inp["cu_kv"])
+                B.gs_lm_head_logits_w4(inp["H"], layer["qweight"], layer["scales"], layer["zeros"], 128, lg_full, rnd.d_status)
+                rnd.accept(inp["q_probs"], inp["draft_tok"], inp["cu_q"], inp["u_accept"], inp["u_sample"], inp["tau"],
+                           logits=lg_full, update=False)
+                rnd.schedule(s_min, s_max)
+
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                step4()
+            torch.cuda.current_stream().wait_stream(side)
+            g4 = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g4):
+                step4()
+            for _ in range(5):
+                g4.replay()
+            torch.cuda.synchronize()
+            n4 = 200
+            a.record()
+            for _ in range(n4):
+                g4.replay()
+            b.record()
+            torch.cuda.synchronize()
+            assert int(rnd.d_status.item()) == 0, "device status after the steps with the 4-bit head"
+            step4_us = a.elapsed_time(b) * 1e3 / n4
+            w4["step_us"] = step4_us
+            w4["step_verified_tokens_per_s"] = Gamma / (step4_us * 1e-6)
+            w4["step_speedup_over_bf16_step"] = ms_step * 1e3 / step4_us
+            del lg_full, g4
         del layer, lg, Hs
     out = {"cfg": cfg, "inp": inp, "host": host, "rnd": rnd, "first": first, "N": N, "Tq": Tq, "Gamma": Gamma, "C": C, "w4": w4,
            "ms_step": ms_step, "gamma_all": gamma_all, "clocks": clocks, "kernels": kernels, "roofline": roofline,
