@@ -505,7 +505,13 @@ def measure_config(args, cfg, rank, world, local_rank, steps, warmup, detail):
                ("Q", "H", "q_probs", "draft_tok", "u_accept", "u_sample", "cu_q", "cu_kv")}
         outs = {k: torch.empty(n, dtype=torch.int32).pin_memory() for k, n in
                 (("accepted", N), ("out_tok", Tq), ("n_out", N), ("S_next", N), ("status", 1))}
-        h2d = sum(t.numel() * t.element_size() for t in pin.values())
+        # Bytes that cross the bus host -> device per step.  Pinned draft distributions are not copied:
+        # the acceptance kernels read q(s_j) of each drafted token (a 32-byte sector each) and at most one
+        # row per server where they lie; everything else is staged with copies.
+        in_place = B.gs_verify_round_reads_in_place(pin["q_probs"])
+        staged = sum(t.numel() * t.element_size() for k, t in pin.items() if not (in_place and k == "q_probs"))
+        pulled = (N * V * 4 + 32 * Gamma) if in_place else 0
+        h2d = staged + pulled
         d2h = sum(t.numel() * t.element_size() for t in outs.values())
 
         def e2e_step():
@@ -527,7 +533,21 @@ def measure_config(args, cfg, rank, world, local_rank, steps, warmup, detail):
             e2e_step()
         dt = (time.time() - t0) / n_e
         out["e2e"] = {"value": Gamma / dt, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                      "ms_per_step": dt * 1e3, "matches_device_path": bool(e2e_ok)}
+                      "ms_per_step": dt * 1e3, "matches_device_path": bool(e2e_ok),
+                      "h2d_detail": {"copied": staged, "read_in_place_by_kernels_at_most": pulled,
+                                     "draft_distributions_bytes": pin["q_probs"].numel() * 4,
+                                     "draft_distributions": "read in place (pinned host memory)" if in_place else "copied"}}
+        if in_place:        # the same with the distributions staged by a copy, for comparison
+            B.gs_verify_round_configure(False)
+            try:
+                for _ in range(3):
+                    e2e_step()
+                t0 = time.time()
+                for _ in range(n_e):
+                    e2e_step()
+                out["e2e"]["ms_per_step_with_distributions_copied"] = (time.time() - t0) / n_e * 1e3
+            finally:
+                B.gs_verify_round_configure(True)
         del ws
 
     # ---- CPU baseline = the oracle on the host cores, and a parity check of this launch configuration

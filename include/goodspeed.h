@@ -358,7 +358,12 @@ gs_status gs_schedule_host(const double* X, const double* alpha_hat, int N, int 
  * make that first call outside any stream capture) while attention and the LM head run on `stream`;
  * `stream` waits for them before gs_spec_accept, and they wait for `stream` to reach this call, so
  * back-to-back rounds on one stream are ordered.  Rounds issued on DIFFERENT streams with the same
- * d_ws race, as they would anyway.  Errors: as the four calls; CUDA if a copy could not be enqueued.
+ * d_ws race, as they would anyway.
+ * Draft distributions in pinned memory that the device can address (cudaHostAlloc, or cudaHostRegister
+ * with the mapped flag) are NOT copied: the acceptance pass needs q(s_j) of the drafted tokens and one
+ * row per server (the row of its first rejection), and its kernels read those from the host buffer
+ * over the bus -- at most N*V*4 + 32*Gamma bytes instead of Gamma*V*4 (see gs_verify_round_configure).
+ * Errors: as the four calls; CUDA if a copy could not be enqueued.
  */
 typedef struct gs_round_desc {
   int N, Tq, total_kv, max_kv_len, Hq, Hkv, hd, d, V, C;
@@ -368,6 +373,13 @@ typedef struct gs_round_desc {
 } gs_round_desc;
 
 size_t gs_verify_round_workspace(const gs_round_desc* r);
+/* Whether gs_verify_round_host may read the draft distributions where they lie (process-wide, not
+ * thread-safe; 1 = yes, the default, 0 = always stage them in the workspace).  Results do not depend on it.
+ * Errors: INVALID_ARG. */
+gs_status gs_verify_round_configure(int read_in_place);
+/* 1 if gs_verify_round_host would read this host buffer of draft distributions in place (it is pinned
+ * memory with a device address and in-place reads are on), 0 if it would stage it. */
+int gs_verify_round_reads_in_place(const float* h_q_probs);
 gs_status gs_verify_round_host(const gs_round_desc* r,
                                const void* h_Q, const void* h_H, const float* h_q_probs,
                                const int32_t* h_draft_tok, const float* h_u_accept, const float* h_u_sample,

@@ -61,6 +61,8 @@ SIGNATURES = {
     "gs_schedule_host": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp]),
     "gs_selftest_wait_timeout": (_i, [C.c_uint, _vp, _vp, _vp]),
     "gs_verify_round_workspace": (_sz, [_vp]),
+    "gs_verify_round_configure": (_i, [_i]),
+    "gs_verify_round_reads_in_place": (_i, [_vp]),
     "gs_verify_round_host": (_i, [_vp] + [_vp] * 8 + [_vp] * 7 + [_vp, _sz] + [_vp] * 5 + [_vp]),
     "gs_launch_count": (C.c_ulonglong, []),
 }
@@ -335,6 +337,15 @@ def gs_launch_count() -> int:
 
 def gs_verify_round_workspace(desc: RoundDesc) -> int:
     return lib().gs_verify_round_workspace(C.byref(desc))
+
+
+def gs_verify_round_configure(read_in_place: bool = True):
+    _check("gs_verify_round_configure", lib().gs_verify_round_configure(1 if read_in_place else 0))
+
+
+def gs_verify_round_reads_in_place(h_q_probs) -> bool:
+    """Whether gs_verify_round_host would read this CPU tensor of draft distributions where it lies."""
+    return bool(lib().gs_verify_round_reads_in_place(_ptr(h_q_probs, torch.float32, cuda=False)))
 
 
 def gs_verify_round_host(desc: RoundDesc, h_Q, h_H, h_q_probs, h_draft_tok, h_u_accept, h_u_sample,

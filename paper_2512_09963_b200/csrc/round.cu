@@ -2,9 +2,12 @@
 // host memory (what the draft servers sent this round), with the model state resident on the GPU.
 // It stages the inputs with cudaMemcpyAsync, enqueues the four steps of the round and copies the
 // small results back; nothing here computes.  The draft distributions are by far the largest
-// input (Gamma x V floats) and only the acceptance pass reads them, so they travel on a copy stream
-// of the library's own while attention and the LM head run; an event hands them to the caller's
-// stream before gs_spec_accept.
+// input (Gamma x V floats), and the acceptance pass reads little of them: q(s_j) of every drafted
+// token and ONE row per server, the row of its first rejection.  Where the caller's buffer is pinned
+// memory that the device can address, the kernels therefore read it where it lies (a few MB cross
+// the bus instead of Gamma x V x 4 bytes, which at cfg2 take longer than the whole round on the
+// device).  Otherwise the distributions travel on a copy stream of the library's own while attention
+// and the LM head run, and an event hands them to the caller's stream before gs_spec_accept.
 #include "common.cuh"
 
 namespace gs {
@@ -81,7 +84,30 @@ static bool desc_ok(const gs_round_desc* r) {
          r->Hkv > 0 && r->hd > 0 && r->d > 0 && r->V > 0 && r->C >= 0 && (r->dt == GS_F32 || r->dt == GS_BF16);
 }
 
+
+// 1 = read the draft distributions in place where possible (default), 0 = always stage them.
+static int g_round_in_place = 1;
+
+// The address under which the device can read a host buffer where it lies, or NULL.
+static const float* device_view_of_host(const float* h) {
+  if (h == nullptr || !g_round_in_place) return nullptr;
+  cudaPointerAttributes at;
+  if (cudaPointerGetAttributes(&at, h) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
+  if (at.type != cudaMemoryTypeHost || at.devicePointer == nullptr) return nullptr;
+  return static_cast<const float*>(at.devicePointer);
+}
+
 }  // namespace gs
+
+extern "C" gs_status gs_verify_round_configure(int read_in_place) {
+  if (read_in_place != 0 && read_in_place != 1) return GS_ERR_INVALID_ARG;
+  gs::g_round_in_place = read_in_place;
+  return GS_OK;
+}
+
+extern "C" int gs_verify_round_reads_in_place(const float* h_q_probs) {
+  return gs::device_view_of_host(h_q_probs) != nullptr ? 1 : 0;
+}
 
 extern "C" size_t gs_verify_round_workspace(const gs_round_desc* r) {
   if (!gs::desc_ok(r)) return 0;
@@ -129,8 +155,10 @@ extern "C" gs_status gs_verify_round_host(const gs_round_desc* r,
   if (side == nullptr) return GS_ERR_CUDA;
   if (cudaEventRecord(side->begin, st) != cudaSuccess || cudaStreamWaitEvent(side->copy, side->begin, 0) != cudaSuccess)
     return GS_ERR_CUDA;
+  const float* q_in_place = (Gamma > 0) ? device_view_of_host(h_q_probs) : nullptr;
   ok = h2d_on(side->copy, L.draft_tok, h_draft_tok, Gamma * 4) && h2d_on(side->copy, L.u_accept, h_u_accept, Gamma * 4) &&
-       h2d_on(side->copy, L.u_sample, h_u_sample, N * 4) && h2d_on(side->copy, L.q_probs, h_q_probs, Gamma * V * 4);
+       h2d_on(side->copy, L.u_sample, h_u_sample, N * 4) &&
+       (q_in_place != nullptr || h2d_on(side->copy, L.q_probs, h_q_probs, Gamma * V * 4));
   if (!ok || cudaEventRecord(side->staged, side->copy) != cudaSuccess) return GS_ERR_CUDA;
   int32_t* d_status = reinterpret_cast<int32_t*>(w + L.status);
   const int32_t* cu_q = reinterpret_cast<const int32_t*>(w + L.cu_q);
@@ -153,7 +181,7 @@ extern "C" gs_status gs_verify_round_host(const gs_round_desc* r,
   if (s != GS_OK) return s;
   if (cudaStreamWaitEvent(st, side->staged, 0) != cudaSuccess) return GS_ERR_CUDA;
   const float* lg = reinterpret_cast<const float*>(w + L.logits);
-  const float* qp = reinterpret_cast<const float*>(w + L.q_probs);
+  const float* qp = (q_in_place != nullptr) ? q_in_place : reinterpret_cast<const float*>(w + L.q_probs);
   const int32_t* dtok = reinterpret_cast<const int32_t*>(w + L.draft_tok);
   const float* ua = reinterpret_cast<const float*>(w + L.u_accept);
   const float* us = reinterpret_cast<const float*>(w + L.u_sample);

@@ -659,11 +659,14 @@ def test_fused_head_statistics_unsupported_shapes_fall_back():
 
 
 # ------------------------------------------------------------------ the round from host buffers
+@pytest.mark.parametrize("q_mode", ["in-place", "copied", "pageable"])
 @pytest.mark.parametrize("gamma", [[3, 1, 8, 2, 5, 4, 7, 6], [8, 8, 8, 8, 8, 8, 8, 8]], ids=["44-positions", "72-positions"])
-def test_verify_round_host_matches_device_path(gamma):
-    """gs_verify_round_host (inputs in pinned host memory, draft distributions copied on the
-    library's copy stream while attention and the LM head run) gives what the four calls give on
-    device-resident inputs; two rounds back to back with different drafts reuse the staging area."""
+def test_verify_round_host_matches_device_path(gamma, q_mode):
+    """gs_verify_round_host gives what the four calls give on device-resident inputs, whether the
+    acceptance kernels read the pinned draft distributions where they lie (the default), the library
+    copies them on its copy stream while attention and the LM head run (in-place reads switched off),
+    or the buffer is pageable memory, which can only be copied; two rounds back to back with different
+    drafts reuse the staging area."""
     cfg = wl.shrink(wl.CONFIGS["cfg2"], d=256, V=16384, prefix_scale=0.1, name="host_round")
     for round_idx in (0, 1):
         inp = wl.make_step(cfg, round_idx=round_idx, gamma=gamma)     # same shapes, new drafts
@@ -680,15 +683,22 @@ def test_verify_round_host_matches_device_path(gamma):
             ws = torch.empty(B.gs_verify_round_workspace(desc), dtype=torch.uint8, device=DEV)
         pin = {k: inp[k].contiguous().pin_memory() for k in
                ("Q", "H", "q_probs", "draft_tok", "u_accept", "u_sample", "cu_q", "cu_kv")}
+        if q_mode == "pageable":
+            pin["q_probs"] = inp["q_probs"].contiguous().clone()
         outs = {k: torch.full((n,), -9, dtype=torch.int32).pin_memory() for k, n in
                 (("accepted", N), ("out_tok", Tq), ("n_out", N), ("S_next", N), ("status", 1))}
         a_hat = torch.full((N,), 0.5, dtype=torch.float64, device=DEV)
         X = torch.ones(N, dtype=torch.float64, device=DEV)
-        B.gs_verify_round_host(desc, pin["Q"], pin["H"], pin["q_probs"], pin["draft_tok"], pin["u_accept"],
-                               pin["u_sample"], pin["cu_q"], pin["cu_kv"], d["K"], d["V"], d["W"], a_hat, X,
-                               None, None, ws, outs["accepted"], outs["out_tok"], outs["n_out"], outs["S_next"],
-                               outs["status"])
-        torch.cuda.synchronize()
+        B.gs_verify_round_configure(q_mode != "copied")
+        try:
+            assert B.gs_verify_round_reads_in_place(pin["q_probs"]) == (q_mode == "in-place")
+            B.gs_verify_round_host(desc, pin["Q"], pin["H"], pin["q_probs"], pin["draft_tok"], pin["u_accept"],
+                                   pin["u_sample"], pin["cu_q"], pin["cu_kv"], d["K"], d["V"], d["W"], a_hat, X,
+                                   None, None, ws, outs["accepted"], outs["out_tok"], outs["n_out"], outs["S_next"],
+                                   outs["status"])
+            torch.cuda.synchronize()
+        finally:
+            B.gs_verify_round_configure(True)
         assert int(outs["status"][0]) == 0
         for k in ("accepted", "out_tok", "n_out", "S_next"):
             assert torch.equal(outs[k], getattr(rnd, k).cpu()), (round_idx, k)
