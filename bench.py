@@ -511,6 +511,9 @@ def measure_config(args, cfg, rank, world, local_rank, steps, warmup, detail):
         in_place = B.gs_verify_round_reads_in_place(pin["q_probs"])
         staged = sum(t.numel() * t.element_size() for k, t in pin.items() if not (in_place and k == "q_probs"))
         pulled = (N * V * 4 + 32 * Gamma) if in_place else 0
+        if in_place:        # ... and the first rows of every server, which the copy engine brings over meanwhile
+            near = B.gs_verify_round_near_rows(desc)
+            staged += int(np.minimum(np.asarray(host["gamma"]), near).sum()) * V * 4
         h2d = staged + pulled
         d2h = sum(t.numel() * t.element_size() for t in outs.values())
 

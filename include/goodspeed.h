@@ -362,7 +362,8 @@ gs_status gs_schedule_host(const double* X, const double* alpha_hat, int N, int 
  * Draft distributions in pinned memory that the device can address (cudaHostAlloc, or cudaHostRegister
  * with the mapped flag) are NOT copied: the acceptance pass needs q(s_j) of the drafted tokens and one
  * row per server (the row of its first rejection), and its kernels read those from the host buffer
- * over the bus -- at most N*V*4 + 32*Gamma bytes instead of Gamma*V*4 (see gs_verify_round_configure).
+ * over the bus -- at most N*V*4 + 32*Gamma bytes instead of Gamma*V*4 (see gs_verify_round_configure);
+ * the first rows of every server are copied meanwhile (gs_verify_round_near_rows) and read on the device.
  * Errors: as the four calls; CUDA if a copy could not be enqueued.
  */
 typedef struct gs_round_desc {
@@ -380,6 +381,11 @@ gs_status gs_verify_round_configure(int read_in_place);
 /* 1 if gs_verify_round_host would read this host buffer of draft distributions in place (it is pinned
  * memory with a device address and in-place reads are on), 0 if it would stage it. */
 int gs_verify_round_reads_in_place(const float* h_q_probs);
+/* Beside the in-place reads the copy engine still brings the FIRST rows of every server's draft
+ * distributions to the device while attention and the LM head run (a rejection is most likely early, and
+ * a row that is already there need not cross the bus when the acceptance pass wants it): this many
+ * positions per server, as many as about 10 MB hold, at most 8 (0 for an invalid descriptor). */
+int gs_verify_round_near_rows(const gs_round_desc* r);
 gs_status gs_verify_round_host(const gs_round_desc* r,
                                const void* h_Q, const void* h_H, const float* h_q_probs,
                                const int32_t* h_draft_tok, const float* h_u_accept, const float* h_u_sample,

@@ -63,6 +63,7 @@ SIGNATURES = {
     "gs_verify_round_workspace": (_sz, [_vp]),
     "gs_verify_round_configure": (_i, [_i]),
     "gs_verify_round_reads_in_place": (_i, [_vp]),
+    "gs_verify_round_near_rows": (_i, [_vp]),
     "gs_verify_round_host": (_i, [_vp] + [_vp] * 8 + [_vp] * 7 + [_vp, _sz] + [_vp] * 5 + [_vp]),
     "gs_launch_count": (C.c_ulonglong, []),
 }
@@ -346,6 +347,10 @@ def gs_verify_round_configure(read_in_place: bool = True):
 def gs_verify_round_reads_in_place(h_q_probs) -> bool:
     """Whether gs_verify_round_host would read this CPU tensor of draft distributions where it lies."""
     return bool(lib().gs_verify_round_reads_in_place(_ptr(h_q_probs, torch.float32, cuda=False)))
+
+
+def gs_verify_round_near_rows(desc: RoundDesc) -> int:
+    return int(lib().gs_verify_round_near_rows(C.byref(desc)))
 
 
 def gs_verify_round_host(desc: RoundDesc, h_Q, h_H, h_q_probs, h_draft_tok, h_u_accept, h_u_sample,

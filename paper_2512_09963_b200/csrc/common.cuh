@@ -153,4 +153,14 @@ GS_DEVINL void warp_argmax(float& m, int& a) {
   }
 }
 
+// The acceptance step as the host-buffer round calls it (spec_accept.cu): like gs_spec_accept /
+// gs_spec_accept_prestats (stats != NULL), but the row of a server's first rejection is read from q_near
+// when its position is below q_near_rows and from q_probs otherwise.
+gs_status spec_accept_near(const float* logits, const float* q_probs, const float* q_near, int q_near_rows,
+                           const int32_t* draft_tok, const int32_t* cu_q, const float* u_accept, const float* u_sample,
+                           float temperature, int N, int Tq, int V, int32_t* accepted, int32_t* out_tok, int32_t* n_out,
+                           float* ratio, float* p_tok, double* alpha_hat, double* X, double eta, double beta,
+                           double alpha_min, double alpha_max, const void* stats, int n_chunk, void* ws,
+                           size_t ws_bytes, int32_t* d_status, void* stream);
+
 }  // namespace gs

@@ -9,6 +9,7 @@
 // device).  Otherwise the distributions travel on a copy stream of the library's own while attention
 // and the LM head run, and an event hands them to the caller's stream before gs_spec_accept.
 #include "common.cuh"
+#include <algorithm>
 
 namespace gs {
 
@@ -87,6 +88,15 @@ static bool desc_ok(const gs_round_desc* r) {
 
 // 1 = read the draft distributions in place where possible (default), 0 = always stage them.
 static int g_round_in_place = 1;
+// Bytes of first draft rows the copy engine brings over beside the in-place reads: about what crosses the
+// bus while the LM head streams its weight (a quarter of a millisecond at 40-50 GB/s).
+constexpr size_t kRoundNearBytes = 10u << 20;
+
+// First draft rows per server that the copy engine brings over beside the in-place reads.
+static int round_near_rows(const gs_round_desc& r) {
+  const size_t layer = (size_t)r.N * (size_t)r.V * 4;               // one position of every server
+  return (int)std::min<size_t>(kRoundNearBytes / layer, (size_t)8);
+}
 
 // The address under which the device can read a host buffer where it lies, or NULL.
 static const float* device_view_of_host(const float* h) {
@@ -107,6 +117,10 @@ extern "C" gs_status gs_verify_round_configure(int read_in_place) {
 
 extern "C" int gs_verify_round_reads_in_place(const float* h_q_probs) {
   return gs::device_view_of_host(h_q_probs) != nullptr ? 1 : 0;
+}
+
+extern "C" int gs_verify_round_near_rows(const gs_round_desc* r) {
+  return gs::desc_ok(r) ? gs::round_near_rows(*r) : 0;
 }
 
 extern "C" size_t gs_verify_round_workspace(const gs_round_desc* r) {
@@ -149,17 +163,9 @@ extern "C" gs_status gs_verify_round_host(const gs_round_desc* r,
   bool ok = h2d(L.Q, h_Q, Tq * r->Hq * r->hd * es) && h2d(L.H, h_H, Tq * r->d * es) &&
             h2d(L.cu_q, h_cu_q, (N + 1) * 4) && h2d(L.cu_kv, h_cu_kv, (N + 1) * 4);
   if (!ok || cudaMemsetAsync(w + L.status, 0, 4, st) != cudaSuccess) return GS_ERR_CUDA;
-  // ... then what only the acceptance pass reads, over the copy stream.  It starts once the caller's
-  // stream has reached this call (the previous round may still be reading the staging area).
   RoundSide* side = round_side();
   if (side == nullptr) return GS_ERR_CUDA;
-  if (cudaEventRecord(side->begin, st) != cudaSuccess || cudaStreamWaitEvent(side->copy, side->begin, 0) != cudaSuccess)
-    return GS_ERR_CUDA;
-  const float* q_in_place = (Gamma > 0) ? device_view_of_host(h_q_probs) : nullptr;
-  ok = h2d_on(side->copy, L.draft_tok, h_draft_tok, Gamma * 4) && h2d_on(side->copy, L.u_accept, h_u_accept, Gamma * 4) &&
-       h2d_on(side->copy, L.u_sample, h_u_sample, N * 4) &&
-       (q_in_place != nullptr || h2d_on(side->copy, L.q_probs, h_q_probs, Gamma * V * 4));
-  if (!ok || cudaEventRecord(side->staged, side->copy) != cudaSuccess) return GS_ERR_CUDA;
+  if (cudaEventRecord(side->begin, st) != cudaSuccess) return GS_ERR_CUDA;
   int32_t* d_status = reinterpret_cast<int32_t*>(w + L.status);
   const int32_t* cu_q = reinterpret_cast<const int32_t*>(w + L.cu_q);
   const int32_t* cu_kv = reinterpret_cast<const int32_t*>(w + L.cu_kv);
@@ -179,6 +185,31 @@ extern "C" gs_status gs_verify_round_host(const gs_round_desc* r,
     s = gs_lm_head_logits(w + L.H, d_W, reinterpret_cast<float*>(w + L.logits), r->Tq, r->d, r->V, r->dt,
                           w + L.ws_head, L.ws_head_bytes, d_status, st);
   if (s != GS_OK) return s;
+  // ... then what only the acceptance pass reads, over the copy stream.  It starts once the caller's
+  // stream has reached this call (the event recorded above: the previous round may still be reading the
+  // staging area).  Enqueued after attention and the LM head, so that the device is already at work while
+  // the host issues these copies.
+  if (cudaStreamWaitEvent(side->copy, side->begin, 0) != cudaSuccess) return GS_ERR_CUDA;
+  const float* q_in_place = (Gamma > 0) ? device_view_of_host(h_q_probs) : nullptr;
+  ok = h2d_on(side->copy, L.draft_tok, h_draft_tok, Gamma * 4) && h2d_on(side->copy, L.u_accept, h_u_accept, Gamma * 4) &&
+       h2d_on(side->copy, L.u_sample, h_u_sample, N * 4);
+  // In place: the copy engine still brings the FIRST rows of every server over while attention and the
+  // LM head run (a rejection is most likely early), as many positions as cross the bus in about the time
+  // the LM head takes whatever the batch; the acceptance kernels read a later row from the host buffer.
+  int near_rows = 0;
+  if (ok && q_in_place != nullptr) {
+    near_rows = round_near_rows(*r);
+    for (int i = 0; ok && near_rows > 0 && i < r->N; ++i) {
+      // a server with inconsistent offsets gets no rows here (the kernels skip and flag it)
+      const long long g0 = (long long)h_cu_q[i] - i, gam = (long long)h_cu_q[i + 1] - h_cu_q[i] - 1;
+      if (g0 < 0 || gam <= 0 || g0 + gam > (long long)Gamma) continue;
+      const size_t rows = (size_t)std::min<long long>(gam, near_rows);
+      ok = h2d_on(side->copy, L.q_probs + (size_t)g0 * V * 4, h_q_probs + (size_t)g0 * V, rows * V * 4);
+    }
+  } else if (ok) {
+    ok = h2d_on(side->copy, L.q_probs, h_q_probs, Gamma * V * 4);
+  }
+  if (!ok || cudaEventRecord(side->staged, side->copy) != cudaSuccess) return GS_ERR_CUDA;
   if (cudaStreamWaitEvent(st, side->staged, 0) != cudaSuccess) return GS_ERR_CUDA;
   const float* lg = reinterpret_cast<const float*>(w + L.logits);
   const float* qp = (q_in_place != nullptr) ? q_in_place : reinterpret_cast<const float*>(w + L.q_probs);
@@ -190,15 +221,16 @@ extern "C" gs_status gs_verify_round_host(const gs_round_desc* r,
   int32_t* o_n = reinterpret_cast<int32_t*>(w + L.n_out);
   float* o_ratio = reinterpret_cast<float*>(w + L.ratio);
   float* o_p = reinterpret_cast<float*>(w + L.p_tok);
+  const float* q_near = reinterpret_cast<const float*>(w + L.q_probs);
   s = GS_ERR_UNSUPPORTED;
   if (have_stats)
-    s = gs_spec_accept_prestats(lg, qp, dtok, cu_q, ua, us, r->temperature, r->N, r->Tq, r->V, o_acc, o_tok, o_n,
-                                o_ratio, o_p, nullptr, d_alpha_hat, d_X, r->eta, r->beta, r->alpha_min, r->alpha_max,
-                                w + L.stats, n_chunk, w + L.ws_acc, L.ws_acc_bytes, d_status, st);
+    s = spec_accept_near(lg, qp, q_near, near_rows, dtok, cu_q, ua, us, r->temperature, r->N, r->Tq, r->V, o_acc, o_tok,
+                         o_n, o_ratio, o_p, d_alpha_hat, d_X, r->eta, r->beta, r->alpha_min, r->alpha_max,
+                         w + L.stats, n_chunk, w + L.ws_acc, L.ws_acc_bytes, d_status, st);
   if (s == GS_ERR_UNSUPPORTED)
-    s = gs_spec_accept(lg, qp, dtok, cu_q, ua, us, r->temperature, r->N, r->Tq, r->V, o_acc, o_tok, o_n, o_ratio, o_p,
-                       nullptr, d_alpha_hat, d_X, r->eta, r->beta, r->alpha_min, r->alpha_max, w + L.ws_acc,
-                       L.ws_acc_bytes, d_status, st);
+    s = spec_accept_near(lg, qp, q_near, near_rows, dtok, cu_q, ua, us, r->temperature, r->N, r->Tq, r->V, o_acc, o_tok,
+                         o_n, o_ratio, o_p, d_alpha_hat, d_X, r->eta, r->beta, r->alpha_min, r->alpha_max,
+                         nullptr, 0, w + L.ws_acc, L.ws_acc_bytes, d_status, st);
   if (s != GS_OK) return s;
   s = gs_schedule(d_X, d_alpha_hat, r->N, r->C, d_s_min, d_s_max, reinterpret_cast<int32_t*>(w + L.S_next),
                   d_status, st);

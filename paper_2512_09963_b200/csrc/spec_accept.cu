@@ -152,7 +152,15 @@ struct SaFinishArgs {
   int32_t* d_status;
   int smem_bytes;
   int stats_from_predecessor;   // the statistics come from the kernel right before this one: read nothing of its output before the wait
+  // Second home of the first draft rows of every server (same layout as q_probs): the row of the first
+  // rejection is read from there when its position is below q_near_rows, from q_probs otherwise.  The
+  // host-buffer round sets it when q_probs is host memory read over the bus and the first rows have been
+  // copied to the device meanwhile; everywhere else q_near == q_probs.
+  const float* q_near; int q_near_rows;
 };
+GS_DEVINL const float* sa_q_row(const SaFinishArgs& A, int g0, int a) {
+  return ((a < A.q_near_rows) ? A.q_near : A.q_probs) + (size_t)(g0 + a) * A.V;
+}
 
 // Mass of element v of the selected row: max(0, p - q) or p, in fp64 from an fp32 exponential.
 GS_DEVINL double elem_mass(float l, float M, float k2, double invZ, bool resid, float q) {
@@ -425,7 +433,7 @@ __global__ void __launch_bounds__(kSaThreads) sa_finish(SaFinishArgs A) {
     return;
   }
   const float* lrow = A.logits + (size_t)row * A.V;
-  const float* qrow = resid ? A.q_probs + (size_t)(g0 + a) * A.V : nullptr;
+  const float* qrow = resid ? sa_q_row(A, g0, a) : nullptr;
 
   // ---- mass of this CTA's chunk of the selected row
   {
@@ -603,7 +611,7 @@ __global__ void __launch_bounds__(kFcThreads, LOADS > 4 ? 1 : 2) sa_finish_clust
   const float4* l4 = reinterpret_cast<const float4*>(A.logits + (size_t)row * A.V + start);
   // ---- this CTA's slice of the draft row -> shared memory (bulk copies, one barrier)
   if (resid && len > 0 && wid == 0) {
-    const char* qsrc = reinterpret_cast<const char*>(A.q_probs + (size_t)(g0 + a) * A.V + start);
+    const char* qsrc = reinterpret_cast<const char*>(sa_q_row(A, g0, a) + start);
     const uint32_t bytes = (uint32_t)len * 4u;
     if (lane == 0) mbar_arrive_expect_tx(bar, bytes);
     __syncwarp();
@@ -768,8 +776,25 @@ static gs_status spec_accept_impl(const float* logits, const float* q_probs, con
                                   double* alpha_hat, double* X, double eta, double beta,
                                   double alpha_min, double alpha_max,
                                   void* ws, size_t ws_bytes, int32_t* d_status, void* stream,
-                                  const ChunkStat* pre_stats, int pre_chunks);
+                                  const ChunkStat* pre_stats, int pre_chunks, const float* q_near = nullptr,
+                                  int q_near_rows = 0);
 }
+
+// The acceptance step of the host-buffer round: q_probs may be host memory that the device reads over
+// the bus, with the first q_near_rows draft rows of every server also present at q_near (device memory,
+// same layout).  stats == NULL runs the statistics pass.
+gs_status gs::spec_accept_near(const float* logits, const float* q_probs, const float* q_near, int q_near_rows,
+                               const int32_t* draft_tok, const int32_t* cu_q, const float* u_accept,
+                               const float* u_sample, float temperature, int N, int Tq, int V, int32_t* accepted,
+                               int32_t* out_tok, int32_t* n_out, float* ratio, float* p_tok, double* alpha_hat,
+                               double* X, double eta, double beta, double alpha_min, double alpha_max,
+                               const void* stats, int n_chunk, void* ws, size_t ws_bytes, int32_t* d_status,
+                               void* stream) {
+  return spec_accept_impl(logits, q_probs, draft_tok, cu_q, u_accept, u_sample, temperature, N, Tq, V, accepted, out_tok,
+                          n_out, ratio, p_tok, nullptr, alpha_hat, X, eta, beta, alpha_min, alpha_max, ws, ws_bytes, d_status,
+                          stream, static_cast<const ChunkStat*>(stats), n_chunk, q_near, q_near_rows);
+}
+
 
 extern "C" gs_status gs_spec_accept(const float* logits, const float* q_probs, const int32_t* draft_tok,
                                     const int32_t* cu_q, const float* u_accept, const float* u_sample,
@@ -808,7 +833,8 @@ static gs_status gs::spec_accept_impl(const float* logits, const float* q_probs,
                                       double* alpha_hat, double* X, double eta, double beta,
                                       double alpha_min, double alpha_max,
                                       void* ws, size_t ws_bytes, int32_t* d_status, void* stream,
-                                      const ChunkStat* pre_stats, int pre_chunks) {
+                                      const ChunkStat* pre_stats, int pre_chunks, const float* q_near,
+                                      int q_near_rows) {
   using namespace gs;
   if (N < 0 || Tq < 0 || V < 0 || !(temperature >= 0.f)) return GS_ERR_INVALID_ARG;
   if (N == 0) return GS_OK;
@@ -826,7 +852,8 @@ static gs_status gs::spec_accept_impl(const float* logits, const float* q_probs,
   const int n_chunk = (V + kSaChunk - 1) / kSaChunk;
   const float k2 = temperature > 0.f ? kLog2e / temperature : 0.f;
   const bool vec = (V % 4 == 0) && (reinterpret_cast<uintptr_t>(logits) % 16 == 0) &&
-                   (q_probs == nullptr || reinterpret_cast<uintptr_t>(q_probs) % 16 == 0);
+                   (q_probs == nullptr || reinterpret_cast<uintptr_t>(q_probs) % 16 == 0) &&
+                   (q_near == nullptr || reinterpret_cast<uintptr_t>(q_near) % 16 == 0);
 
   dim3 g1(n_chunk, Tq);
   if (pre_stats == nullptr &&
@@ -843,6 +870,8 @@ static gs_status gs::spec_accept_impl(const float* logits, const float* q_probs,
   A.alpha_hat = alpha_hat; A.X = X; A.eta = eta; A.beta = beta; A.alpha_min = alpha_min; A.alpha_max = alpha_max;
   A.stats = w.stats; A.tickets = w.tickets; A.mass = w.mass; A.d_status = d_status;
   A.stats_from_predecessor = 0;
+  A.q_near = (q_near != nullptr && q_near_rows > 0) ? q_near : q_probs;
+  A.q_near_rows = (q_near != nullptr && q_near_rows > 0) ? q_near_rows : 0;
   if (pre_stats != nullptr) { A.stats = pre_stats; A.n_chunk = pre_chunks; A.stats_from_predecessor = 1; }
   // rows of one server are bounded by Tq - (N-1); size the dynamic shared memory for that
   const size_t max_rows = (size_t)(Tq - N + 1);
