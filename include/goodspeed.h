@@ -353,11 +353,11 @@ gs_status gs_schedule_host(const double* X, const double* alpha_hat, int N, int 
  * The call enqueues host->device copies, gs_verify_attn, gs_lm_head_logits, gs_spec_accept (with
  * the estimator update), gs_schedule and the device->host copies and returns; the host outputs are
  * valid after the caller synchronises `stream`.  Host buffers must stay untouched until then.
- * The draft distributions, tokens and uniforms (read only by the acceptance pass) are copied on a
- * stream of the library's own (one per device, created on the first call together with two events;
- * make that first call outside any stream capture) while attention and the LM head run on `stream`;
- * `stream` waits for them before gs_spec_accept, and they wait for `stream` to reach this call, so
- * back-to-back rounds on one stream are ordered.  Rounds issued on DIFFERENT streams with the same
+ * The hidden states (read only by the LM head) and the draft distributions, tokens and uniforms (read
+ * only by the acceptance pass) are copied on a stream of the library's own (one per device, created on
+ * the first call together with three events; make that first call outside any stream capture) while
+ * attention and the LM head run on `stream`; `stream` waits for them before the call that reads them,
+ * and they wait for `stream` to reach this call, so back-to-back rounds on one stream are ordered.  Rounds issued on DIFFERENT streams with the same
  * d_ws race, as they would anyway.
  * Draft distributions in pinned memory that the device can address (cudaHostAlloc, or cudaHostRegister
  * with the mapped flag) are NOT copied: the acceptance pass needs q(s_j) of the drafted tokens and one

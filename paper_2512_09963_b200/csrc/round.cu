@@ -60,7 +60,7 @@ static RoundLayout round_layout(const gs_round_desc& r) {
 // One copy stream and two events per device, created on first use and kept for the process.
 struct RoundSide {
   cudaStream_t copy = nullptr;
-  cudaEvent_t begin = nullptr, staged = nullptr;
+  cudaEvent_t begin = nullptr, staged = nullptr, h_ready = nullptr;
   bool ok = false;
 };
 static RoundSide* round_side() {
@@ -71,7 +71,8 @@ static RoundSide* round_side() {
   if (!s.ok) {
     if (cudaStreamCreateWithFlags(&s.copy, cudaStreamNonBlocking) != cudaSuccess ||
         cudaEventCreateWithFlags(&s.begin, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&s.staged, cudaEventDisableTiming) != cudaSuccess) {
+        cudaEventCreateWithFlags(&s.staged, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&s.h_ready, cudaEventDisableTiming) != cudaSuccess) {
       (void)cudaGetLastError();
       return nullptr;
     }
@@ -160,18 +161,22 @@ extern "C" gs_status gs_verify_round_host(const gs_round_desc* r,
   };
   // First what attention and the LM head need, on the caller's stream (copies are served in the
   // order they are issued, so the large one must not be queued ahead of these) ...
-  bool ok = h2d(L.Q, h_Q, Tq * r->Hq * r->hd * es) && h2d(L.H, h_H, Tq * r->d * es) &&
-            h2d(L.cu_q, h_cu_q, (N + 1) * 4) && h2d(L.cu_kv, h_cu_kv, (N + 1) * 4);
+  bool ok = h2d(L.Q, h_Q, Tq * r->Hq * r->hd * es) && h2d(L.cu_q, h_cu_q, (N + 1) * 4) && h2d(L.cu_kv, h_cu_kv, (N + 1) * 4);
   if (!ok || cudaMemsetAsync(w + L.status, 0, 4, st) != cudaSuccess) return GS_ERR_CUDA;
   RoundSide* side = round_side();
   if (side == nullptr) return GS_ERR_CUDA;
   if (cudaEventRecord(side->begin, st) != cudaSuccess) return GS_ERR_CUDA;
+  // The hidden states are the LM head's input only: they cross on the copy stream while attention runs.
+  if (cudaStreamWaitEvent(side->copy, side->begin, 0) != cudaSuccess || !h2d_on(side->copy, L.H, h_H, Tq * r->d * es) ||
+      cudaEventRecord(side->h_ready, side->copy) != cudaSuccess)
+    return GS_ERR_CUDA;
   int32_t* d_status = reinterpret_cast<int32_t*>(w + L.status);
   const int32_t* cu_q = reinterpret_cast<const int32_t*>(w + L.cu_q);
   const int32_t* cu_kv = reinterpret_cast<const int32_t*>(w + L.cu_kv);
   gs_status s = gs_verify_attn(w + L.Q, d_K, d_V, w + L.O, cu_q, cu_kv, r->N, r->Tq, r->total_kv, r->max_kv_len,
                                r->Hq, r->Hkv, r->hd, r->scale, r->dt, w + L.ws_attn, L.ws_attn_bytes, d_status, st);
   if (s != GS_OK) return s;
+  if (cudaStreamWaitEvent(st, side->h_ready, 0) != cudaSuccess) return GS_ERR_CUDA;
   // LM head with the softmax statistics in its epilogue where the shape has that kernel, so that the
   // acceptance step does not read the logits a second time; the plain pair of calls otherwise.
   int n_chunk = 0;
@@ -189,7 +194,6 @@ extern "C" gs_status gs_verify_round_host(const gs_round_desc* r,
   // stream has reached this call (the event recorded above: the previous round may still be reading the
   // staging area).  Enqueued after attention and the LM head, so that the device is already at work while
   // the host issues these copies.
-  if (cudaStreamWaitEvent(side->copy, side->begin, 0) != cudaSuccess) return GS_ERR_CUDA;
   const float* q_in_place = (Gamma > 0) ? device_view_of_host(h_q_probs) : nullptr;
   ok = h2d_on(side->copy, L.draft_tok, h_draft_tok, Gamma * 4) && h2d_on(side->copy, L.u_accept, h_u_accept, Gamma * 4) &&
        h2d_on(side->copy, L.u_sample, h_u_sample, N * 4);
