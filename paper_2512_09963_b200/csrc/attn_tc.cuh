@@ -27,9 +27,10 @@
 // instantiation instead: one thread-block cluster of 2, 4 or 8 CTAs per group, CTA k taking the k-th
 // part of the group's visible tiles, exactly one item per CTA.  Each CTA leaves its unnormalised
 // (O, m, l) rows in its own shared memory (the K/V ring is free by then), the cluster meets at one
-// barrier, and CTA 0 merges the parts through distributed shared memory and stores the rows: no
-// workspace, no tickets, no clearing kernel, and a set-up that finds the CTA's one item with a single
-// round of loads.
+// barrier, and the CTAs that hold a part share the rows out and merge them through distributed shared
+// memory: no workspace, no tickets, no clearing kernel, and a set-up that finds the CTA's one item with a
+// single round of loads.  Batches with more groups than that but no more than SMs run the same
+// instantiation with "clusters" of one CTA (one item per CTA, nothing to merge).
 #pragma once
 #include "common.cuh"
 #include "sm100_ptx.cuh"
