@@ -36,17 +36,18 @@ FALLBACK_HBM_GBS = 6650.0
 ETA, BETA = 0.1, 0.5
 
 # DRAM traffic of the LM-head kernel from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum
-# per launch), keyed by the sha256 of the kernel source it was taken on; a changed kernel reports null.
+# per launch), keyed by the sha256 of the kernel's sources (lm_head_pair.cuh and the PTX wrappers it uses)
+# as they were when it was taken; a changed kernel reports null.
 # cfg2's full launch is within ncu's single-pass size rule only for the launch list, so the counters
 # were taken on a smaller vocabulary and scale with the units processed (see profiles/).
-# small case (V = 32768), the kernel with the statistics epilogue: 336.083 MB read + 3.528 MB written
+# small case (V = 32768), the kernel with the statistics epilogue: 336.082 MB read + 3.510 MB written
 # per launch (part of the logits was still in L2 when the capture ended), times 151936/32768
-NCU_TRAFFIC = {"4722f17fd07b2b8e": {"cfg2": 1574683696}}
+NCU_TRAFFIC = {"76d66cc5d5348fec": {"cfg2": 1574592297}}
 
 
 def _kernel_hash():
     h = hashlib.sha256()
-    for f in ("lm_head.cu", "lm_head_pair.cuh", "sm100_ptx.cuh"):
+    for f in ("lm_head_pair.cuh", "sm100_ptx.cuh"):
         h.update(open(os.path.join(ROOT, "paper_2512_09963_b200", "csrc", f), "rb").read())
     return h.hexdigest()[:16]
 
