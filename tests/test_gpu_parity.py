@@ -705,6 +705,43 @@ def test_verify_round_host_matches_device_path(gamma, q_mode):
         assert torch.equal(a_hat, rnd.alpha_hat) and torch.equal(X, rnd.X)
 
 
+def test_verify_round_host_flags_bad_offsets():
+    """Query offsets that leave a server without a row: the host-buffer round (which reads the offsets on
+    the host to place its copies of the first draft rows) copies nothing for such a server, every kernel
+    skips it, and the device status says GS_ERR_SHAPE; the call after it, with good offsets, is right."""
+    cfg = wl.shrink(wl.CONFIGS["cfg2"], d=256, V=16384, N=2, prefix_scale=0.05, name="host_round_bad")
+    inp = wl.make_step(cfg, gamma=[3, 4])
+    d = to_dev(inp)
+    N, Tq = 2, int(inp["cu_q"][-1])
+    rnd = VerifyRound.for_inputs(d, C=8)
+    rnd.run(d, fused=True)
+    torch.cuda.synchronize()
+    desc = B.RoundDesc(N=N, Tq=Tq, total_kv=d["K"].shape[0], max_kv_len=rnd.max_kv_len, Hq=cfg.Hq, Hkv=cfg.Hkv,
+                       hd=cfg.hd, d=cfg.d, V=cfg.V, C=8, dt=B.GS_BF16, scale=cfg.hd ** -0.5,
+                       temperature=float(inp["tau"]), eta=0.1, beta=0.5, alpha_min=1e-3, alpha_max=0.999)
+    ws = torch.empty(B.gs_verify_round_workspace(desc), dtype=torch.uint8, device=DEV)
+    pin = {k: inp[k].contiguous().pin_memory() for k in
+           ("Q", "H", "q_probs", "draft_tok", "u_accept", "u_sample", "cu_q", "cu_kv")}
+    good_cu = pin["cu_q"].clone()
+    for cu, want_status in (([0, Tq, Tq], 2), (good_cu.tolist(), 0)):
+        pin["cu_q"].copy_(torch.tensor(cu, dtype=torch.int32))
+        outs = {k: torch.full((n,), -9, dtype=torch.int32).pin_memory() for k, n in
+                (("accepted", N), ("out_tok", Tq), ("n_out", N), ("S_next", N), ("status", 1))}
+        a_hat = torch.full((N,), 0.5, dtype=torch.float64, device=DEV)
+        X = torch.ones(N, dtype=torch.float64, device=DEV)
+        B.gs_verify_round_host(desc, pin["Q"], pin["H"], pin["q_probs"], pin["draft_tok"], pin["u_accept"],
+                               pin["u_sample"], pin["cu_q"], pin["cu_kv"], d["K"], d["V"], d["W"], a_hat, X,
+                               None, None, ws, outs["accepted"], outs["out_tok"], outs["n_out"], outs["S_next"],
+                               outs["status"])
+        torch.cuda.synchronize()
+        assert int(outs["status"][0]) == want_status
+        if want_status == 0:
+            for k in ("accepted", "out_tok", "n_out", "S_next"):
+                assert torch.equal(outs[k], getattr(rnd, k).cpu()), k
+        else:
+            assert int(outs["accepted"][1]) == 0 and int(outs["n_out"][1]) == 0
+
+
 # ------------------------------------------------------------------ LM head
 @pytest.mark.parametrize("variant", [2, 1], ids=["cta-pairs", "one-cta"])
 @pytest.mark.parametrize("T,d,V", [(44, 512, 9000), (96, 1024, 4104), (288, 256, 8192), (1, 64, 8), (130, 136, 1000),
