@@ -325,6 +325,22 @@ GS_DEVINL int sa_decide(const SaFinishArgs& A, int i, int r0, int gamma, bool wr
         if (c0s.m > -INFINITY) z += c0s.z * (double)fast_exp2((c0s.m - M) * A.k2);
         if (c1s.m > -INFINITY) z += c1s.z * (double)fast_exp2((c1s.m - M) * A.k2);
       }
+    } else if (A.n_chunk <= 160) {
+      // up to five per lane (the LM head writes one entry per CTA: 148 on this device): one round of loads
+      ChunkStat c[5];
+#pragma unroll
+      for (int k = 0; k < 5; ++k) {
+        c[k].m = -INFINITY; c[k].arg = INT_MAX; c[k].z = 0.0;
+        if (lane + 32 * k < A.n_chunk) c[k] = st[lane + 32 * k];
+      }
+#pragma unroll
+      for (int k = 0; k < 5; ++k) argmax_merge(M, arg, c[k].m, c[k].arg);
+      warp_argmax(M, arg);
+      if (A.tau > 0.f) {
+#pragma unroll
+        for (int k = 0; k < 5; ++k)
+          if (c[k].m > -INFINITY) z += c[k].z * (double)fast_exp2((c[k].m - M) * A.k2);
+      }
     } else {
       for (int cc = lane; cc < A.n_chunk; cc += 32) argmax_merge(M, arg, st[cc].m, st[cc].arg);
       warp_argmax(M, arg);
