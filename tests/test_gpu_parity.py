@@ -553,6 +553,20 @@ def test_attention_many_short_servers():
     pu.assert_close_rel(O, orc.ref_attention(inp["Q"], inp["K"], inp["V"], inp["cu_q"], inp["cu_kv"]), "many servers")
 
 
+def test_attention_more_servers_than_the_offset_cache():
+    """1100 servers: more than the kernel keeps offsets and prefix sums for in shared memory, so the item
+    scheduler finds every item by a walk over the offsets in global memory."""
+    base = wl.shrink(wl.CONFIGS["cfg2"], prefix_scale=0.0, N=1100, name="attn_1100")
+    r = np.random.default_rng(11)
+    gamma = r.integers(0, 3, 1100)
+    prefix = r.integers(0, 24, 1100)
+    prefix[[7, 1099]] = [900, 300]
+    inp = wl.make_attention_inputs(base, gamma, prefix)
+    O, st = run_attn(inp)
+    assert st == 0
+    pu.assert_close_rel(O, orc.ref_attention(inp["Q"], inp["K"], inp["V"], inp["cu_q"], inp["cu_kv"]), "1100 servers")
+
+
 def test_attention_edge_shapes():
     base = wl.shrink(wl.CONFIGS["cfg2"], prefix_scale=0.0, N=4, name="attn_edge")   # prefix 1
     inp = wl.make_attention_inputs(base, np.array([0, 1, 16, 3]), np.array([1, 1, 1, 700]))
