@@ -783,11 +783,12 @@ def test_lm_head_small(T, d, V, variant):
 # ------------------------------------------------------------------ LM head on 4-bit weights
 @pytest.mark.parametrize("T,d,V,group", [(46, 512, 9008, 128), (96, 1024, 4112, 128), (1, 128, 16, 64), (130, 384, 1008, 64),
                                          (256, 256, 2048, 128), (300, 128, 528, 128), (16, 5120, 4096, 128),
-                                         (144, 384, 20000, 128)])
+                                         (144, 384, 20000, 128), (16, 256, 151552, 128), (46, 256, 151936, 64)])
 def test_lm_head_w4_small(T, d, V, group):
     """gs_lm_head_logits_w4 against the oracle's dequantised weight and plain product: ragged vocabulary
-    tails, tiles of one to four units, one and two accumulator buffers, more than 256 rows (two
-    launches), the real model width."""
+    tails, tiles of one to four units (the last two shapes: four units everywhere, and the real vocabulary
+    with three and two), one and two accumulator buffers, more than 256 rows (two launches), both group
+    sizes, the real model width."""
     cfg = wl.shrink(wl.CONFIGS["cfg2"], d=d, V=V, name=f"w4_{T}_{d}_{V}")
     layer = wl.make_w4_layer(cfg, group)
     H = wl.make_hidden(cfg, T)
