@@ -375,7 +375,8 @@ typedef struct gs_round_desc {
 
 size_t gs_verify_round_workspace(const gs_round_desc* r);
 /* Whether gs_verify_round_host may read the draft distributions where they lie (process-wide, not
- * thread-safe; 1 = yes, the default, 0 = always stage them in the workspace).  Results do not depend on it.
+ * thread-safe; 1 = yes, with the first rows of every server copied meanwhile: the default; 2 = yes, and
+ * nothing of them is copied; 0 = always stage them in the workspace).  Results do not depend on it.
  * Errors: INVALID_ARG. */
 gs_status gs_verify_round_configure(int read_in_place);
 /* 1 if gs_verify_round_host would read this host buffer of draft distributions in place (it is pinned

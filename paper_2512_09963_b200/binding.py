@@ -340,8 +340,9 @@ def gs_verify_round_workspace(desc: RoundDesc) -> int:
     return lib().gs_verify_round_workspace(C.byref(desc))
 
 
-def gs_verify_round_configure(read_in_place: bool = True):
-    _check("gs_verify_round_configure", lib().gs_verify_round_configure(1 if read_in_place else 0))
+def gs_verify_round_configure(read_in_place=True):
+    """True / 1: in place with the first rows copied meanwhile (default); 2: in place only; False / 0: copy."""
+    _check("gs_verify_round_configure", lib().gs_verify_round_configure(int(read_in_place)))
 
 
 def gs_verify_round_reads_in_place(h_q_probs) -> bool:

@@ -87,7 +87,8 @@ static bool desc_ok(const gs_round_desc* r) {
 }
 
 
-// 1 = read the draft distributions in place where possible (default), 0 = always stage them.
+// 1 = read the draft distributions in place where possible, with the first rows copied meanwhile (default);
+// 2 = in place, nothing copied; 0 = always stage them.
 static int g_round_in_place = 1;
 // Bytes of first draft rows the copy engine brings over beside the in-place reads: about what crosses the
 // bus while the LM head streams its weight (a quarter of a millisecond at 40-50 GB/s).
@@ -95,6 +96,7 @@ constexpr size_t kRoundNearBytes = 10u << 20;
 
 // First draft rows per server that the copy engine brings over beside the in-place reads.
 static int round_near_rows(const gs_round_desc& r) {
+  if (g_round_in_place == 2) return 0;
   const size_t layer = (size_t)r.N * (size_t)r.V * 4;               // one position of every server
   return (int)std::min<size_t>(kRoundNearBytes / layer, (size_t)8);
 }
@@ -111,7 +113,7 @@ static const float* device_view_of_host(const float* h) {
 }  // namespace gs
 
 extern "C" gs_status gs_verify_round_configure(int read_in_place) {
-  if (read_in_place != 0 && read_in_place != 1) return GS_ERR_INVALID_ARG;
+  if (read_in_place < 0 || read_in_place > 2) return GS_ERR_INVALID_ARG;
   gs::g_round_in_place = read_in_place;
   return GS_OK;
 }

@@ -673,12 +673,13 @@ def test_fused_head_statistics_unsupported_shapes_fall_back():
 
 
 # ------------------------------------------------------------------ the round from host buffers
-@pytest.mark.parametrize("q_mode", ["in-place", "copied", "pageable"])
+@pytest.mark.parametrize("q_mode", ["in-place", "in-place-only", "copied", "pageable"])
 @pytest.mark.parametrize("gamma", [[3, 1, 8, 2, 5, 4, 7, 6], [8, 8, 8, 8, 8, 8, 8, 8]], ids=["44-positions", "72-positions"])
 def test_verify_round_host_matches_device_path(gamma, q_mode):
     """gs_verify_round_host gives what the four calls give on device-resident inputs, whether the
-    acceptance kernels read the pinned draft distributions where they lie (the default), the library
-    copies them on its copy stream while attention and the LM head run (in-place reads switched off),
+    acceptance kernels read the pinned draft distributions where they lie (the default: the first rows of
+    every server are copied meanwhile and read on the device; "in-place-only": every row that is needed
+    crosses the bus inside the acceptance kernel), the library copies them on its copy stream while attention and the LM head run (in-place reads switched off),
     or the buffer is pageable memory, which can only be copied; two rounds back to back with different
     drafts reuse the staging area."""
     cfg = wl.shrink(wl.CONFIGS["cfg2"], d=256, V=16384, prefix_scale=0.1, name="host_round")
@@ -703,9 +704,10 @@ def test_verify_round_host_matches_device_path(gamma, q_mode):
                 (("accepted", N), ("out_tok", Tq), ("n_out", N), ("S_next", N), ("status", 1))}
         a_hat = torch.full((N,), 0.5, dtype=torch.float64, device=DEV)
         X = torch.ones(N, dtype=torch.float64, device=DEV)
-        B.gs_verify_round_configure(q_mode != "copied")
+        B.gs_verify_round_configure({"in-place": 1, "in-place-only": 2, "copied": 0, "pageable": 1}[q_mode])
         try:
-            assert B.gs_verify_round_reads_in_place(pin["q_probs"]) == (q_mode == "in-place")
+            assert B.gs_verify_round_reads_in_place(pin["q_probs"]) == q_mode.startswith("in-place")
+            assert (B.gs_verify_round_near_rows(desc) == 0) == (q_mode == "in-place-only")
             B.gs_verify_round_host(desc, pin["Q"], pin["H"], pin["q_probs"], pin["draft_tok"], pin["u_accept"],
                                    pin["u_sample"], pin["cu_q"], pin["cu_kv"], d["K"], d["V"], d["W"], a_hat, X,
                                    None, None, ws, outs["accepted"], outs["out_tok"], outs["n_out"], outs["S_next"],
