@@ -688,8 +688,16 @@ def test_verify_round_host_matches_device_path(gamma, q_mode):
         d = to_dev(inp)
         N, Tq = cfg.N, int(inp["cu_q"][-1])
         rnd = VerifyRound.for_inputs(d, C=4 * N)
-        rnd.run(d, fused=True)         # the host-buffer round takes the same kernels (statistics from the LM head)
-        torch.cuda.synchronize()
+        # second round of the in-place-only case: the ticket kernel of the acceptance step (which takes no
+        # statistics from the LM head, so both sides run the statistics pass) reads the host rows
+        ticket = (q_mode == "in-place-only" and round_idx == 1)
+        B.gs_spec_accept_select(1 if ticket else 0)
+        try:
+            rnd.run(d, fused=not ticket)   # the host-buffer round takes the same kernels (statistics from the LM head)
+            torch.cuda.synchronize()
+        except Exception:
+            B.gs_spec_accept_select(0)
+            raise
         assert int(rnd.d_status.item()) == 0
         desc = B.RoundDesc(N=N, Tq=Tq, total_kv=d["K"].shape[0], max_kv_len=rnd.max_kv_len, Hq=cfg.Hq, Hkv=cfg.Hkv,
                            hd=cfg.hd, d=cfg.d, V=cfg.V, C=4 * N, dt=B.GS_BF16, scale=cfg.hd ** -0.5,
@@ -715,6 +723,7 @@ def test_verify_round_host_matches_device_path(gamma, q_mode):
             torch.cuda.synchronize()
         finally:
             B.gs_verify_round_configure(True)
+            B.gs_spec_accept_select(0)
         assert int(outs["status"][0]) == 0
         for k in ("accepted", "out_tok", "n_out", "S_next"):
             assert torch.equal(outs[k], getattr(rnd, k).cpu()), (round_idx, k)
